@@ -1,0 +1,226 @@
+"""ctypes/numpy front end of the CPU oracle (TEST INFRASTRUCTURE).
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this module.  It wraps oracle/kv_oracle.cpp, which states what the hot path
+computes (sizing per Eq. "unified", the Beta posterior of Eq. "reuse", and this
+build's readings of the EMA, score, selection, demotion and promotion steps).
+All arrays handed out are live numpy views of the oracle's own state.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+AUTO, MHA, GQA, MQA, MLA = -1, 0, 1, 2, 3
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_UNSUPPORTED_VARIANT = -2
+ERR_K_TOO_LARGE = -3
+ERR_NO_FREE_SLOT = -4
+ERR_BAD_HOST_SLOT = -5
+ERR_HOST_TIER_TOO_SMALL = -6
+ERR_TAGS_EXHAUSTED = -10
+NONE = 0xFFFFFFFF
+HOST_BIT = 0x80000000
+FREE, RESIDENT = 0, 1
+
+
+class Model(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("variant", "n_layers", "n_q_heads", "n_kv_heads", "head_dim",
+                 "d_latent", "d_rope", "dtype_bits")]
+
+
+class PartDesc(C.Structure):
+    _fields_ = [("model", Model), ("block_tokens", C.c_int32), ("reserved", C.c_int32),
+                ("blocks_per_layer", C.c_int64), ("ring_slots", C.c_int64)]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(_build.build())
+        L.okv_size_bytes.restype = C.c_int64
+        L.okv_size_bytes.argtypes = [C.POINTER(Model), C.c_int64, C.c_int32]
+        L.okv_infer_variant.restype = C.c_int32
+        L.okv_infer_variant.argtypes = [C.POINTER(Model)]
+        L.okv_entry_bytes.restype = C.c_int64
+        L.okv_entry_bytes.argtypes = [C.POINTER(Model), C.c_int32]
+        L.okv_max_batch.restype = C.c_int64
+        L.okv_max_batch.argtypes = [C.POINTER(Model), C.c_int64, C.c_int64]
+        L.okv_create.restype = C.c_void_p
+        L.okv_create.argtypes = [C.c_int32, C.POINTER(PartDesc), C.c_float, C.c_float,
+                                 C.c_uint64, C.c_int32]
+        L.okv_destroy.argtypes = [C.c_void_p]
+        L.okv_num_entries.restype = C.c_int64
+        L.okv_num_entries.argtypes = [C.c_void_p]
+        L.okv_array.restype = C.c_void_p
+        L.okv_array.argtypes = [C.c_void_p, C.c_int32]
+        L.okv_part_array.restype = C.c_void_p
+        L.okv_part_array.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+        L.okv_part_info.restype = C.c_int64
+        L.okv_part_info.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+        L.okv_get_stats.argtypes = [C.c_void_p, C.c_void_p]
+        L.okv_next_tag.restype = C.c_uint64
+        L.okv_next_tag.argtypes = [C.c_void_p]
+        L.okv_epoch_score.restype = C.c_int32
+        L.okv_epoch_score.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64]
+        L.okv_select_victims.restype = C.c_int32
+        L.okv_select_victims.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        L.okv_demote.restype = C.c_int32
+        L.okv_demote.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
+        L.okv_promote.restype = C.c_int32
+        L.okv_promote.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_uint64]
+        L.okv_admit.restype = C.c_int64
+        L.okv_admit.argtypes = [C.c_void_p, C.c_uint32, C.c_float, C.c_void_p, C.c_uint64,
+                                C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def model(variant=AUTO, n_layers=1, n_q_heads=0, n_kv_heads=0, head_dim=0, d_latent=0,
+          d_rope=0, dtype_bits=16):
+    return Model(variant, n_layers, n_q_heads, n_kv_heads, head_dim, d_latent, d_rope, dtype_bits)
+
+
+def size_bytes(m, n_tokens, per_layer=True):
+    return lib().okv_size_bytes(C.byref(m), n_tokens, 1 if per_layer else 0)
+
+
+def infer_variant(m):
+    return lib().okv_infer_variant(C.byref(m))
+
+
+def entry_bytes(m, block_tokens):
+    return lib().okv_entry_bytes(C.byref(m), block_tokens)
+
+
+def max_batch(m, budget_bytes, n_max):
+    return lib().okv_max_batch(C.byref(m), budget_bytes, n_max)
+
+
+def _view(ptr, dtype, n):
+    if n == 0 or not ptr:
+        return np.zeros(0, dtype=dtype)
+    buf = (C.c_uint8 * (n * np.dtype(dtype).itemsize)).from_address(ptr)
+    return np.frombuffer(buf, dtype=dtype, count=n)
+
+
+def _ptr(a):
+    return a.ctypes.data_as(C.c_void_p) if a is not None and a.size else None
+
+
+class OraclePool:
+    """One pool of up to four partitions.
+
+    parts: list of dicts {model: Model, block_tokens, blocks_per_layer, ring_slots}.
+    """
+
+    _ARR = {"ema": (0, np.float32), "decay": (1, np.float32), "touch": (2, np.uint32),
+            "last_epoch": (3, np.uint32), "pair": (4, np.uint8), "state": (5, np.uint8),
+            "tag": (6, np.uint32), "score": (7, np.float32)}
+    _PARR = {"slab": (0, np.uint8), "ring": (1, np.uint8), "r_tag": (2, np.uint32),
+             "r_pair": (3, np.uint8), "r_ema": (4, np.float32), "r_decay": (5, np.float32),
+             "r_last_epoch": (6, np.uint32), "r_live": (7, np.uint8)}
+
+    def __init__(self, parts, alpha0=1.0, beta0=1.0, n_tags=None, payload=True):
+        L = lib()
+        arr = (PartDesc * len(parts))()
+        for q, p in enumerate(parts):
+            arr[q] = PartDesc(p["model"], p["block_tokens"], 0, p["blocks_per_layer"],
+                              p["ring_slots"])
+        self.n_parts = len(parts)
+        self._n_tags = int(n_tags) if n_tags is not None else 0
+        self._h = L.okv_create(len(parts), arr, alpha0, beta0, self._n_tags, 1 if payload else 0)
+        if not self._h:
+            raise ValueError("oracle: invalid pool description")
+        self.payload = bool(payload)
+        self.N = L.okv_num_entries(self._h)
+
+    def close(self):
+        if self._h:
+            lib().okv_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    def __getattr__(self, name):
+        if name in OraclePool._ARR:
+            which, dt = OraclePool._ARR[name]
+            return _view(lib().okv_array(self._h, which), dt, self.N)
+        raise AttributeError(name)
+
+    @property
+    def hits(self):
+        return _view(lib().okv_array(self._h, 8), np.uint64, 16)
+
+    @property
+    def misses(self):
+        return _view(lib().okv_array(self._h, 9), np.uint64, 16)
+
+    @property
+    def P(self):
+        return _view(lib().okv_array(self._h, 10), np.float32, 16)
+
+    @property
+    def loc(self):
+        return _view(lib().okv_array(self._h, 11), np.uint32, self._n_tags)
+
+    @property
+    def next_tag(self):
+        return int(lib().okv_next_tag(self._h))
+
+    def info(self, q):
+        L = lib()
+        names = ("base", "n", "entry_bytes", "chunk_bytes", "n_chunks", "H", "R", "cursor")
+        return {n: int(L.okv_part_info(self._h, q, i)) for i, n in enumerate(names)}
+
+    def part_array(self, q, name):
+        which, dt = OraclePool._PARR[name]
+        inf = self.info(q)
+        if name == "slab":
+            n = inf["n"] * inf["entry_bytes"] if self.payload else 0
+        elif name == "ring":
+            n = inf["R"] * inf["entry_bytes"] if self.payload else 0
+        else:
+            n = inf["R"]
+        return _view(lib().okv_part_array(self._h, q, which), dt, n)
+
+    def stats(self):
+        out = np.zeros(8, dtype=np.uint64)
+        lib().okv_get_stats(self._h, _ptr(out))
+        names = ("epochs", "events", "victims", "promoted", "admitted", "bytes_demoted",
+                 "bytes_promoted", "bytes_dropped")
+        return {n: int(v) for n, v in zip(names, out)}
+
+    def epoch_score(self, epoch, ev_entry, ev_hit):
+        ev_entry = np.ascontiguousarray(ev_entry, dtype=np.uint32)
+        ev_hit = np.ascontiguousarray(ev_hit, dtype=np.uint8)
+        assert ev_entry.size == ev_hit.size
+        return lib().okv_epoch_score(self._h, epoch, _ptr(ev_entry), _ptr(ev_hit), ev_entry.size)
+
+    def select_victims(self, k):
+        out = np.zeros(int(k), dtype=np.uint32)
+        rc = lib().okv_select_victims(self._h, int(k), _ptr(out))
+        return rc, out
+
+    def demote(self, victims):
+        victims = np.ascontiguousarray(victims, dtype=np.uint32)
+        return lib().okv_demote(self._h, _ptr(victims), victims.size)
+
+    def promote(self, q, slots):
+        slots = np.ascontiguousarray(slots, dtype=np.uint64)
+        return lib().okv_promote(self._h, q, _ptr(slots), slots.size)
+
+    def admit(self, epoch, decay, new_pairs, new_payload=None):
+        new_pairs = np.ascontiguousarray(new_pairs, dtype=np.uint8)
+        if new_payload is not None:
+            new_payload = np.ascontiguousarray(new_payload, dtype=np.uint8)
+        return int(lib().okv_admit(self._h, epoch, decay, _ptr(new_pairs), new_pairs.size,
+                                   _ptr(new_payload) if new_payload is not None else None))
