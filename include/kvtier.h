@@ -1,0 +1,265 @@
+/* kvtier.h -- C ABI of the per-epoch hot path of a predictive two-tier KV-cache
+ * manager (paged HBM pool above a pinned-host ring), for NVIDIA B200 (sm_100a).
+ *
+ * Operations and where the paper defines them:
+ *   kv_size_bytes      sizing section, Eq. "unified" (B(n) per attention
+ *                      variant) and Eq. "total" (L * B(n))
+ *   kv_epoch_score     Bayesian reuse section, Eq. "reuse" (Beta posterior mean
+ *                      with +1 updates per reuse/miss) and head-granular
+ *                      eviction section (EMA importance per (layer, head))
+ *   kv_select_victims  head-granular eviction section ("lowest ... score")
+ *   kv_demote          six-tier hierarchy section, Tier 1 (pinned host memory,
+ *                      asynchronous DMA on CUDA streams)
+ *   kv_promote         RoPE-aware prefetching section (asynchronous promotion
+ *                      requests from lower tiers)
+ * The paper withholds the EMA recurrence, the way the reuse probability and the
+ * importance are combined, and the organisation of the host tier; the
+ * definitions used here are stated at each function.
+ *
+ * Conventions
+ *   - plain C; every pointer is marked (device), (pinned host) or (host);
+ *   - the caller allocates ALL memory (device, pinned host) and the streams;
+ *     the library allocates no device memory and never synchronises the device;
+ *     GPU work is enqueued on the given streams and results are valid once the
+ *     caller has synchronised them.  Use the same compute and copy streams for
+ *     every call on one pool (or order differing streams yourself);
+ *   - device and pinned pointers must be 16-byte aligned;
+ *   - functions return KV_OK (0) or a negative kv_status; on a negative status
+ *     detected by the host nothing has been enqueued and no state has changed;
+ *   - an entry is one head-granular KV block: physical slot (layer, block, head)
+ *     of a partition, local id (layer*blocks_per_layer + block)*heads + head,
+ *     global id = partition base + local id (partitions are laid end to end in
+ *     the order given).  MLA partitions have heads = 1.
+ */
+#ifndef KVTIER_H
+#define KVTIER_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void* kv_stream_t; /* a cudaStream_t */
+typedef struct kv_pool kv_pool;
+
+typedef enum {
+  KV_OK = 0,
+  KV_ERR_INVALID_ARG = -1,
+  KV_ERR_UNSUPPORTED_VARIANT = -2,
+  KV_ERR_K_TOO_LARGE = -3,         /* k exceeds the number of resident entries */
+  KV_ERR_NO_FREE_SLOT = -4,        /* fewer free HBM slots than entries to promote */
+  KV_ERR_BAD_HOST_SLOT = -5,       /* promote list names a dead, duplicate or out-of-range slot */
+  KV_ERR_HOST_TIER_TOO_SMALL = -6, /* more victims in one call than ring slots */
+  KV_ERR_CUDA = -7,                /* a CUDA call failed; see kv_last_cuda_error */
+  KV_ERR_INTERNAL = -8,            /* a kernel reported an inconsistency (kv_device_status) */
+  KV_ERR_UNIMPLEMENTED = -9,
+  KV_ERR_TAGS_EXHAUSTED = -10      /* admission would exceed n_tags */
+} kv_status;
+
+typedef enum { KV_AUTO = -1, KV_MHA = 0, KV_GQA = 1, KV_MQA = 2, KV_MLA = 3 } kv_variant_t;
+
+/* Entry states and block-table encoding. */
+#define KV_STATE_FREE 0u
+#define KV_STATE_RESIDENT 1u
+#define KV_NONE 0xFFFFFFFFu     /* no tag / block not cached */
+#define KV_LOC_HOST 0x80000000u /* d_loc[tag]: bit 31 set = host ring slot in bits 0..30 */
+
+/* Bits of the device status word (kv_device_status). */
+#define KV_DEV_EVENT_BAD_ID 1u       /* an event named an id >= N */
+#define KV_DEV_EVENT_NOT_RESIDENT 2u /* an event named a FREE entry (event skipped) */
+#define KV_DEV_SELECT_MISMATCH 4u    /* selection wrote a count other than k */
+#define KV_DEV_VICTIM_NOT_RESIDENT 8u
+#define KV_DEV_BAD_INDEX 16u         /* an index was out of range and the access was skipped */
+#define KV_DEV_WAIT_EXPIRED 32u      /* a bounded wait inside a kernel gave up */
+
+typedef struct {
+  int32_t variant;    /* kv_variant_t; KV_AUTO infers it from the fields below */
+  int32_t n_layers;   /* L */
+  int32_t n_q_heads;  /* h (h_q) */
+  int32_t n_kv_heads; /* h_kv */
+  int32_t head_dim;   /* d */
+  int32_t d_latent;   /* MLA latent dimension (0 = not MLA) */
+  int32_t d_rope;     /* MLA RoPE dimension */
+  int32_t dtype_bits; /* precision p in bits: 16 = BF16, 8 = INT8, 4 = INT4 (p = 0.5) */
+} kv_model_desc;
+
+/* Bytes of KV cache for n_tokens tokens (sizing section, Eq. "unified"):
+ *   MHA 2*h*d*p*n, GQA/MQA 2*h_kv*d*p*n, MLA (d_latent+d_rope)*p*n   per layer;
+ * per_layer == 0 multiplies by n_layers (one sequence of Eq. "total").
+ * KV_AUTO: a latent dimension selects MLA, else h_q == h_kv is MHA, h_kv == 1 is
+ * MQA, 1 < h_kv < h_q is GQA (h_q == h_kv == 1 reports MHA; same bytes).
+ * Returns bytes, or a negative kv_status (fields inconsistent with the variant,
+ * or a size that is not a whole number of bytes).  Host only; no CUDA. */
+int64_t kv_size_bytes(const kv_model_desc* model, int64_t n_tokens, int32_t per_layer);
+
+/* The variant kv_size_bytes would use, or a negative kv_status. */
+int32_t kv_infer_variant(const kv_model_desc* model);
+
+/* Bytes of one entry: B(block_tokens) / kv heads (one head's K and V), or
+ * B(block_tokens) for MLA, whose importance matrix collapses to one column.
+ * Must come out a multiple of 16. */
+int64_t kv_entry_bytes(const kv_model_desc* model, int32_t block_tokens);
+
+/* Slab layout of a partition (PagedAttention-style paging, head-major inside a
+ * block so that one head's K and V of a block are each one contiguous chunk):
+ *   MHA/GQA/MQA: [layer][block][K,V][head][token][dim]   two chunks per entry
+ *   MLA:         [layer][block][token][d_latent+d_rope]  one chunk per entry
+ * Ring / staging image of an entry: K chunk then V chunk (or the MLA chunk),
+ * entry_bytes long, entries back to back. */
+typedef struct {
+  kv_model_desc model;
+  int32_t block_tokens;
+  int32_t reserved;
+  int64_t blocks_per_layer;
+  void* d_slab;        /* (device) n_layers*blocks_per_layer*heads*entry_bytes */
+  void* h_ring;        /* (pinned host) ring_slots*entry_bytes */
+  uint64_t ring_slots; /* < 2^31 */
+  void* h_meta;        /* (pinned host, optional, may be NULL) ring_slots records of
+                          kv_slot_meta: metadata of the block last demoted into each slot */
+} kv_partition_desc;
+
+typedef struct {
+  uint32_t tag;
+  uint32_t last_epoch;
+  float ema;
+  float decay;
+  uint32_t pair;
+  uint32_t reserved;
+} kv_slot_meta; /* 24 bytes */
+
+typedef struct {
+  int32_t n_partitions; /* 1..4 */
+  int32_t reserved;
+  kv_partition_desc part[4];
+  /* per-entry state, struct of arrays of length N in global id order (device) */
+  float* d_ema;           /* EMA access score */
+  float* d_decay;         /* EMA decay per entry */
+  uint32_t* d_touch;      /* touches seen in the current epoch */
+  uint32_t* d_last_epoch; /* epoch of the last touch */
+  uint8_t* d_pair;        /* 4*block_type + transition_type, 0..15 */
+  uint8_t* d_state;       /* KV_STATE_* */
+  uint32_t* d_tag;        /* logical handle of the block in the slot, KV_NONE if FREE */
+  float* d_score;         /* eviction score, +inf for FREE entries */
+  /* predictor (device) */
+  uint64_t* d_hits;   /* [16] reuse events per pair  (alpha - alpha0) */
+  uint64_t* d_misses; /* [16] miss events per pair   (beta - beta0) */
+  float* d_P;         /* [16] posterior reuse probability */
+  float alpha0, beta0; /* Beta prior, both > 0 */
+  /* block table (device): d_loc[tag] = entry id, KV_LOC_HOST|ring slot, or KV_NONE */
+  uint32_t* d_loc;
+  uint64_t n_tags;
+  /* two device staging buffers of staging_bytes each */
+  void* d_staging[2];
+  uint64_t staging_bytes;
+  uint64_t max_promote; /* longest promote list this pool will be given */
+  /* scratch of the sizes kv_workspace_bytes reports */
+  void* d_workspace;
+  uint64_t workspace_bytes;
+  void* h_workspace; /* (pinned host) */
+  uint64_t h_workspace_bytes;
+} kv_pool_desc;
+
+/* Scratch sizes for a pool description (pointer fields are ignored). */
+int32_t kv_workspace_bytes(const kv_pool_desc* desc, uint64_t* dev_bytes, uint64_t* host_bytes);
+
+/* Validates and copies the description, creates the library's CUDA events, and
+ * enqueues on `stream` the initialisation of all state: every entry FREE, every
+ * ring slot dead, counters zero, d_P = alpha0/(alpha0+beta0), d_loc = KV_NONE.
+ * The pool must be destroyed before the caller frees the memory it was given. */
+int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** out);
+int32_t kv_pool_destroy(kv_pool* pool);
+
+/* One epoch of scoring over every entry, update-then-decide:
+ *  1. each event e (entry id d_ev_entry[e], flag d_ev_hit[e]) adds one to the
+ *     reuse count (flag != 0) or the miss count of the entry's pair -- the
+ *     alpha += 1 / beta += 1 update of the Bayesian reuse section -- and one to
+ *     the entry's touch count;
+ *  2. EMA step of every RESIDENT entry, in binary32 with each operation rounded
+ *     once:  ema = decay*ema + (1-decay)*float(touch);  last_epoch = epoch if
+ *     touched;  touch = 0.  [The paper names an EMA importance per (layer, head)
+ *     but withholds its recurrence; this is the standard one.]
+ *  3. P[p] = (alpha0+hits[p]) / (alpha0+hits[p] + beta0+misses[p])   (Eq. "reuse");
+ *  4. score = P[pair]*ema for RESIDENT entries, +inf for FREE ones.  [The paper
+ *     says in words that placement weighs reuse probability and importance; the
+ *     product is this library's reading.]
+ * d_ev_entry (device, u32[n_events]) and d_ev_hit (device, u8[n_events]) may be
+ * NULL when n_events == 0.  An event on an id >= N or on a FREE entry is
+ * skipped and sets a bit of the device status word. */
+int32_t kv_epoch_score(kv_pool* pool, uint32_t epoch, const uint32_t* d_ev_entry,
+                       const uint8_t* d_ev_hit, uint64_t n_events, kv_stream_t stream);
+
+/* Writes to d_victims (device, u32[k]) the k RESIDENT entries that come first in
+ * the total order (score, global id), in ascending id order: the k lowest
+ * scores, ties broken by lowest (partition, layer, block, head).
+ * KV_ERR_K_TOO_LARGE if k exceeds the resident count (tracked on the host). */
+int32_t kv_select_victims(kv_pool* pool, uint64_t k, uint32_t* d_victims, kv_stream_t stream);
+
+/* Demotes the m entries listed in d_victims (device, ascending distinct ids of
+ * RESIDENT entries, as kv_select_victims writes them): packs their K/V (or MLA)
+ * chunks into the staging buffers in chunks of at most batch_bytes on `compute`,
+ * and copies each chunk to the partition's host ring on `copy`.  The j-th victim
+ * of a partition takes ring slot (cursor + j) mod ring_slots; a live slot that
+ * is overwritten is dropped (d_loc of its tag becomes KV_NONE).  Each victim's
+ * slot becomes FREE, its tag KV_NONE, and d_loc[tag] = KV_LOC_HOST | slot.
+ * With more than one partition the call waits on the host for a 32-byte
+ * readback of the per-partition victim counts (everything enqueued before it on
+ * `compute` must finish first); single-partition pools never wait.
+ * batch_bytes must be in [entry_bytes, staging_bytes - metadata room]; see
+ * kv_max_batch_bytes. */
+int32_t kv_demote(kv_pool* pool, const uint32_t* d_victims, uint64_t m, uint64_t batch_bytes,
+                  kv_stream_t compute, kv_stream_t copy);
+
+/* Promotes the m host ring slots listed in h_host_slots (host, read during the
+ * call; all live and distinct) into partition `partition`: runs of consecutive
+ * slots are copied to staging on `copy`, and the j-th listed entry is scattered
+ * into the j-th lowest FREE slot of the partition on `compute`, with the pair,
+ * EMA, decay, last epoch and tag it had when demoted; the host slot dies. */
+int32_t kv_promote(kv_pool* pool, int32_t partition, const uint64_t* h_host_slots, uint64_t m,
+                   uint64_t batch_bytes, kv_stream_t compute, kv_stream_t copy);
+
+/* Largest batch_bytes the staging buffers allow for a partition. */
+uint64_t kv_max_batch_bytes(const kv_pool* pool, int32_t partition);
+
+/* Harness step, not part of the paper's method: fills every FREE slot, in
+ * ascending id order, with a fresh block: tag = next unused handle, pair =
+ * d_new_pairs[j] for the j-th admitted (device, u8, at least as many as there
+ * are FREE slots), ema 0, the given decay, last_epoch = epoch, touch 0.  With
+ * fill_pattern != 0 the block's bytes are set so that 8-byte word j of the entry
+ * image holds SplitMix64(tag * 2^20 + j).  *n_admitted (host, optional)
+ * receives the count, which the host knows without reading the device. */
+int32_t kv_admit(kv_pool* pool, uint32_t epoch, float decay, const uint8_t* d_new_pairs,
+                 uint64_t n_new_pairs, int32_t fill_pattern, uint64_t* n_admitted,
+                 kv_stream_t stream);
+
+typedef struct {
+  uint64_t epochs, events, victims, promoted, admitted;
+  uint64_t bytes_demoted, bytes_promoted, bytes_dropped;
+  uint64_t n_entries, n_free;
+} kv_stats;
+
+/* Host-side counters, kept eagerly at call time. */
+int32_t kv_get_stats(const kv_pool* pool, kv_stats* out);
+
+/* Host-side view of a partition's ring: cursor, and (optional) one byte per ring
+ * slot, 1 = live.  h_live (host) must hold ring_slots bytes if not NULL. */
+int32_t kv_ring_query(const kv_pool* pool, int32_t partition, uint64_t* cursor, uint64_t* n_live,
+                      uint8_t* h_live);
+
+/* Number of victims per partition of the last kv_demote (host, 4 values). */
+int32_t kv_last_demote_counts(const kv_pool* pool, uint64_t* counts4);
+
+/* Reads and clears the device status word (KV_DEV_* bits).  This one call
+ * blocks the host until `stream` has drained. */
+int32_t kv_device_status(kv_pool* pool, kv_stream_t stream, uint32_t* status_bits);
+
+/* The last CUDA error code seen by a call on this pool (0 = none). */
+int32_t kv_last_cuda_error(const kv_pool* pool);
+
+const char* kv_status_string(int32_t status);
+const char* kv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVTIER_H */

@@ -1,0 +1,175 @@
+// Scoring kernels: event reduction, Beta posterior, fused EMA + score pass.
+//
+// All binary32 arithmetic uses the explicitly rounded intrinsics (__fmul_rn,
+// __fadd_rn, __fsub_rn, __fdiv_rn), which the compiler never contracts into a
+// fused multiply-add, and denormals are kept (no flush-to-zero), so results
+// are bit-identical to the same operations done one at a time on a CPU.
+#include "kvtier_internal.cuh"
+
+namespace kvt {
+
+// ---- event reduction ---------------------------------------------------------
+// Each event adds one to the (pair, hit) counter of its entry's pair -- the
+// alpha += 1 / beta += 1 update of the Bayesian reuse section -- and one to the
+// entry's touch count.  Counters are integers, so the order of the atomics does
+// not matter.  Lanes of a warp that hit the same counter are merged first
+// (match.any), then a 32-counter shared-memory table per block, then one 64-bit
+// global atomic per non-zero counter per block.
+__global__ void __launch_bounds__(kThreads)
+event_reduce_kernel(const uint32_t* __restrict__ ev_entry, const uint8_t* __restrict__ ev_hit,
+                    uint64_t n_events, const uint8_t* __restrict__ pair,
+                    const uint8_t* __restrict__ state, uint32_t* __restrict__ touch, uint64_t n,
+                    unsigned long long* __restrict__ delta, uint32_t* __restrict__ status) {
+  __shared__ uint32_t s_cnt[32];
+  if (threadIdx.x < 32) s_cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const uint64_t iters = (n_events + stride - 1) / stride;  // same for every thread
+  const unsigned lane = threadIdx.x & 31u;
+  uint32_t bad = 0;
+  for (uint64_t it = 0; it < iters; ++it) {
+    const uint64_t e = it * stride + gtid;
+    uint32_t key = 32;  // 32 = nothing to count
+    if (e < n_events) {
+      const uint32_t i = ev_entry[e];
+      const uint32_t hit = ev_hit[e] != 0;
+      if (i >= n) {
+        bad |= KV_DEV_EVENT_BAD_ID;
+      } else if (state[i] != KV_STATE_RESIDENT) {
+        bad |= KV_DEV_EVENT_NOT_RESIDENT;
+      } else {
+        key = (uint32_t)pair[i] * 2u + hit;
+        atomicAdd(&touch[i], 1u);
+      }
+    }
+    const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
+    if (key < 32 && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_cnt[key], __popc(peers));
+  }
+  if (bad) atomicOr(status, bad);
+  __syncthreads();
+  if (threadIdx.x < 32 && s_cnt[threadIdx.x])
+    atomicAdd(&delta[threadIdx.x], (unsigned long long)s_cnt[threadIdx.x]);
+}
+
+cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit, uint64_t n_events,
+                                const EntryState& st, const Workspace& ws, cudaStream_t s) {
+  if (n_events == 0) return cudaSuccess;
+  uint64_t blocks = (n_events + kThreads - 1) / kThreads;
+  const uint64_t cap = (uint64_t)kSMs * 8;
+  if (blocks > cap) blocks = cap;
+  event_reduce_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(ev_entry, ev_hit, n_events, st.pair,
+                                                            st.state, st.touch, st.n, ws.delta,
+                                                            ws.status);
+  return cudaGetLastError();
+}
+
+// ---- posterior ----------------------------------------------------------------
+// Folds the epoch's counts into the running totals and forms the posterior mean
+// of Eq. "reuse": P = alpha / (alpha + beta) with alpha = alpha0 + hits,
+// beta = beta0 + misses.  The 64-bit counts convert to binary32 with round to
+// nearest even.
+__global__ void posterior_kernel(uint64_t* __restrict__ hits, uint64_t* __restrict__ misses,
+                                 float* __restrict__ P, float alpha0, float beta0,
+                                 unsigned long long* __restrict__ delta) {
+  const unsigned p = threadIdx.x;
+  if (p >= 16) return;
+  const unsigned long long h = hits[p] + delta[2 * p + 1];
+  const unsigned long long m = misses[p] + delta[2 * p];
+  hits[p] = h;
+  misses[p] = m;
+  delta[2 * p] = 0;
+  delta[2 * p + 1] = 0;
+  const float a = __fadd_rn(alpha0, __ull2float_rn(h));
+  const float b = __fadd_rn(beta0, __ull2float_rn(m));
+  P[p] = __fdiv_rn(a, __fadd_rn(a, b));
+}
+
+cudaError_t launch_posterior(uint64_t* hits, uint64_t* misses, float* P, float alpha0, float beta0,
+                             const Workspace& ws, cudaStream_t s) {
+  posterior_kernel<<<1, 32, 0, s>>>(hits, misses, P, alpha0, beta0, ws.delta);
+  return cudaGetLastError();
+}
+
+// ---- fused entry pass ------------------------------------------------------------
+// One step of the per-entry EMA, then the eviction score.
+__device__ __forceinline__ void entry_step(float& ema, float decay, uint32_t touch, uint32_t pair,
+                                           uint32_t state, const float* sP, float& score) {
+  if (state == KV_STATE_RESIDENT) {
+    const float x = __uint2float_rn(touch);
+    const float t1 = __fmul_rn(decay, ema);
+    const float t2 = __fsub_rn(1.0f, decay);
+    const float t3 = __fmul_rn(t2, x);
+    ema = __fadd_rn(t1, t3);
+    score = __fmul_rn(sP[pair & 15u], ema);
+  } else {
+    score = __int_as_float(0x7F800000);  // +inf: not a candidate
+  }
+}
+
+// Four entries per thread and iteration: every array is read and written with
+// 16-byte (or, for the byte arrays, 4-byte) accesses, consecutive threads touch
+// consecutive addresses.  touch and last_epoch are only written where an entry
+// was touched, so an idle pool costs reads of 14 bytes and writes of 8 bytes per
+// entry.
+__global__ void __launch_bounds__(kThreads)
+entry_update_kernel(float* __restrict__ ema, const float* __restrict__ decay,
+                    uint32_t* __restrict__ touch, uint32_t* __restrict__ last_epoch,
+                    const uint8_t* __restrict__ pair, const uint8_t* __restrict__ state,
+                    float* __restrict__ score, const float* __restrict__ P, uint64_t n,
+                    uint32_t epoch) {
+  __shared__ float sP[16];
+  if (threadIdx.x < 16) sP[threadIdx.x] = P[threadIdx.x];
+  __syncthreads();
+  const uint64_t n4 = n / 4;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t v = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; v < n4; v += stride) {
+    float4 e = reinterpret_cast<const float4*>(ema)[v];
+    const float4 d = reinterpret_cast<const float4*>(decay)[v];
+    const uint4 t = reinterpret_cast<const uint4*>(touch)[v];
+    const uchar4 pr = reinterpret_cast<const uchar4*>(pair)[v];
+    const uchar4 st = reinterpret_cast<const uchar4*>(state)[v];
+    float4 sc;
+    entry_step(e.x, d.x, t.x, pr.x, st.x, sP, sc.x);
+    entry_step(e.y, d.y, t.y, pr.y, st.y, sP, sc.y);
+    entry_step(e.z, d.z, t.z, pr.z, st.z, sP, sc.z);
+    entry_step(e.w, d.w, t.w, pr.w, st.w, sP, sc.w);
+    reinterpret_cast<float4*>(ema)[v] = e;
+    reinterpret_cast<float4*>(score)[v] = sc;
+    // touch counts of FREE entries are always zero (events on them are refused)
+    if (t.x | t.y | t.z | t.w) {
+      reinterpret_cast<uint4*>(touch)[v] = make_uint4(0, 0, 0, 0);
+      if (t.x) last_epoch[4 * v + 0] = epoch;
+      if (t.y) last_epoch[4 * v + 1] = epoch;
+      if (t.z) last_epoch[4 * v + 2] = epoch;
+      if (t.w) last_epoch[4 * v + 3] = epoch;
+    }
+  }
+  // ragged tail (n not a multiple of 4)
+  const uint64_t i = n4 * 4 + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    float e = ema[i];
+    float sc;
+    const uint32_t t = touch[i];
+    entry_step(e, decay[i], t, pair[i], state[i], sP, sc);
+    ema[i] = e;
+    score[i] = sc;
+    if (t) {
+      touch[i] = 0;
+      last_epoch[i] = epoch;
+    }
+  }
+}
+
+cudaError_t launch_entry_update(const EntryState& st, const float* P, uint32_t epoch, cudaStream_t s) {
+  if (st.n == 0) return cudaSuccess;
+  uint64_t blocks = (st.n / 4 + kThreads - 1) / kThreads;
+  if (blocks == 0) blocks = 1;
+  const uint64_t cap = (uint64_t)kSMs * 8;
+  if (blocks > cap) blocks = cap;
+  entry_update_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(st.ema, st.decay, st.touch, st.last_epoch,
+                                                            st.pair, st.state, st.score, P, st.n, epoch);
+  return cudaGetLastError();
+}
+
+}  // namespace kvt

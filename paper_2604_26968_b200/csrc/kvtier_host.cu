@@ -1,0 +1,609 @@
+// C ABI of kvtier: argument checking, host-side bookkeeping (ring cursors, live
+// slots, free counts), and the stream/event choreography of demotion and
+// promotion.  Every step of the path itself runs in the kernels of kv_score.cu,
+// kv_select.cu and kv_move.cu.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kvtier_internal.cuh"
+
+using namespace kvt;
+
+namespace {
+
+constexpr uint64_t kAlign = 256;
+inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- sizing (sizing section, Eq. "unified") ---------------------------------------
+int32_t infer_variant(const kv_model_desc& m) {
+  if (m.variant != KV_AUTO) {
+    if (m.variant < KV_MHA || m.variant > KV_MLA) return KV_ERR_UNSUPPORTED_VARIANT;
+    return m.variant;
+  }
+  if (m.d_latent > 0) return KV_MLA;
+  if (m.n_q_heads <= 0 || m.n_kv_heads <= 0) return KV_ERR_INVALID_ARG;
+  if (m.n_q_heads == m.n_kv_heads) return KV_MHA;
+  if (m.n_kv_heads == 1) return KV_MQA;
+  if (m.n_kv_heads < m.n_q_heads) return KV_GQA;
+  return KV_ERR_UNSUPPORTED_VARIANT;
+}
+
+// elements of KV state per token per layer, or a negative status
+int64_t token_elems(const kv_model_desc& m, int32_t variant) {
+  if (variant == KV_MLA) {
+    if (m.d_latent <= 0 || m.d_rope < 0) return KV_ERR_INVALID_ARG;
+    return (int64_t)m.d_latent + (int64_t)m.d_rope;
+  }
+  if (m.head_dim <= 0) return KV_ERR_INVALID_ARG;
+  int64_t heads;
+  if (variant == KV_MHA) {
+    heads = m.n_q_heads;
+  } else {
+    heads = m.n_kv_heads;
+    if (variant == KV_MQA && heads != 1) return KV_ERR_INVALID_ARG;
+  }
+  if (heads <= 0) return KV_ERR_INVALID_ARG;
+  return 2 * heads * (int64_t)m.head_dim;
+}
+
+int64_t kv_heads(const kv_model_desc& m, int32_t variant) {
+  if (variant == KV_MLA) return 1;
+  return variant == KV_MHA ? m.n_q_heads : m.n_kv_heads;
+}
+
+struct PartHost {
+  int32_t variant = 0;
+  uint64_t cursor = 0;
+  uint64_t n_live = 0;
+  uint64_t n_free = 0;
+  std::vector<uint8_t> live;
+  uint8_t* h_ring = nullptr;
+  uint8_t* h_meta = nullptr;
+};
+
+}  // namespace
+
+struct kv_pool {
+  kv_pool_desc desc;
+  int n_parts = 0;
+  PartGeom geom[4];
+  PartHost host[4];
+  uint64_t bases[5] = {0, 0, 0, 0, 0};
+  EntryState st;
+  Workspace ws;
+  uint8_t* staging[2] = {nullptr, nullptr};
+  uint64_t staging_bytes = 0;
+  uint64_t max_promote = 0;
+  uint32_t* h_list[2] = {nullptr, nullptr};
+  uint64_t* h_counts = nullptr;
+  uint32_t* h_status = nullptr;
+  uint64_t next_tag = 0;
+  kv_stats stats;
+  uint64_t last_counts[4] = {0, 0, 0, 0};
+  cudaEvent_t ev_staging_free[2], ev_ready[2], ev_list_copied[2], ev_list_free[2], ev_counts;
+  bool events_made = false;
+  int staging_turn = 0, list_turn = 0;
+  int last_cuda_error = 0;
+};
+
+namespace {
+
+struct Layout {
+  uint64_t delta, hist, sel, status, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
+  uint64_t ring[4][5];
+  uint64_t dev_total;
+  uint64_t h_list[2], h_counts, h_status, host_total;
+  uint32_t n_tiles;
+};
+
+struct Derived {
+  int n_parts;
+  int32_t variant[4];
+  uint64_t heads[4], n[4], entry_bytes[4], chunk_bytes[4], n_chunks[4];
+  uint64_t bases[5];
+  uint64_t N;
+};
+
+int32_t derive(const kv_pool_desc* d, Derived* out) {
+  if (!d || d->n_partitions < 1 || d->n_partitions > 4) return KV_ERR_INVALID_ARG;
+  out->n_parts = d->n_partitions;
+  uint64_t base = 0;
+  for (int q = 0; q < d->n_partitions; ++q) {
+    const kv_partition_desc& p = d->part[q];
+    const int32_t v = infer_variant(p.model);
+    if (v < 0) return v;
+    const int64_t eb = kv_entry_bytes(&p.model, p.block_tokens);
+    if (eb < 0) return (int32_t)eb;
+    if (p.model.n_layers <= 0 || p.blocks_per_layer <= 0) return KV_ERR_INVALID_ARG;
+    if (p.ring_slots >= 0x80000000ull) return KV_ERR_INVALID_ARG;
+    out->variant[q] = v;
+    out->heads[q] = (uint64_t)kv_heads(p.model, v);
+    out->n_chunks[q] = (v == KV_MLA) ? 1 : 2;
+    out->entry_bytes[q] = (uint64_t)eb;
+    out->chunk_bytes[q] = (uint64_t)eb / out->n_chunks[q];
+    if (out->chunk_bytes[q] % 16 != 0 || (uint64_t)eb >= (1ull << 23)) return KV_ERR_INVALID_ARG;
+    out->n[q] = (uint64_t)p.model.n_layers * (uint64_t)p.blocks_per_layer * out->heads[q];
+    out->bases[q] = base;
+    base += out->n[q];
+  }
+  for (int q = d->n_partitions; q <= 4; ++q) out->bases[q] = base;
+  if (base == 0 || base >= 0x80000000ull) return KV_ERR_INVALID_ARG;  // ids must fit 31 bits
+  out->N = base;
+  return KV_OK;
+}
+
+void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
+  uint64_t o = 0;
+  auto take = [&o](uint64_t bytes) { uint64_t at = o; o = align_up(o + bytes, kAlign); return at; };
+  L->n_tiles = (uint32_t)((g.N + kTileEntries - 1) / kTileEntries + 2);
+  L->delta = take(32 * 8);
+  L->hist = take(3 * kHistBins * 4);
+  L->sel = take(sizeof(SelectScalars));
+  L->status = take(4);
+  L->part_counts = take(4 * 8);
+  L->tile_counts = take((uint64_t)L->n_tiles * 8);
+  L->tile_offsets = take((uint64_t)L->n_tiles * 8);
+  L->free_list = take(g.N * 4);
+  L->slot_list[0] = take(d->max_promote * 4);
+  L->slot_list[1] = take(d->max_promote * 4);
+  for (int q = 0; q < g.n_parts; ++q) {
+    const uint64_t R = d->part[q].ring_slots;
+    for (int a = 0; a < 4; ++a) L->ring[q][a] = take(R * 4);
+    L->ring[q][4] = take(R);
+  }
+  L->dev_total = o;
+  uint64_t h = 0;
+  auto htake = [&h](uint64_t bytes) { uint64_t at = h; h = align_up(h + bytes, kAlign); return at; };
+  L->h_list[0] = htake(d->max_promote * 4);
+  L->h_list[1] = htake(d->max_promote * 4);
+  L->h_counts = htake(4 * 8);
+  L->h_status = htake(4);
+  L->host_total = h;
+}
+
+inline cudaStream_t S(kv_stream_t s) { return static_cast<cudaStream_t>(s); }
+
+int32_t cuda_fail(kv_pool* p, cudaError_t e) {
+  p->last_cuda_error = (int)e;
+  return KV_ERR_CUDA;
+}
+
+#define KV_CUDA(pool, call)                          \
+  do {                                               \
+    cudaError_t e__ = (call);                        \
+    if (e__ != cudaSuccess) return cuda_fail(pool, e__); \
+  } while (0)
+
+// entries of one chunk: payload plus (optional) metadata records must fit a staging buffer
+uint64_t entries_per_batch(const kv_pool* p, int q, uint64_t batch_bytes) {
+  const uint64_t eb = p->geom[q].entry_bytes;
+  const uint64_t meta = p->host[q].h_meta ? sizeof(kv_slot_meta) : 0;
+  const uint64_t by_batch = batch_bytes / eb;
+  const uint64_t by_staging = (p->staging_bytes >= 16 ? p->staging_bytes - 16 : 0) / (eb + meta);
+  return by_batch < by_staging ? by_batch : by_staging;
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t kv_size_bytes(const kv_model_desc* model, int64_t n_tokens, int32_t per_layer) {
+  if (!model || n_tokens < 0 || model->dtype_bits <= 0) return KV_ERR_INVALID_ARG;
+  if (!per_layer && model->n_layers <= 0) return KV_ERR_INVALID_ARG;
+  const int32_t v = infer_variant(*model);
+  if (v < 0) return v;
+  const int64_t elems = token_elems(*model, v);
+  if (elems < 0) return elems;
+  // 128-bit intermediate: n_tokens is caller-chosen
+  const __int128 bits = (__int128)elems * model->dtype_bits * n_tokens;
+  if (bits % 8 != 0) return KV_ERR_INVALID_ARG;
+  __int128 bytes = bits / 8;
+  if (!per_layer) bytes *= model->n_layers;
+  if (bytes > (__int128)INT64_MAX) return KV_ERR_INVALID_ARG;
+  return (int64_t)bytes;
+}
+
+int32_t kv_infer_variant(const kv_model_desc* model) {
+  if (!model) return KV_ERR_INVALID_ARG;
+  return infer_variant(*model);
+}
+
+int64_t kv_entry_bytes(const kv_model_desc* model, int32_t block_tokens) {
+  if (!model || block_tokens <= 0) return KV_ERR_INVALID_ARG;
+  const int64_t b = kv_size_bytes(model, block_tokens, 1);
+  if (b < 0) return b;
+  const int64_t h = kv_heads(*model, infer_variant(*model));
+  if (h <= 0 || b % h != 0) return KV_ERR_INVALID_ARG;
+  const int64_t eb = b / h;
+  if (eb <= 0 || eb % 16 != 0) return KV_ERR_INVALID_ARG;
+  return eb;
+}
+
+int32_t kv_workspace_bytes(const kv_pool_desc* desc, uint64_t* dev_bytes, uint64_t* host_bytes) {
+  Derived g;
+  const int32_t rc = derive(desc, &g);
+  if (rc != KV_OK) return rc;
+  Layout L;
+  make_layout(desc, g, &L);
+  if (dev_bytes) *dev_bytes = L.dev_total;
+  if (host_bytes) *host_bytes = L.host_total;
+  return KV_OK;
+}
+
+int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** out) {
+  if (!out) return KV_ERR_INVALID_ARG;
+  *out = nullptr;
+  Derived g;
+  const int32_t rc = derive(desc, &g);
+  if (rc != KV_OK) return rc;
+  if (!(desc->alpha0 > 0.0f) || !(desc->beta0 > 0.0f)) return KV_ERR_INVALID_ARG;
+  const void* need[] = {desc->d_ema, desc->d_decay, desc->d_touch, desc->d_last_epoch, desc->d_pair,
+                        desc->d_state, desc->d_tag, desc->d_score, desc->d_hits, desc->d_misses,
+                        desc->d_P, desc->d_staging[0], desc->d_staging[1], desc->d_workspace,
+                        desc->h_workspace};
+  for (const void* p : need)
+    if (!p || !aligned16(p)) return KV_ERR_INVALID_ARG;
+  if (desc->n_tags > 0 && (!desc->d_loc || !aligned16(desc->d_loc))) return KV_ERR_INVALID_ARG;
+  if (desc->n_tags >= 0xFFFFFFFFull) return KV_ERR_INVALID_ARG;
+  for (int q = 0; q < g.n_parts; ++q) {
+    const kv_partition_desc& p = desc->part[q];
+    if (!p.d_slab || !aligned16(p.d_slab)) return KV_ERR_INVALID_ARG;
+    if (p.ring_slots > 0 && (!p.h_ring || !aligned16(p.h_ring))) return KV_ERR_INVALID_ARG;
+    if (p.h_meta && !aligned16(p.h_meta)) return KV_ERR_INVALID_ARG;
+    if (desc->staging_bytes < g.entry_bytes[q] + 64) return KV_ERR_INVALID_ARG;
+  }
+  Layout L;
+  make_layout(desc, g, &L);
+  if (desc->workspace_bytes < L.dev_total || desc->h_workspace_bytes < L.host_total)
+    return KV_ERR_INVALID_ARG;
+
+  kv_pool* p = new (std::nothrow) kv_pool();
+  if (!p) return KV_ERR_INVALID_ARG;
+  p->desc = *desc;
+  p->n_parts = g.n_parts;
+  std::memset(&p->stats, 0, sizeof(p->stats));
+  for (int q = 0; q <= 4; ++q) p->bases[q] = g.bases[q];
+  uint8_t* w = static_cast<uint8_t*>(desc->d_workspace);
+  p->ws.delta = reinterpret_cast<unsigned long long*>(w + L.delta);
+  p->ws.hist = reinterpret_cast<uint32_t*>(w + L.hist);
+  p->ws.sel = reinterpret_cast<SelectScalars*>(w + L.sel);
+  p->ws.status = reinterpret_cast<uint32_t*>(w + L.status);
+  p->ws.part_counts = reinterpret_cast<unsigned long long*>(w + L.part_counts);
+  p->ws.tile_counts = reinterpret_cast<uint2*>(w + L.tile_counts);
+  p->ws.tile_offsets = reinterpret_cast<uint2*>(w + L.tile_offsets);
+  p->ws.free_list = reinterpret_cast<uint32_t*>(w + L.free_list);
+  p->ws.slot_list[0] = reinterpret_cast<uint32_t*>(w + L.slot_list[0]);
+  p->ws.slot_list[1] = reinterpret_cast<uint32_t*>(w + L.slot_list[1]);
+  p->ws.n_tiles = L.n_tiles;
+  uint8_t* hw = static_cast<uint8_t*>(desc->h_workspace);
+  p->h_list[0] = reinterpret_cast<uint32_t*>(hw + L.h_list[0]);
+  p->h_list[1] = reinterpret_cast<uint32_t*>(hw + L.h_list[1]);
+  p->h_counts = reinterpret_cast<uint64_t*>(hw + L.h_counts);
+  p->h_status = reinterpret_cast<uint32_t*>(hw + L.h_status);
+  p->st = EntryState{desc->d_ema, desc->d_decay, desc->d_touch, desc->d_last_epoch, desc->d_pair,
+                     desc->d_state, desc->d_tag, desc->d_score, g.N};
+  for (int q = 0; q < g.n_parts; ++q) {
+    PartGeom& pg = p->geom[q];
+    pg.slab = static_cast<uint8_t*>(desc->part[q].d_slab);
+    pg.base = g.bases[q];
+    pg.n = g.n[q];
+    pg.heads = (uint32_t)g.heads[q];
+    pg.n_chunks = (uint32_t)g.n_chunks[q];
+    pg.chunk_bytes = (uint32_t)g.chunk_bytes[q];
+    pg.entry_bytes = (uint32_t)g.entry_bytes[q];
+    pg.ring_slots = (uint32_t)desc->part[q].ring_slots;
+    pg.r_tag = reinterpret_cast<uint32_t*>(w + L.ring[q][0]);
+    pg.r_last_epoch = reinterpret_cast<uint32_t*>(w + L.ring[q][1]);
+    pg.r_ema = reinterpret_cast<float*>(w + L.ring[q][2]);
+    pg.r_decay = reinterpret_cast<float*>(w + L.ring[q][3]);
+    pg.r_pair = w + L.ring[q][4];
+    PartHost& ph = p->host[q];
+    ph.variant = g.variant[q];
+    ph.n_free = g.n[q];
+    ph.live.assign((size_t)desc->part[q].ring_slots, 0);
+    ph.h_ring = static_cast<uint8_t*>(desc->part[q].h_ring);
+    ph.h_meta = static_cast<uint8_t*>(desc->part[q].h_meta);
+  }
+  p->staging[0] = static_cast<uint8_t*>(desc->d_staging[0]);
+  p->staging[1] = static_cast<uint8_t*>(desc->d_staging[1]);
+  p->staging_bytes = desc->staging_bytes;
+  p->max_promote = desc->max_promote;
+  p->stats.n_entries = g.N;
+  p->stats.n_free = g.N;
+
+  cudaEvent_t* evs[] = {&p->ev_staging_free[0], &p->ev_staging_free[1], &p->ev_ready[0], &p->ev_ready[1],
+                        &p->ev_list_copied[0], &p->ev_list_copied[1], &p->ev_list_free[0],
+                        &p->ev_list_free[1], &p->ev_counts};
+  int made = 0;
+  cudaError_t e = cudaSuccess;
+  for (cudaEvent_t* ev : evs) {
+    e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+    if (e != cudaSuccess) break;
+    ++made;
+  }
+  if (e == cudaSuccess) {
+    p->events_made = true;
+    const float p0 = desc->alpha0 / (desc->alpha0 + desc->beta0);
+    e = launch_init(p->st, desc->d_hits, desc->d_misses, desc->d_P, p0, desc->d_loc, desc->n_tags,
+                    p->geom, p->n_parts, p->ws, S(stream));
+  }
+  if (e != cudaSuccess) {
+    for (int i = 0; i < made; ++i) cudaEventDestroy(*evs[i]);
+    delete p;
+    return KV_ERR_CUDA;
+  }
+  *out = p;
+  return KV_OK;
+}
+
+int32_t kv_pool_destroy(kv_pool* p) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  if (p->events_made) {
+    cudaEvent_t evs[] = {p->ev_staging_free[0], p->ev_staging_free[1], p->ev_ready[0], p->ev_ready[1],
+                         p->ev_list_copied[0], p->ev_list_copied[1], p->ev_list_free[0],
+                         p->ev_list_free[1], p->ev_counts};
+    for (cudaEvent_t ev : evs) cudaEventDestroy(ev);
+  }
+  delete p;
+  return KV_OK;
+}
+
+int32_t kv_epoch_score(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_entry, const uint8_t* d_ev_hit,
+                       uint64_t n_events, kv_stream_t stream) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  if (n_events > 0 && (!d_ev_entry || !d_ev_hit || !aligned16(d_ev_entry) || !aligned16(d_ev_hit)))
+    return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_event_reduce(d_ev_entry, d_ev_hit, n_events, p->st, p->ws, S(stream)));
+  KV_CUDA(p, launch_posterior(p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
+                              p->desc.beta0, p->ws, S(stream)));
+  KV_CUDA(p, launch_entry_update(p->st, p->desc.d_P, epoch, S(stream)));
+  p->stats.epochs += 1;
+  p->stats.events += n_events;
+  return KV_OK;
+}
+
+int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream_t stream) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  if (k > p->stats.n_entries - p->stats.n_free) return KV_ERR_K_TOO_LARGE;
+  if (k == 0) return KV_OK;
+  if (!d_victims || !aligned16(d_victims)) return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_select(p->st, k, d_victims, p->ws, S(stream)));
+  return KV_OK;
+}
+
+uint64_t kv_max_batch_bytes(const kv_pool* p, int32_t q) {
+  if (!p || q < 0 || q >= p->n_parts) return 0;
+  const uint64_t eb = p->geom[q].entry_bytes;
+  return entries_per_batch(p, q, p->staging_bytes) * eb;
+}
+
+int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t batch_bytes,
+                  kv_stream_t compute_, kv_stream_t copy_) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  if (m == 0) {
+    for (int q = 0; q < 4; ++q) p->last_counts[q] = 0;
+    return KV_OK;
+  }
+  if (!d_victims || !aligned16(d_victims) || m > p->stats.n_entries - p->stats.n_free)
+    return KV_ERR_INVALID_ARG;
+  cudaStream_t compute = S(compute_), copy = S(copy_);
+  uint64_t kq[4] = {0, 0, 0, 0};
+  if (p->n_parts == 1) {
+    kq[0] = m;
+  } else {
+    KV_CUDA(p, launch_partition_counts(d_victims, m, p->bases, p->n_parts, p->ws, compute));
+    KV_CUDA(p, cudaMemcpyAsync(p->h_counts, p->ws.part_counts, 4 * sizeof(uint64_t),
+                               cudaMemcpyDeviceToHost, compute));
+    KV_CUDA(p, cudaEventRecord(p->ev_counts, compute));
+    KV_CUDA(p, cudaEventSynchronize(p->ev_counts));
+    uint64_t sum = 0;
+    for (int q = 0; q < p->n_parts; ++q) { kq[q] = p->h_counts[q]; sum += kq[q]; }
+    if (sum != m) return KV_ERR_INTERNAL;  // ids outside every partition
+  }
+  uint64_t per[4] = {0, 0, 0, 0};
+  for (int q = 0; q < p->n_parts; ++q) {
+    if (kq[q] == 0) continue;
+    if (kq[q] > p->geom[q].ring_slots) return KV_ERR_HOST_TIER_TOO_SMALL;
+    if (kq[q] > p->geom[q].n - p->host[q].n_free) return KV_ERR_INVALID_ARG;
+    if (batch_bytes < p->geom[q].entry_bytes) return KV_ERR_INVALID_ARG;
+    per[q] = entries_per_batch(p, q, batch_bytes);
+    if (per[q] == 0 || batch_bytes > p->staging_bytes) return KV_ERR_INVALID_ARG;
+  }
+  uint64_t off = 0;
+  for (int q = 0; q < p->n_parts; ++q) {
+    const PartGeom& g = p->geom[q];
+    PartHost& h = p->host[q];
+    const uint64_t eb = g.entry_bytes, R = g.ring_slots;
+    for (uint64_t c0 = 0; c0 < kq[q]; c0 += per[q]) {
+      const uint64_t cnt = (kq[q] - c0 < per[q]) ? kq[q] - c0 : per[q];
+      const int b = p->staging_turn;
+      p->staging_turn ^= 1;
+      KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_staging_free[b], 0));
+      const uint64_t meta_off = h.h_meta ? align_up(cnt * eb, 16) : ~0ull;
+      const uint64_t slot0 = (h.cursor + c0) % R;
+      KV_CUDA(p, launch_pack(g, p->st, p->desc.d_loc, d_victims + off + c0, cnt, slot0, p->staging[b],
+                             meta_off, p->ws, compute));
+      KV_CUDA(p, cudaEventRecord(p->ev_ready[b], compute));
+      KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_ready[b], 0));
+      const uint64_t first = (cnt < R - slot0) ? cnt : R - slot0;
+      KV_CUDA(p, cudaMemcpyAsync(h.h_ring + slot0 * eb, p->staging[b], first * eb,
+                                 cudaMemcpyDeviceToHost, copy));
+      if (cnt > first)
+        KV_CUDA(p, cudaMemcpyAsync(h.h_ring, p->staging[b] + first * eb, (cnt - first) * eb,
+                                   cudaMemcpyDeviceToHost, copy));
+      if (h.h_meta) {
+        const uint64_t mb = sizeof(kv_slot_meta);
+        KV_CUDA(p, cudaMemcpyAsync(h.h_meta + slot0 * mb, p->staging[b] + meta_off, first * mb,
+                                   cudaMemcpyDeviceToHost, copy));
+        if (cnt > first)
+          KV_CUDA(p, cudaMemcpyAsync(h.h_meta, p->staging[b] + meta_off + first * mb,
+                                     (cnt - first) * mb, cudaMemcpyDeviceToHost, copy));
+      }
+      KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], copy));
+    }
+    // host mirror of the ring: overwritten live slots are dropped
+    for (uint64_t j = 0; j < kq[q]; ++j) {
+      const uint64_t slot = (h.cursor + j) % R;
+      if (h.live[slot]) {
+        p->stats.bytes_dropped += eb;
+      } else {
+        h.live[slot] = 1;
+        h.n_live += 1;
+      }
+    }
+    if (R) h.cursor = (h.cursor + kq[q]) % R;
+    h.n_free += kq[q];
+    p->stats.bytes_demoted += kq[q] * eb;
+    off += kq[q];
+  }
+  for (int q = 0; q < 4; ++q) p->last_counts[q] = kq[q];
+  p->stats.victims += m;
+  p->stats.n_free += m;
+  return KV_OK;
+}
+
+int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, uint64_t batch_bytes,
+                   kv_stream_t compute_, kv_stream_t copy_) {
+  if (!p || q < 0 || q >= p->n_parts) return KV_ERR_INVALID_ARG;
+  if (m == 0) return KV_OK;
+  if (!h_slots || m > p->max_promote) return KV_ERR_INVALID_ARG;
+  const PartGeom& g = p->geom[q];
+  PartHost& h = p->host[q];
+  const uint64_t eb = g.entry_bytes, R = g.ring_slots;
+  if (batch_bytes < eb || batch_bytes > p->staging_bytes) return KV_ERR_INVALID_ARG;
+  // every listed slot live and distinct: mark with 2 while checking, restore on failure
+  uint64_t checked = 0;
+  bool ok = true;
+  for (; checked < m; ++checked) {
+    const uint64_t s = h_slots[checked];
+    if (s >= R || h.live[s] != 1) { ok = false; break; }
+    h.live[s] = 2;
+  }
+  if (!ok || m > h.n_free) {
+    for (uint64_t j = 0; j < checked; ++j) h.live[h_slots[j]] = 1;
+    return ok ? KV_ERR_NO_FREE_SLOT : KV_ERR_BAD_HOST_SLOT;
+  }
+  cudaStream_t compute = S(compute_), copy = S(copy_);
+  const uint64_t per = batch_bytes / eb;
+  const int li = p->list_turn;
+  p->list_turn ^= 1;
+  auto restore = [&]() { for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 1; };
+  cudaError_t e = cudaEventSynchronize(p->ev_list_copied[li]);  // the pinned list buffer is ours again
+  if (e != cudaSuccess) { restore(); return cuda_fail(p, e); }
+  for (uint64_t j = 0; j < m; ++j) p->h_list[li][j] = (uint32_t)h_slots[j];
+  e = cudaStreamWaitEvent(copy, p->ev_list_free[li], 0);  // older kernels are done reading the device list
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(p->ws.slot_list[li], p->h_list[li], m * 4, cudaMemcpyHostToDevice, copy);
+  if (e == cudaSuccess) e = cudaEventRecord(p->ev_list_copied[li], copy);
+  if (e == cudaSuccess) e = launch_free_list(p->st, g.base, g.base + g.n, m, p->ws, compute);
+  if (e != cudaSuccess) { restore(); return cuda_fail(p, e); }
+  for (uint64_t c0 = 0; c0 < m; c0 += per) {
+    const uint64_t cnt = (m - c0 < per) ? m - c0 : per;
+    const int b = p->staging_turn;
+    p->staging_turn ^= 1;
+    KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_staging_free[b], 0));
+    // runs of consecutive ring slots become single copies
+    uint64_t j = 0;
+    while (j < cnt) {
+      const uint64_t s0 = h_slots[c0 + j];
+      uint64_t len = 1;
+      while (j + len < cnt && h_slots[c0 + j + len] == s0 + len) ++len;
+      KV_CUDA(p, cudaMemcpyAsync(p->staging[b] + j * eb, h.h_ring + s0 * eb, len * eb,
+                                 cudaMemcpyHostToDevice, copy));
+      j += len;
+    }
+    KV_CUDA(p, cudaEventRecord(p->ev_ready[b], copy));
+    KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_ready[b], 0));
+    KV_CUDA(p, launch_unpack(g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, p->ws.free_list + c0,
+                             cnt, p->staging[b], p->ws, compute));
+    KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], compute));
+  }
+  KV_CUDA(p, cudaEventRecord(p->ev_list_free[li], compute));
+  for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 0;
+  h.n_live -= m;
+  h.n_free -= m;
+  p->stats.n_free -= m;
+  p->stats.promoted += m;
+  p->stats.bytes_promoted += m * eb;
+  return KV_OK;
+}
+
+int32_t kv_admit(kv_pool* p, uint32_t epoch, float decay, const uint8_t* d_new_pairs, uint64_t n_new_pairs,
+                 int32_t fill_pattern, uint64_t* n_admitted, kv_stream_t stream) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  const uint64_t n_free = p->stats.n_free;
+  if (n_admitted) *n_admitted = 0;
+  if (n_free == 0) return KV_OK;
+  if (!d_new_pairs || n_new_pairs < n_free) return KV_ERR_INVALID_ARG;
+  if (p->next_tag + n_free > p->desc.n_tags) return KV_ERR_TAGS_EXHAUSTED;
+  KV_CUDA(p, launch_free_list(p->st, 0, p->st.n, n_free, p->ws, S(stream)));
+  uint64_t first = 0;
+  for (int q = 0; q < p->n_parts; ++q) {
+    const uint64_t cnt = p->host[q].n_free;
+    KV_CUDA(p, launch_admit(p->geom[q], p->st, p->desc.d_loc, p->ws.free_list, first, cnt, p->next_tag,
+                            d_new_pairs, epoch, decay, fill_pattern, p->ws, S(stream)));
+    first += cnt;
+    p->host[q].n_free = 0;
+  }
+  p->next_tag += n_free;
+  p->stats.admitted += n_free;
+  p->stats.n_free = 0;
+  if (n_admitted) *n_admitted = n_free;
+  return KV_OK;
+}
+
+int32_t kv_get_stats(const kv_pool* p, kv_stats* out) {
+  if (!p || !out) return KV_ERR_INVALID_ARG;
+  *out = p->stats;
+  return KV_OK;
+}
+
+int32_t kv_ring_query(const kv_pool* p, int32_t q, uint64_t* cursor, uint64_t* n_live, uint8_t* h_live) {
+  if (!p || q < 0 || q >= p->n_parts) return KV_ERR_INVALID_ARG;
+  if (cursor) *cursor = p->host[q].cursor;
+  if (n_live) *n_live = p->host[q].n_live;
+  if (h_live && !p->host[q].live.empty())
+    std::memcpy(h_live, p->host[q].live.data(), p->host[q].live.size());
+  return KV_OK;
+}
+
+int32_t kv_last_demote_counts(const kv_pool* p, uint64_t* counts4) {
+  if (!p || !counts4) return KV_ERR_INVALID_ARG;
+  for (int q = 0; q < 4; ++q) counts4[q] = p->last_counts[q];
+  return KV_OK;
+}
+
+int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) {
+  if (!p || !status_bits) return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, cudaMemcpyAsync(p->h_status, p->ws.status, 4, cudaMemcpyDeviceToHost, S(stream)));
+  KV_CUDA(p, cudaMemsetAsync(p->ws.status, 0, 4, S(stream)));
+  KV_CUDA(p, cudaStreamSynchronize(S(stream)));
+  *status_bits = *p->h_status;
+  return KV_OK;
+}
+
+int32_t kv_last_cuda_error(const kv_pool* p) { return p ? p->last_cuda_error : 0; }
+
+const char* kv_status_string(int32_t s) {
+  switch (s) {
+    case KV_OK: return "ok";
+    case KV_ERR_INVALID_ARG: return "invalid argument";
+    case KV_ERR_UNSUPPORTED_VARIANT: return "unsupported attention variant";
+    case KV_ERR_K_TOO_LARGE: return "k exceeds the resident entries";
+    case KV_ERR_NO_FREE_SLOT: return "not enough free HBM slots";
+    case KV_ERR_BAD_HOST_SLOT: return "dead, duplicate or out-of-range host slot";
+    case KV_ERR_HOST_TIER_TOO_SMALL: return "host ring smaller than the victim batch";
+    case KV_ERR_CUDA: return "CUDA error";
+    case KV_ERR_INTERNAL: return "internal inconsistency";
+    case KV_ERR_UNIMPLEMENTED: return "not implemented";
+    case KV_ERR_TAGS_EXHAUSTED: return "block handles exhausted";
+    default: return "unknown status";
+  }
+}
+
+const char* kv_version(void) { return "kvtier 0.1 (sm_100a)"; }
+
+}  // extern "C"

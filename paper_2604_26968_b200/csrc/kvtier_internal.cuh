@@ -1,0 +1,105 @@
+// Internal declarations shared by the kvtier translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvtier.h"
+
+namespace kvt {
+
+constexpr int kSMs = 148;            // B200: 2 dies x 74 SMs
+constexpr int kThreads = 256;
+constexpr uint32_t kRadixBits1 = 11, kRadixBits2 = 11, kRadixBits3 = 10;
+constexpr uint32_t kHistBins = 2048;  // bins of the widest digit
+constexpr uint32_t kTileEntries = 2048;  // entries per compaction tile (256 threads x 8)
+
+// Geometry of one partition, as the kernels need it.
+struct PartGeom {
+  uint8_t* slab;         // device
+  uint64_t base;         // first global id
+  uint64_t n;            // entries
+  uint32_t heads;        // KV heads per block (1 for MLA)
+  uint32_t n_chunks;     // 2 (K, V) or 1 (MLA)
+  uint32_t chunk_bytes;  // bytes of one contiguous chunk in the slab
+  uint32_t entry_bytes;  // n_chunks * chunk_bytes
+  uint32_t ring_slots;
+  // device mirror of per-ring-slot metadata
+  uint32_t* r_tag;
+  uint32_t* r_last_epoch;
+  float* r_ema;
+  float* r_decay;
+  uint8_t* r_pair;
+};
+
+// Per-entry state arrays.
+struct EntryState {
+  float* ema;
+  float* decay;
+  uint32_t* touch;
+  uint32_t* last_epoch;
+  uint8_t* pair;
+  uint8_t* state;
+  uint32_t* tag;
+  float* score;
+  uint64_t n;
+};
+
+// Small block of device scalars used by selection and compaction.
+struct SelectScalars {
+  uint32_t prefix;        // key bits fixed so far
+  uint32_t tau;           // key of the k-th smallest entry
+  unsigned long long k_rem;    // rank still to resolve inside the current bucket
+  unsigned long long need_eq;  // how many entries with key == tau are taken
+  unsigned long long written;  // entries written by the last compaction
+  unsigned long long pad;
+};
+
+struct Workspace {
+  unsigned long long* delta;   // [32] per-epoch (pair, hit) counts: index pair*2+hit
+  uint32_t* hist;              // [3][kHistBins]
+  SelectScalars* sel;
+  uint32_t* status;            // device status word
+  uint2* tile_counts;          // [n_tiles] (less, equal) or (free, 0)
+  uint2* tile_offsets;         // [n_tiles] exclusive prefix of tile_counts
+  uint32_t* free_list;         // [max(N, ..)] ascending ids of FREE entries
+  uint32_t* slot_list[2];      // [max_promote] promote lists (ring slots)
+  unsigned long long* part_counts;  // [4] victims per partition
+  uint32_t n_tiles;
+};
+
+// ---- kv_score.cu ----
+cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit, uint64_t n_events,
+                                const EntryState& st, const Workspace& ws, cudaStream_t s);
+cudaError_t launch_posterior(uint64_t* hits, uint64_t* misses, float* P, float alpha0, float beta0,
+                             const Workspace& ws, cudaStream_t s);
+cudaError_t launch_entry_update(const EntryState& st, const float* P, uint32_t epoch, cudaStream_t s);
+
+// ---- kv_select.cu ----
+cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims, const Workspace& ws,
+                          cudaStream_t s);
+// ascending ids of FREE entries in [lo, hi), at most `limit` of them, into ws.free_list
+cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uint64_t limit,
+                             const Workspace& ws, cudaStream_t s);
+cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const uint64_t* bases5,
+                                    int n_parts, const Workspace& ws, cudaStream_t s);
+
+// ---- kv_move.cu ----
+cudaError_t launch_init(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P, float p0,
+                        uint32_t* loc, uint64_t n_tags, const PartGeom* parts, int n_parts,
+                        const Workspace& ws, cudaStream_t s);
+// packs victims[first .. first+count) of one partition into staging (images back to back)
+// followed, at meta_offset, by kv_slot_meta records; also moves the metadata.
+cudaError_t launch_pack(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* victims,
+                        uint64_t count, uint64_t ring_start, uint8_t* staging, uint64_t meta_offset,
+                        const Workspace& ws, cudaStream_t s);
+// scatters staging images [0, count) into free_list[first_free ..] slots of the partition
+cudaError_t launch_unpack(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
+                          const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
+                          const Workspace& ws, cudaStream_t s);
+// admits free_list[first .. first+count) of one partition
+cudaError_t launch_admit(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* free_ids,
+                         uint64_t first, uint64_t count, uint64_t first_tag, const uint8_t* new_pairs,
+                         uint32_t epoch, float decay, int fill_pattern, const Workspace& ws,
+                         cudaStream_t s);
+
+}  // namespace kvt

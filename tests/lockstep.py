@@ -1,0 +1,147 @@
+"""Runs the CUDA library and the CPU oracle side by side on identical inputs and
+compares every piece of state after every call."""
+import numpy as np
+
+from oracle import kv_oracle as O
+from paper_2604_26968_b200 import workloads as W
+from paper_2604_26968_b200.harness import EpochRunner, INITIAL_EPOCH_KEY
+
+
+def oracle_parts(w):
+    return [dict(model=O.Model(p.variant, p.n_layers, p.n_q_heads, p.n_kv_heads, p.head_dim,
+                               p.d_latent, p.d_rope, p.dtype_bits),
+                 block_tokens=p.block_tokens, blocks_per_layer=p.blocks_per_layer,
+                 ring_slots=p.ring_slots) for p in w.parts]
+
+
+def oracle_admit(w, pool, epoch, key=None):
+    """Admits into every FREE slot of the oracle pool; payload = pattern(tag)."""
+    n_free = int((pool.state == O.FREE).sum())
+    pairs = w.new_pairs(epoch if key is None else key, n_free)
+    payload = None
+    if pool.payload and n_free:
+        imgs, t = [], pool.next_tag
+        for q in range(pool.n_parts):
+            inf = pool.info(q)
+            nf = int((pool.state[inf["base"]:inf["base"] + inf["n"]] == O.FREE).sum())
+            imgs.append(W.pattern_bytes(np.arange(t, t + nf), inf["entry_bytes"]).reshape(-1))
+            t += nf
+        payload = np.concatenate(imgs)
+    got = pool.admit(epoch, w.decay, pairs, payload)
+    assert got == n_free, got
+    return n_free
+
+
+class Lockstep:
+    def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True):
+        self.w = w
+        self.payload = payload
+        self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
+                               fill_pattern=True, host_meta=host_meta)
+        self.ora = O.OraclePool(oracle_parts(w), w.alpha0, w.beta0, n_tags=w.n_tags, payload=payload)
+        oracle_admit(w, self.ora, 0, key=INITIAL_EPOCH_KEY)
+        self.compare_state("initial fill")
+        if payload:
+            self.compare_payload("initial fill")
+
+    # ---- comparisons (bit-exact everywhere) --------------------------------
+    def compare_state(self, where, scores=True):
+        g, o = self.gpu, self.ora
+        st = g.host_array("state")
+        assert np.array_equal(st, o.state), where
+        res = o.state == O.RESIDENT
+        for name in ("pair", "decay", "ema", "last_epoch", "tag", "touch"):
+            a, b = g.host_array(name), getattr(o, name)
+            if name == "tag":
+                assert np.array_equal(a, b), (where, name)
+            else:   # arrays of FREE slots are don't-care on both sides
+                assert np.array_equal(a[res].view(np.uint32 if a.dtype.itemsize == 4 else a.dtype),
+                                      b[res].view(np.uint32 if b.dtype.itemsize == 4 else b.dtype)), (where, name)
+        if scores:
+            assert np.array_equal(g.host_array("score").view(np.uint32), o.score.view(np.uint32)), where
+        assert np.array_equal(g.host_array("hits"), o.hits), where
+        assert np.array_equal(g.host_array("misses"), o.misses), where
+        assert np.array_equal(g.host_array("P").view(np.uint32), o.P.view(np.uint32)), where
+        assert np.array_equal(g.host_array("loc"), o.loc), where
+        assert g.pool.kv_device_status() == 0, where
+
+    def compare_ring(self, where):
+        g, o = self.gpu, self.ora
+        g.pool.sync()
+        for q, p in enumerate(self.w.parts):
+            cur, n_live, live = g.pool.kv_ring_query(q)
+            o_live = o.part_array(q, "r_live")
+            assert cur == o.info(q)["cursor"], where
+            assert np.array_equal(live, o_live), where
+            assert n_live == int(o_live.sum())
+            meta = g.pool.ring_meta(q)
+            lv = o_live != 0
+            # the mirror keeps the record of the last demotion into a slot; compare where the
+            # oracle still holds that block (a promoted slot is dead and its record stale)
+            for name in ("tag", "pair", "last_epoch"):
+                assert np.array_equal(meta[name.replace("r_", "")][lv].astype(np.uint32),
+                                      o.part_array(q, "r_" + name)[lv].astype(np.uint32)), (where, name)
+            for name in ("ema", "decay"):
+                assert np.array_equal(meta[name][lv].view(np.uint32),
+                                      o.part_array(q, "r_" + name)[lv].view(np.uint32)), (where, name)
+            if self.payload:
+                ring = g.pool.rings[q].numpy()[: p.ring_slots * p.entry_bytes].reshape(p.ring_slots, p.entry_bytes)
+                oring = o.part_array(q, "ring").reshape(p.ring_slots, p.entry_bytes)
+                assert np.array_equal(ring[lv], oring[lv]), where
+
+    def compare_payload(self, where):
+        g, o = self.gpu, self.ora
+        g.pool.sync()
+        for q in range(len(self.w.parts)):
+            slab = g.pool.slabs[q].cpu().numpy()
+            oslab = o.part_array(q, "slab")
+            inf = o.info(q)
+            # bytes of FREE slots are don't-care: compare resident entries only
+            res = o.state[inf["base"]:inf["base"] + inf["n"]] == O.RESIDENT
+            H, cb, nc = inf["H"], inf["chunk_bytes"], inf["n_chunks"]
+            lb = inf["n"] // H
+            a = slab.reshape(lb, nc, H, cb)
+            b = oslab.reshape(lb, nc, H, cb)
+            mask = res.reshape(lb, H)
+            for c in range(nc):
+                assert np.array_equal(a[:, c][mask], b[:, c][mask]), (where, q, c)
+
+    # ---- one epoch -----------------------------------------------------------
+    def epoch(self, e, k=None, check_payload=None):
+        w, g, o = self.w, self.gpu, self.ora
+        k = w.k if k is None else k
+        ev_entry, ev_hit = w.events(e, o.pair)
+        d_e, d_h, n = g.stage_events(ev_entry, ev_hit)
+        assert o.epoch_score(e, ev_entry, ev_hit) == O.OK
+        g.check(g.pool.kv_epoch_score(e, d_e, d_h, n), "kv_epoch_score")
+        self.compare_state("epoch %d score" % e)
+        rc, v = o.select_victims(k)
+        assert rc == O.OK
+        g.check(g.pool.kv_select_victims(k, g.victims), "kv_select_victims")
+        g.pool.sync()
+        got = g.victims[:k].cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, v), "epoch %d victims" % e
+        assert o.demote(v) == O.OK
+        g.check(g.pool.kv_demote(g.victims, k, g.batch_bytes), "kv_demote")
+        self.compare_state("epoch %d demote" % e, scores=False)
+        self.compare_ring("epoch %d demote" % e)
+        lists = g.promote_lists(e)
+        for q, lst in enumerate(lists):
+            assert o.promote(q, lst) == O.OK
+            g.check(g.pool.kv_promote(q, lst, g.batch_bytes), "kv_promote")
+        self.compare_state("epoch %d promote" % e, scores=False)
+        self.compare_ring("epoch %d promote" % e)
+        n_free = oracle_admit(w, o, e)
+        g.check(g.admit(e, n_free=n_free), "kv_admit")
+        self.compare_state("epoch %d admit" % e, scores=False)
+        if self.payload and (check_payload is None or check_payload):
+            self.compare_payload("epoch %d" % e)
+        so, sg = o.stats(), g.pool.kv_get_stats()
+        for name in ("epochs", "events", "victims", "promoted", "bytes_demoted", "bytes_promoted",
+                     "bytes_dropped"):
+            assert so[name] == sg[name], (name, so[name], sg[name])
+        return dict(events=n, promoted=sum(len(x) for x in lists), admitted=n_free)
+
+    def close(self):
+        self.gpu.close()
+        self.ora.close()
