@@ -1,0 +1,439 @@
+#!/usr/bin/env python
+"""Benchmark of the per-epoch KV-cache management pass.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one epoch of the whole hot path on one pool: event reduction + EMA +
+posterior + score (kv_epoch_score), k-lowest selection (kv_select_victims),
+pack + D2H to the pinned host ring (kv_demote), H2D + unpack of prefetched
+entries (kv_promote).  Admission of fresh blocks, which keeps the pool full, is
+a harness step and runs untimed between steps, as does an L2 flush.
+
+Prints ONE JSON line.  `value` is KV head-blocks scored + selected per second,
+N / t(kv_epoch_score + kv_select_victims), measured inside full steps; the line
+also carries the whole-step rate, per-phase bandwidths, the roofline of the
+dominant kernel, the host-link peak measured in the same run, and the CPU
+oracle timed on the host cores.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "KV head-blocks scored+selected/s"
+UNIT = "head-blocks/s"
+
+# DRAM traffic per launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum),
+# keyed by kernel; None until a capture of the current kernel exists.
+NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE = {"pack_kernel": None}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="pool 1..5")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrinks blocks per layer")
+    ap.add_argument("--ring-slots", type=int, default=None)
+    ap.add_argument("--batch-mb", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while running."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.lines = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for ln in self.lines:
+            c = [x.strip() for x in ln.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                smax.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                  "sw_power_cap"), c[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def hostlink_probe(torch, dev, nbytes=1 << 30, reps=10):
+    """cudaMemcpyAsync of 1 GiB pinned<->device, best of `reps`, CUDA events."""
+    h = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    d = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    h2 = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    d2 = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    s1, s2 = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    out = {}
+
+    def run(fn, streams):
+        best = 1e30
+        for _ in range(reps):
+            torch.cuda.synchronize(dev)
+            a = [torch.cuda.Event(enable_timing=True) for _ in streams]
+            b = [torch.cuda.Event(enable_timing=True) for _ in streams]
+            for i, s in enumerate(streams):
+                a[i].record(s)
+            fn()
+            for i, s in enumerate(streams):
+                b[i].record(s)
+            torch.cuda.synchronize(dev)
+            best = min(best, max(x.elapsed_time(y) for x, y in zip(a, b)))
+        return best
+
+    def d2h():
+        with torch.cuda.stream(s1):
+            h.copy_(d, non_blocking=True)
+
+    def h2d():
+        with torch.cuda.stream(s1):
+            d.copy_(h, non_blocking=True)
+
+    def both():
+        with torch.cuda.stream(s1):
+            h.copy_(d, non_blocking=True)
+        with torch.cuda.stream(s2):
+            d2.copy_(h2, non_blocking=True)
+
+    out["d2h_gbs"] = nbytes / run(d2h, [s1]) / 1e6
+    out["h2d_gbs"] = nbytes / run(h2d, [s1]) / 1e6
+    out["bidir_gbs_per_dir"] = nbytes / run(both, [s1, s2]) / 1e6
+    out["how"] = "1 GiB pinned<->device copies, best of %d, CUDA events" % reps
+    del h, d, h2, d2
+    return out
+
+
+def oracle_pool(w):
+    from oracle import kv_oracle as O
+    parts = [dict(model=O.Model(p.variant, p.n_layers, p.n_q_heads, p.n_kv_heads, p.head_dim,
+                                p.d_latent, p.d_rope, p.dtype_bits),
+                  block_tokens=p.block_tokens, blocks_per_layer=p.blocks_per_layer,
+                  ring_slots=p.ring_slots) for p in w.parts]
+    return O, O.OraclePool(parts, w.alpha0, w.beta0, n_tags=w.n_tags, payload=False)
+
+
+def oracle_epochs(w, n_epochs, warm=0):
+    """Times the CPU oracle (metadata mode: state, tables and counters, no payload
+    bytes) on the workload.  Returns (seconds in score+select, seconds per full
+    epoch, epochs timed)."""
+    from paper_2604_26968_b200.harness import INITIAL_EPOCH_KEY
+    O, pool = oracle_pool(w)
+    n_free = int((pool.state == O.FREE).sum())
+    pool.admit(0, w.decay, w.new_pairs(INITIAL_EPOCH_KEY, n_free), None)
+    t_ss, t_all, done = 0.0, 0.0, 0
+    for e in range(warm + n_epochs):
+        ev_entry, ev_hit = w.events(e, pool.pair)
+        t0 = time.perf_counter()
+        assert pool.epoch_score(e, ev_entry, ev_hit) == O.OK
+        rc, v = pool.select_victims(w.k)
+        t1 = time.perf_counter()
+        assert rc == O.OK and pool.demote(v) == O.OK
+        t_move = time.perf_counter() - t1
+        for q, p in enumerate(w.parts):
+            inf = pool.info(q)
+            live = pool.part_array(q, "r_live")
+            n_fq = int((pool.state[inf["base"]:inf["base"] + inf["n"]] == O.FREE).sum())
+            m_q = min(int(w.promote_frac * p.n_entries), n_fq, int(live.sum()))
+            lst = w.promote_list(e, q, m_q, inf["cursor"], live)
+            t2 = time.perf_counter()
+            assert pool.promote(q, lst) == O.OK
+            t_move += time.perf_counter() - t2
+        if e >= warm:
+            t_ss += t1 - t0
+            t_all += (t1 - t0) + t_move
+            done += 1
+        n_free = int((pool.state == O.FREE).sum())
+        pool.admit(e, w.decay, w.new_pairs(e, n_free), None)
+    pool.close()
+    return t_ss, t_all, done
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2604_26968_b200 import workloads as W
+    w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots)
+    t_ss, t_all, done = oracle_epochs(w, args.steps, warm=args.warmup)
+    value = w.N * done / t_ss
+    sample = "%d full epochs of pool %d (N=%d) in metadata mode (no payload bytes), 1 thread" % (
+        done, args.config, w.N)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_ss / done,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": w.name, "pool": args.config, "n_entries": w.N,
+                                        "k": w.k, "scale": args.scale},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    import torch.distributed as dist
+    from paper_2604_26968_b200 import workloads as W
+    from paper_2604_26968_b200.harness import EpochRunner
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots)
+    w.seed = w.seed + 1000 * rank     # every rank owns its own pool and trace (weak scaling)
+    link = hostlink_probe(torch, dev) if rank == 0 else None
+    runner = EpochRunner(w, batch_bytes=args.batch_mb << 20, fill_pattern=True, host_meta=True,
+                         device=str(dev))
+    pool = runner.pool
+    pool.kv_timing_enable(True)
+    N, k = w.N, w.k
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    counts = pool.kv_epoch_counts() if world > 1 else None
+
+    def gen_events(e):
+        pair = runner.host_array("pair")
+        return w.events(e, pair)
+
+    def one_step(e, d_e, d_h, n, ev):
+        """Enqueues one full step; ev = (start, selected, demoted, end) CUDA events."""
+        with torch.cuda.stream(pool.compute):
+            ev[0].record(pool.compute)
+        if world > 1:
+            runner.check(pool.kv_epoch_events(d_e, d_h, n), "kv_epoch_events")
+            with torch.cuda.stream(pool.compute):
+                dist.all_reduce(counts)          # 32 int64 counters shared by all pools
+            runner.check(pool.kv_epoch_update(e), "kv_epoch_update")
+        else:
+            runner.check(pool.kv_epoch_score(e, d_e, d_h, n), "kv_epoch_score")
+        runner.check(pool.kv_select_victims(k, runner.victims), "kv_select_victims")
+        ev[1].record(pool.compute)
+        runner.check(pool.kv_demote(runner.victims, k, runner.batch_bytes), "kv_demote")
+        ev[2].record(pool.copy)
+        lists = runner.promote_lists(e)
+        for q, lst in enumerate(lists):
+            runner.check(pool.kv_promote(q, lst, runner.batch_bytes), "kv_promote")
+        ev[3].record(pool.compute)
+        return sum(len(x) for x in lists), lists
+
+    def between_steps(e):
+        runner.check(runner.admit(e), "kv_admit")
+        flush.fill_(e & 0xFF)                     # > L2 capacity: the next step starts cold
+        torch.cuda.synchronize(dev)
+
+    tot = {"ss": 0.0, "dem": 0.0, "pro": 0.0, "all": 0.0, "events": 0, "promoted_bytes": 0}
+    sampler = ClockSampler(local)
+    epoch = 0
+    launches0 = 0
+    for it in range(args.warmup + args.steps):
+        timed = it >= args.warmup
+        if it == args.warmup:
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize(dev)
+            pool.kv_timing_read()                 # discard warm-up launches
+            launches0 = pool.kv_get_stats()["kernel_launches"]
+            sampler.start()
+        ev_entry, ev_hit = gen_events(epoch)
+        d_e, d_h, n = runner.stage_events(ev_entry, ev_hit)
+        torch.cuda.synchronize(dev)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        launches_before = pool.kv_get_stats()["kernel_launches"]
+        m, lists = one_step(epoch, d_e, d_h, n, ev)
+        torch.cuda.synchronize(dev)
+        launches_step = pool.kv_get_stats()["kernel_launches"] - launches_before
+        if timed:
+            tot["ss"] += ev[0].elapsed_time(ev[1])
+            tot["dem"] += ev[1].elapsed_time(ev[2])
+            tot["pro"] += ev[2].elapsed_time(ev[3])
+            tot["all"] += ev[0].elapsed_time(ev[3])
+            tot["events"] += n
+            tot["promoted_bytes"] += sum(len(l) * p.entry_bytes for l, p in zip(lists, w.parts))
+            tot["launches"] = tot.get("launches", 0) + launches_step
+        between_steps(epoch)
+        epoch += 1
+    torch.cuda.synchronize(dev)
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    timing = pool.kv_timing_read()
+    status = pool.kv_device_status()
+    K = args.steps
+    t = torch.tensor([tot["ss"], tot["dem"], tot["pro"], tot["all"]], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ss_ms, dem_ms, pro_ms, all_ms = [float(x) / K for x in t.tolist()]
+
+    # ---- end-to-end: host buffers in, host result out, copies inside the timed region -----
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(2, min(K, 5))
+        h_vict = torch.empty(max(k, 4), dtype=torch.int32, pin_memory=True)
+        wall, h2d_b, d2h_b = 0.0, 0, 0
+        for it in range(e2e_steps):
+            ev_entry, ev_hit = gen_events(epoch)
+            n = int(ev_entry.size)
+            h_e = torch.empty(max(n, 4), dtype=torch.int32, pin_memory=True)
+            h_h = torch.empty(max(n, 16), dtype=torch.uint8, pin_memory=True)
+            h_e[:n] = torch.from_numpy(ev_entry.view(np.int32))
+            h_h[:n] = torch.from_numpy(ev_hit)
+            d_e = torch.empty_like(h_e, device=dev)
+            d_h = torch.empty_like(h_h, device=dev)
+            torch.cuda.synchronize(dev)
+            if world > 1:
+                dist.barrier()
+            t0 = time.perf_counter()
+            with torch.cuda.stream(pool.compute):
+                d_e.copy_(h_e, non_blocking=True)
+                d_h.copy_(h_h, non_blocking=True)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            m, lists = one_step(epoch, d_e, d_h, n, ev)
+            with torch.cuda.stream(pool.compute):
+                h_vict[:max(k, 1)].copy_(runner.victims[:max(k, 1)], non_blocking=True)
+            torch.cuda.synchronize(dev)
+            wall += time.perf_counter() - t0
+            h2d_b += n * 5 + sum(len(l) * (p.entry_bytes + 4) for l, p in zip(lists, w.parts))
+            d2h_b += k * 4 + sum(c * (p.entry_bytes + 24) for c, p in zip(pool.kv_last_demote_counts(), w.parts))
+            between_steps(epoch)
+            epoch += 1
+        tw = torch.tensor([wall], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(tw, op=dist.ReduceOp.MAX)
+        e2e = {"value": N * world * e2e_steps / float(tw.item()), "unit": "head-blocks/s (whole epoch, host in/out)",
+               "h2d_bytes_per_step": h2d_b // e2e_steps, "d2h_bytes_per_step": d2h_b // e2e_steps,
+               "steps": e2e_steps, "ms_per_step": 1e3 * float(tw.item()) / e2e_steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    eb_bytes = sum(c * p.entry_bytes for c, p in zip(pool.kv_last_demote_counts(), w.parts))
+    demoted_per_step = eb_bytes
+    promoted_per_step = tot["promoted_bytes"] / K
+    pack_gbs = 2 * timing["pack_bytes"] / max(timing["pack_ms"], 1e-9) / 1e6
+    unpack_gbs = 2 * timing["unpack_bytes"] / max(timing["unpack_ms"], 1e-9) / 1e6
+    ss_bytes = 39 * N + 5 * (tot["events"] / K) + 4 * k
+    tr = NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE["pack_kernel"]
+    line = {
+        "metric": METRIC, "value": N * world / (ss_ms * 1e-3), "unit": UNIT,
+        "value_definition": "N / t(kv_epoch_score + kv_select_victims), timed with CUDA events inside full steps",
+        "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": all_ms,
+        "whole_step_head_blocks_per_s": N * world / (all_ms * 1e-3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "pool": args.config, "n_entries": N, "k": k,
+                   "events_per_step": tot["events"] // K, "pool_bytes": sum(p.slab_bytes for p in w.parts),
+                   "entry_bytes": [p.entry_bytes for p in w.parts], "batch_bytes": runner.batch_bytes,
+                   "ring_slots": [p.ring_slots for p in w.parts], "scale": args.scale,
+                   "parallelism": "1 pool per GPU" + (", 256-byte all-reduce of pair counters" if world > 1 else ""),
+                   "l2": "256 MiB written between steps (flush) and >1 GB of fresh blocks admitted"},
+        "phases": {
+            "score_select_ms": ss_ms,
+            "score_select_effective_gbs": ss_bytes / (ss_ms * 1e-3) / 1e9,
+            "demote_ms": dem_ms, "demote_gbs": demoted_per_step / (dem_ms * 1e-3) / 1e9,
+            "promote_ms": pro_ms, "promote_gbs": promoted_per_step / max(pro_ms * 1e-3, 1e-12) / 1e9,
+            "pack_kernel_gbs": pack_gbs, "pack_kernel_frac_of_%s_hbm" % peak_kind: pack_gbs / peak,
+            "unpack_kernel_gbs": unpack_gbs, "unpack_kernel_frac_of_%s_hbm" % peak_kind: unpack_gbs / peak,
+            "pack_launches": timing["pack_launches"], "unpack_launches": timing["unpack_launches"],
+        },
+        "hostlink": link,
+        "roofline": {"kernel": "pack_kernel", "bound": "hbm", "achieved": pack_gbs, "peak": peak,
+                     "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": pack_gbs / peak,
+                     "traffic": (tr * timing["pack_bytes"] / max(timing["pack_launches"], 1)) if tr else None,
+                     "algorithmic_bytes_per_launch": 2 * timing["pack_bytes"] / max(timing["pack_launches"], 1)},
+        "clocks": clocks,
+        "gpu_launches": tot.get("launches", 0),
+        "device_status": status,
+    }
+    if link:
+        line["phases"]["demote_frac_of_d2h_link"] = line["phases"]["demote_gbs"] / link["d2h_gbs"]
+        line["phases"]["promote_frac_of_h2d_link"] = line["phases"]["promote_gbs"] / link["h2d_gbs"]
+    if e2e:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline:
+        n_ep = 6
+        t_ss, t_all, done = oracle_epochs(w, n_ep, warm=1)
+        line["cpu_baseline"] = {
+            "value": N * done / t_ss, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "%d epochs of the same pool (N=%d, k=%d) in metadata mode, score+select timed; host has %d cores"
+                      % (done, N, k, os.cpu_count() or 0),
+            "ms_per_epoch_score_select": 1e3 * t_ss / done}
+    print(json.dumps(line))
+    runner.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

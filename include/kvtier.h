@@ -189,6 +189,21 @@ int32_t kv_pool_destroy(kv_pool* pool);
 int32_t kv_epoch_score(kv_pool* pool, uint32_t epoch, const uint32_t* d_ev_entry,
                        const uint8_t* d_ev_hit, uint64_t n_events, kv_stream_t stream);
 
+/* kv_epoch_score in two halves, for pools sharded over several GPUs (each GPU
+ * holds its own entries; only the 16 pair counters are shared, since the
+ * predictor keeps one Beta distribution per pair for the whole system):
+ *   kv_epoch_events  step 1 only: adds this GPU's events to the epoch counters;
+ *   kv_epoch_counts  device address of the 32 epoch counters (u64, index
+ *                    2*pair + hit), to be summed over GPUs in place by the
+ *                    caller's collective (e.g. one NCCL all-reduce of 256 bytes);
+ *   kv_epoch_update  folds the epoch counters into d_hits/d_misses, clears them,
+ *                    and runs steps 2-4.
+ * kv_epoch_score(pool, ...) == kv_epoch_events(...) then kv_epoch_update(...). */
+int32_t kv_epoch_events(kv_pool* pool, const uint32_t* d_ev_entry, const uint8_t* d_ev_hit,
+                        uint64_t n_events, kv_stream_t stream);
+uint64_t* kv_epoch_counts(kv_pool* pool);
+int32_t kv_epoch_update(kv_pool* pool, uint32_t epoch, kv_stream_t stream);
+
 /* Writes to d_victims (device, u32[k]) the k RESIDENT entries that come first in
  * the total order (score, global id), in ascending id order: the k lowest
  * scores, ties broken by lowest (partition, layer, block, head).
@@ -236,6 +251,7 @@ typedef struct {
   uint64_t epochs, events, victims, promoted, admitted;
   uint64_t bytes_demoted, bytes_promoted, bytes_dropped;
   uint64_t n_entries, n_free;
+  uint64_t kernel_launches; /* kernels launched by the library in this process so far */
 } kv_stats;
 
 /* Host-side counters, kept eagerly at call time. */
@@ -252,6 +268,18 @@ int32_t kv_last_demote_counts(const kv_pool* pool, uint64_t* counts4);
 /* Reads and clears the device status word (KV_DEV_* bits).  This one call
  * blocks the host until `stream` has drained. */
 int32_t kv_device_status(kv_pool* pool, kv_stream_t stream, uint32_t* status_bits);
+
+/* Measurement aid (no counterpart in the paper): when enabled, every pack and
+ * unpack kernel launch is bracketed by two timing events on the stream it is
+ * launched on.  kv_timing_read waits for the recorded launches to finish, adds
+ * their durations up, reports the totals since the last read and resets them. */
+typedef struct {
+  double pack_ms, unpack_ms;            /* summed kernel durations */
+  uint64_t pack_launches, unpack_launches;
+  uint64_t pack_bytes, unpack_bytes;    /* payload bytes moved (read + written counted once each) */
+} kv_timing;
+int32_t kv_timing_enable(kv_pool* pool, int32_t on);
+int32_t kv_timing_read(kv_pool* pool, kv_timing* out);
 
 /* The last CUDA error code seen by a call on this pool (0 = none). */
 int32_t kv_last_cuda_error(const kv_pool* pool);

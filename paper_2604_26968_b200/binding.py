@@ -58,7 +58,13 @@ class kv_pool_desc(C.Structure):
 class kv_stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in
                 ("epochs", "events", "victims", "promoted", "admitted", "bytes_demoted",
-                 "bytes_promoted", "bytes_dropped", "n_entries", "n_free")]
+                 "bytes_promoted", "bytes_dropped", "n_entries", "n_free", "kernel_launches")]
+
+
+class kv_timing(C.Structure):
+    _fields_ = [("pack_ms", C.c_double), ("unpack_ms", C.c_double),
+                ("pack_launches", C.c_uint64), ("unpack_launches", C.c_uint64),
+                ("pack_bytes", C.c_uint64), ("unpack_bytes", C.c_uint64)]
 
 
 class kv_slot_meta(C.Structure):
@@ -70,9 +76,11 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
                             ("decay", "<f4"), ("pair", "<u4"), ("reserved", "<u4")])
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
-           "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_select_victims", "kv_demote",
+           "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_events", "kv_epoch_counts",
+           "kv_epoch_update", "kv_select_victims", "kv_demote",
            "kv_promote", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
-           "kv_last_demote_counts", "kv_device_status", "kv_last_cuda_error", "kv_status_string",
+           "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
+           "kv_last_cuda_error", "kv_status_string",
            "kv_version")
 
 _lib = None
@@ -102,6 +110,12 @@ def load():
     L.kv_pool_destroy.argtypes = [vp]
     L.kv_epoch_score.restype = i32
     L.kv_epoch_score.argtypes = [vp, u32, vp, vp, u64, vp]
+    L.kv_epoch_events.restype = i32
+    L.kv_epoch_events.argtypes = [vp, vp, vp, u64, vp]
+    L.kv_epoch_counts.restype = vp
+    L.kv_epoch_counts.argtypes = [vp]
+    L.kv_epoch_update.restype = i32
+    L.kv_epoch_update.argtypes = [vp, u32, vp]
     L.kv_select_victims.restype = i32
     L.kv_select_victims.argtypes = [vp, u64, vp, vp]
     L.kv_demote.restype = i32
@@ -120,6 +134,10 @@ def load():
     L.kv_last_demote_counts.argtypes = [vp, C.POINTER(u64 * 4)]
     L.kv_device_status.restype = i32
     L.kv_device_status.argtypes = [vp, vp, C.POINTER(u32)]
+    L.kv_timing_enable.restype = i32
+    L.kv_timing_enable.argtypes = [vp, i32]
+    L.kv_timing_read.restype = i32
+    L.kv_timing_read.argtypes = [vp, C.POINTER(kv_timing)]
     L.kv_last_cuda_error.restype = i32
     L.kv_last_cuda_error.argtypes = [vp]
     L.kv_status_string.restype = C.c_char_p
@@ -256,6 +274,20 @@ class Pool:
                                        d_ev_entry.data_ptr() if n else None,
                                        d_ev_hit.data_ptr() if n else None, n, _stream_ptr(self.compute))
 
+    def kv_epoch_events(self, d_ev_entry, d_ev_hit, n_events=None):
+        n = int(n_events if n_events is not None else (d_ev_entry.numel() if d_ev_entry is not None else 0))
+        return self.lib.kv_epoch_events(self._h, d_ev_entry.data_ptr() if n else None,
+                                        d_ev_hit.data_ptr() if n else None, n, _stream_ptr(self.compute))
+
+    def kv_epoch_counts(self):
+        """The 32 epoch counters as an int64 tensor aliasing the library's device memory."""
+        addr = self.lib.kv_epoch_counts(self._h)
+        off = addr - self.workspace.data_ptr()
+        return self.workspace[off:off + 256].view(self.torch.int64)
+
+    def kv_epoch_update(self, epoch):
+        return self.lib.kv_epoch_update(self._h, epoch, _stream_ptr(self.compute))
+
     def kv_select_victims(self, k, d_victims):
         return self.lib.kv_select_victims(self._h, int(k), d_victims.data_ptr() if k else None,
                                           _stream_ptr(self.compute))
@@ -306,6 +338,16 @@ class Pool:
         if rc != KV_OK:
             raise KVError(rc, "kv_device_status")
         return bits.value
+
+    def kv_timing_enable(self, on=True):
+        return self.lib.kv_timing_enable(self._h, 1 if on else 0)
+
+    def kv_timing_read(self):
+        t = kv_timing()
+        rc = self.lib.kv_timing_read(self._h, C.byref(t))
+        if rc != KV_OK:
+            raise KVError(rc, "kv_timing_read")
+        return {n: getattr(t, n) for n, _ in kv_timing._fields_}
 
     def ring_meta(self, partition):
         """numpy view of the pinned per-slot metadata mirror (after sync)."""

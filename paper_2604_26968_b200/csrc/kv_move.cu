@@ -115,6 +115,7 @@ cudaError_t launch_pack(const PartGeom& g, const EntryState& st, uint32_t* loc, 
   if (count == 0) return cudaSuccess;
   pack_kernel<<<move_grid(count * pieces_per_entry(g)), kThreads, 0, s>>>(
       g, st, loc, victims, count, ring_start, staging, meta_offset, ws.status);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -169,6 +170,7 @@ cudaError_t launch_unpack(const PartGeom& g, const EntryState& st, uint32_t* loc
   if (count == 0) return cudaSuccess;
   unpack_kernel<<<move_grid(count * pieces_per_entry(g)), kThreads, 0, s>>>(
       g, st, loc, slots, free_ids, count, staging, ws.status);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -246,6 +248,7 @@ cudaError_t launch_admit(const PartGeom& g, const EntryState& st, uint32_t* loc,
   const uint64_t pieces = count * (fill_pattern ? pieces_per_entry(g) : 1);
   admit_kernel<<<move_grid(pieces), kThreads, 0, s>>>(g, st, loc, free_ids, first, count, first_tag,
                                                       new_pairs, epoch, decay, fill_pattern, ws.status);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -306,8 +309,10 @@ cudaError_t launch_init(const EntryState& st, uint64_t* hits, uint64_t* misses, 
     uint64_t rb = ((uint64_t)parts[q].ring_slots + kThreads - 1) / kThreads;
     if (rb > cap) rb = cap;
     init_ring_kernel<<<(unsigned)rb, kThreads, 0, s>>>(parts[q]);
+    count_launches(1);
   }
   init_scalars_kernel<<<1, 256, 0, s>>>(hits, misses, P, p0, ws);
+  count_launches(2);
   return cudaGetLastError();
 }
 

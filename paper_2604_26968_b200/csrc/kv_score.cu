@@ -61,6 +61,7 @@ cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit,
   event_reduce_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(ev_entry, ev_hit, n_events, st.pair,
                                                             st.state, st.touch, st.n, ws.delta,
                                                             ws.status);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -88,6 +89,7 @@ __global__ void posterior_kernel(uint64_t* __restrict__ hits, uint64_t* __restri
 cudaError_t launch_posterior(uint64_t* hits, uint64_t* misses, float* P, float alpha0, float beta0,
                              const Workspace& ws, cudaStream_t s) {
   posterior_kernel<<<1, 32, 0, s>>>(hits, misses, P, alpha0, beta0, ws.delta);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -169,6 +171,7 @@ cudaError_t launch_entry_update(const EntryState& st, const float* P, uint32_t e
   if (blocks > cap) blocks = cap;
   entry_update_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(st.ema, st.decay, st.touch, st.last_epoch,
                                                             st.pair, st.state, st.score, P, st.n, epoch);
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -357,6 +357,7 @@ cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims,
   tile_write_kernel<0><<<n_tiles, kThreads, 0, s>>>(st.score, st.state, st.n, 0, st.n, 0, ws.sel,
                                                     ws.tile_offsets, k, d_victims);
   select_check_kernel<<<1, 1, 0, s>>>(ws.tile_counts, ws.tile_offsets, n_tiles, ws.sel, k, ws.status);
+  count_launches(11);
   return cudaGetLastError();
 }
 
@@ -370,6 +371,7 @@ cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uin
   tile_scan_kernel<<<1, 1024, 0, s>>>(ws.tile_counts, ws.tile_offsets, n_tiles);
   tile_write_kernel<1><<<n_tiles, kThreads, 0, s>>>(st.score, st.state, st.n, lo, hi, tile0, ws.sel,
                                                     ws.tile_offsets, limit, ws.free_list);
+  count_launches(3);
   return cudaGetLastError();
 }
 
@@ -398,6 +400,7 @@ cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const
                                     int n_parts, const Workspace& ws, cudaStream_t s) {
   partition_counts_kernel<<<1, 32, 0, s>>>(d_victims, m, bases5[0], bases5[1], bases5[2], bases5[3],
                                            bases5[4], n_parts, ws.part_counts);
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -11,6 +11,10 @@
 
 using namespace kvt;
 
+namespace kvt {
+std::atomic<uint64_t> g_kernel_launches{0};
+}
+
 namespace {
 
 constexpr uint64_t kAlign = 256;
@@ -87,6 +91,12 @@ struct kv_pool {
   bool events_made = false;
   int staging_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
+  // optional per-launch timing of the pack / unpack kernels
+  struct Timed { cudaEvent_t a, b; int kind; uint64_t bytes; bool pending; };
+  bool timing = false;
+  std::vector<Timed> timed;
+  size_t timed_next = 0;
+  kv_timing totals;
 };
 
 namespace {
@@ -177,6 +187,35 @@ int32_t cuda_fail(kv_pool* p, cudaError_t e) {
     if (e__ != cudaSuccess) return cuda_fail(pool, e__); \
   } while (0)
 
+void timing_settle(kv_pool* p, kv_pool::Timed& t) {
+  if (!t.pending) return;
+  float ms = 0.f;
+  if (cudaEventSynchronize(t.b) == cudaSuccess && cudaEventElapsedTime(&ms, t.a, t.b) == cudaSuccess) {
+    if (t.kind == 0) { p->totals.pack_ms += ms; p->totals.pack_launches += 1; p->totals.pack_bytes += t.bytes; }
+    else { p->totals.unpack_ms += ms; p->totals.unpack_launches += 1; p->totals.unpack_bytes += t.bytes; }
+  }
+  t.pending = false;
+}
+
+// Brackets one kernel launch with timing events when timing is on.
+struct TimedScope {
+  kv_pool* p; kv_pool::Timed* t = nullptr; cudaStream_t s;
+  TimedScope(kv_pool* pool, int kind, uint64_t bytes, cudaStream_t stream) : p(pool), s(stream) {
+    if (!p->timing || p->timed.empty()) return;
+    t = &p->timed[p->timed_next];
+    p->timed_next = (p->timed_next + 1) % p->timed.size();
+    timing_settle(p, *t);
+    t->kind = kind;
+    t->bytes = bytes;
+    cudaEventRecord(t->a, s);
+  }
+  ~TimedScope() {
+    if (!t) return;
+    cudaEventRecord(t->b, s);
+    t->pending = true;
+  }
+};
+
 // entries of one chunk: payload plus (optional) metadata records must fit a staging buffer
 uint64_t entries_per_batch(const kv_pool* p, int q, uint64_t batch_bytes) {
   const uint64_t eb = p->geom[q].entry_bytes;
@@ -265,6 +304,7 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
   p->desc = *desc;
   p->n_parts = g.n_parts;
   std::memset(&p->stats, 0, sizeof(p->stats));
+  std::memset(&p->totals, 0, sizeof(p->totals));
   for (int q = 0; q <= 4; ++q) p->bases[q] = g.bases[q];
   uint8_t* w = static_cast<uint8_t*>(desc->d_workspace);
   p->ws.delta = reinterpret_cast<unsigned long long*>(w + L.delta);
@@ -347,22 +387,39 @@ int32_t kv_pool_destroy(kv_pool* p) {
                          p->ev_list_free[1], p->ev_counts};
     for (cudaEvent_t ev : evs) cudaEventDestroy(ev);
   }
+  for (auto& t : p->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
   delete p;
+  return KV_OK;
+}
+
+int32_t kv_epoch_events(kv_pool* p, const uint32_t* d_ev_entry, const uint8_t* d_ev_hit,
+                        uint64_t n_events, kv_stream_t stream) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  if (n_events > 0 && (!d_ev_entry || !d_ev_hit || !aligned16(d_ev_entry) || !aligned16(d_ev_hit)))
+    return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_event_reduce(d_ev_entry, d_ev_hit, n_events, p->st, p->ws, S(stream)));
+  p->stats.events += n_events;
+  return KV_OK;
+}
+
+uint64_t* kv_epoch_counts(kv_pool* p) {
+  return p ? reinterpret_cast<uint64_t*>(p->ws.delta) : nullptr;
+}
+
+int32_t kv_epoch_update(kv_pool* p, uint32_t epoch, kv_stream_t stream) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_posterior(p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
+                              p->desc.beta0, p->ws, S(stream)));
+  KV_CUDA(p, launch_entry_update(p->st, p->desc.d_P, epoch, S(stream)));
+  p->stats.epochs += 1;
   return KV_OK;
 }
 
 int32_t kv_epoch_score(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_entry, const uint8_t* d_ev_hit,
                        uint64_t n_events, kv_stream_t stream) {
-  if (!p) return KV_ERR_INVALID_ARG;
-  if (n_events > 0 && (!d_ev_entry || !d_ev_hit || !aligned16(d_ev_entry) || !aligned16(d_ev_hit)))
-    return KV_ERR_INVALID_ARG;
-  KV_CUDA(p, launch_event_reduce(d_ev_entry, d_ev_hit, n_events, p->st, p->ws, S(stream)));
-  KV_CUDA(p, launch_posterior(p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
-                              p->desc.beta0, p->ws, S(stream)));
-  KV_CUDA(p, launch_entry_update(p->st, p->desc.d_P, epoch, S(stream)));
-  p->stats.epochs += 1;
-  p->stats.events += n_events;
-  return KV_OK;
+  const int32_t rc = kv_epoch_events(p, d_ev_entry, d_ev_hit, n_events, stream);
+  if (rc != KV_OK) return rc;
+  return kv_epoch_update(p, epoch, stream);
 }
 
 int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream_t stream) {
@@ -424,8 +481,11 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
       KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_staging_free[b], 0));
       const uint64_t meta_off = h.h_meta ? align_up(cnt * eb, 16) : ~0ull;
       const uint64_t slot0 = (h.cursor + c0) % R;
-      KV_CUDA(p, launch_pack(g, p->st, p->desc.d_loc, d_victims + off + c0, cnt, slot0, p->staging[b],
-                             meta_off, p->ws, compute));
+      {
+        TimedScope ts(p, 0, cnt * eb, compute);
+        KV_CUDA(p, launch_pack(g, p->st, p->desc.d_loc, d_victims + off + c0, cnt, slot0, p->staging[b],
+                               meta_off, p->ws, compute));
+      }
       KV_CUDA(p, cudaEventRecord(p->ev_ready[b], compute));
       KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_ready[b], 0));
       const uint64_t first = (cnt < R - slot0) ? cnt : R - slot0;
@@ -517,8 +577,11 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
     }
     KV_CUDA(p, cudaEventRecord(p->ev_ready[b], copy));
     KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_ready[b], 0));
-    KV_CUDA(p, launch_unpack(g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, p->ws.free_list + c0,
-                             cnt, p->staging[b], p->ws, compute));
+    {
+      TimedScope ts(p, 1, cnt * eb, compute);
+      KV_CUDA(p, launch_unpack(g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, p->ws.free_list + c0,
+                               cnt, p->staging[b], p->ws, compute));
+    }
     KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], compute));
   }
   KV_CUDA(p, cudaEventRecord(p->ev_list_free[li], compute));
@@ -558,6 +621,7 @@ int32_t kv_admit(kv_pool* p, uint32_t epoch, float decay, const uint8_t* d_new_p
 int32_t kv_get_stats(const kv_pool* p, kv_stats* out) {
   if (!p || !out) return KV_ERR_INVALID_ARG;
   *out = p->stats;
+  out->kernel_launches = g_kernel_launches.load(std::memory_order_relaxed);
   return KV_OK;
 }
 
@@ -582,6 +646,30 @@ int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) 
   KV_CUDA(p, cudaMemsetAsync(p->ws.status, 0, 4, S(stream)));
   KV_CUDA(p, cudaStreamSynchronize(S(stream)));
   *status_bits = *p->h_status;
+  return KV_OK;
+}
+
+int32_t kv_timing_enable(kv_pool* p, int32_t on) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  if (on && p->timed.empty()) {
+    std::memset(&p->totals, 0, sizeof(p->totals));
+    for (int i = 0; i < 256; ++i) {
+      kv_pool::Timed t{};
+      if (cudaEventCreate(&t.a) != cudaSuccess) return KV_ERR_CUDA;
+      if (cudaEventCreate(&t.b) != cudaSuccess) { cudaEventDestroy(t.a); return KV_ERR_CUDA; }
+      t.pending = false;
+      p->timed.push_back(t);
+    }
+  }
+  p->timing = on != 0;
+  return KV_OK;
+}
+
+int32_t kv_timing_read(kv_pool* p, kv_timing* out) {
+  if (!p || !out) return KV_ERR_INVALID_ARG;
+  for (auto& t : p->timed) timing_settle(p, t);
+  *out = p->totals;
+  std::memset(&p->totals, 0, sizeof(p->totals));
   return KV_OK;
 }
 

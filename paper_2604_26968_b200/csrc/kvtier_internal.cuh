@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "kvtier.h"
 
 namespace kvt {
@@ -12,6 +14,10 @@ constexpr int kThreads = 256;
 constexpr uint32_t kRadixBits1 = 11, kRadixBits2 = 11, kRadixBits3 = 10;
 constexpr uint32_t kHistBins = 2048;  // bins of the widest digit
 constexpr uint32_t kTileEntries = 2048;  // entries per compaction tile (256 threads x 8)
+
+// Kernels launched by this library in this process (all pools).
+extern std::atomic<uint64_t> g_kernel_launches;
+inline void count_launches(uint64_t n) { g_kernel_launches.fetch_add(n, std::memory_order_relaxed); }
 
 // Geometry of one partition, as the kernels need it.
 struct PartGeom {
