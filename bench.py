@@ -49,6 +49,7 @@ def parse():
     ap.add_argument("--batch-mb", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-hostlink", action="store_true", help="skip the 1 GiB host-link probe")
     return ap.parse_args()
 
 
@@ -251,7 +252,7 @@ def main():
 
     w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots)
     w.seed = w.seed + 1000 * rank     # every rank owns its own pool and trace (weak scaling)
-    link = hostlink_probe(torch, dev) if rank == 0 else None
+    link = hostlink_probe(torch, dev) if rank == 0 and not args.no_hostlink else None
     runner = EpochRunner(w, batch_bytes=args.batch_mb << 20, fill_pattern=True, host_meta=True,
                          device=str(dev))
     pool = runner.pool
