@@ -233,6 +233,32 @@ int32_t kv_demote(kv_pool* pool, const uint32_t* d_victims, uint64_t m, uint64_t
 int32_t kv_promote(kv_pool* pool, int32_t partition, const uint64_t* h_host_slots, uint64_t m,
                    uint64_t batch_bytes, kv_stream_t compute, kv_stream_t copy);
 
+/* Selection for callers that cannot allocate (the paper has no counterpart; it
+ * is a packaging of kv_select_victims, not another method).  A serving engine
+ * that has given all device memory to its own pools, or code that runs where
+ * cudaMalloc is off limits, has no workspace to hand to kv_pool_create.  This
+ * call needs none: it takes the score and state arrays directly and keeps its
+ * scratch (histograms, scalars, per-tile counts; about 58 KB) in a fixed array
+ * inside the library, which every GPU that loads the library holds until the
+ * process exits.  It calls no allocating routine.
+ *   d_score  (device) f32[n]  eviction scores, as kv_epoch_score writes them
+ *   d_state  (device) u8[n]   KV_STATE_*; only RESIDENT entries are candidates
+ *   d_victims (device) u32[k] receives the k lowest (score, id) entries, ascending id
+ *   d_status (device, optional) one u32 that receives KV_DEV_SELECT_MISMATCH if k
+ *            exceeded the number of RESIDENT entries (the host cannot know that
+ *            count here, so the caller must keep k within it); the caller zeroes it
+ * Limits and rules:
+ *   - n <= 4,194,304 entries; larger n returns KV_ERR_INVALID_ARG, k > n returns
+ *     KV_ERR_K_TOO_LARGE; pointers must be 16-byte aligned;
+ *   - the first call on each device looks up the array's device address (with
+ *     that device current); make that first call before any stream capture;
+ *   - all calls on a device share the one array, which is cleared at the start of
+ *     each call: two calls whose GPU work overlaps (different streams, no
+ *     ordering between them) race and give wrong results.  Order them. */
+int32_t kv_select_victims_static(const float* d_score, const uint8_t* d_state, uint64_t n,
+                                 uint64_t k, uint32_t* d_victims, uint32_t* d_status,
+                                 kv_stream_t stream);
+
 /* Largest batch_bytes the staging buffers allow for a partition. */
 uint64_t kv_max_batch_bytes(const kv_pool* pool, int32_t partition);
 

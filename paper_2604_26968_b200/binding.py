@@ -77,7 +77,7 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
            "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_events", "kv_epoch_counts",
-           "kv_epoch_update", "kv_select_victims", "kv_demote",
+           "kv_epoch_update", "kv_select_victims", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
            "kv_last_cuda_error", "kv_status_string",
@@ -118,6 +118,8 @@ def load():
     L.kv_epoch_update.argtypes = [vp, u32, vp]
     L.kv_select_victims.restype = i32
     L.kv_select_victims.argtypes = [vp, u64, vp, vp]
+    L.kv_select_victims_static.restype = i32
+    L.kv_select_victims_static.argtypes = [vp, vp, u64, u64, vp, vp, vp]
     L.kv_demote.restype = i32
     L.kv_demote.argtypes = [vp, vp, u64, u64, vp, vp]
     L.kv_promote.restype = i32
@@ -174,6 +176,15 @@ def kv_entry_bytes(model: kv_model_desc, block_tokens: int) -> int:
 
 def _stream_ptr(s):
     return C.c_void_p(s.cuda_stream if s is not None else 0)
+
+
+def kv_select_victims_static(d_score, d_state, n, k, d_victims, d_status=None, stream=None) -> int:
+    """Selection with the library's built-in scratch: for callers that cannot
+    allocate a workspace.  Arguments are torch device tensors; returns the status."""
+    return load().kv_select_victims_static(
+        d_score.data_ptr(), d_state.data_ptr(), int(n), int(k),
+        d_victims.data_ptr() if d_victims is not None else None,
+        d_status.data_ptr() if d_status is not None else None, _stream_ptr(stream))
 
 
 class Pool:

@@ -8,6 +8,8 @@
 // of the k-th smallest entry; an ordered compaction then emits, in ascending id
 // order, every entry with key < tau plus the first k - #{key < tau} entries with
 // key == tau.  Nothing waits on another block: each phase is its own launch.
+#include <mutex>
+
 #include "kvtier_internal.cuh"
 
 namespace kvt {
@@ -405,3 +407,82 @@ cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const
 }
 
 }  // namespace kvt
+
+// ---- selection without any caller-provided or allocated scratch -------------------
+// Some callers of this library must not allocate: a serving engine that has
+// already handed every byte of device memory to its own pools, or code running
+// where cudaMalloc is forbidden (inside a latency-critical loop, or under an
+// allocator that owns the whole device).  For them the scratch that selection
+// needs -- three digit histograms, a handful of scalars and the per-tile counts
+// of the compaction -- lives in this fixed array, which every GPU that loads the
+// library holds until the process exits.  Its size bounds the problem:
+// kStaticMaxEntries entries.
+namespace {
+
+constexpr uint64_t kStaticMaxEntries = 1ull << 22;  // 4,194,304 entries
+constexpr uint64_t kStaticMaxTiles = kStaticMaxEntries / kvt::kTileEntries + 2;
+// layout (bytes): [0, 24576) histograms | [24576, 24832) scalars | [24832, 25088) status |
+//                 [25088, +tiles*8) tile counts | then tile offsets
+constexpr uint64_t kOffHist = 0;
+constexpr uint64_t kOffSel = 3 * kvt::kHistBins * 4;
+constexpr uint64_t kOffStatus = kOffSel + 256;
+constexpr uint64_t kOffTileCounts = kOffStatus + 256;
+constexpr uint64_t kOffTileOffsets = kOffTileCounts + ((kStaticMaxTiles * 8 + 255) / 256) * 256;
+constexpr uint64_t kStaticScratchBytes = kOffTileOffsets + ((kStaticMaxTiles * 8 + 255) / 256) * 256;
+
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+unsigned char* g_scratch_addr[kMaxDevices] = {nullptr};
+
+// The array's name is only a stand-in on the host; the address a kernel can use
+// comes from the runtime, once per device, with that device current.
+cudaError_t static_scratch(unsigned char** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_select_scratch);
+    if (e != cudaSuccess) return e;
+    g_scratch_addr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_scratch_addr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int32_t kv_select_victims_static(const float* d_score, const uint8_t* d_state, uint64_t n,
+                                            uint64_t k, uint32_t* d_victims, uint32_t* d_status,
+                                            kv_stream_t stream) {
+  if (n == 0 || n > kStaticMaxEntries) return KV_ERR_INVALID_ARG;  // beyond the built-in scratch
+  if (k > n) return KV_ERR_K_TOO_LARGE;
+  if (!d_score || !d_state || (reinterpret_cast<uintptr_t>(d_score) & 15u) ||
+      (reinterpret_cast<uintptr_t>(d_state) & 15u))
+    return KV_ERR_INVALID_ARG;
+  if (k == 0) return KV_OK;
+  if (!d_victims || (reinterpret_cast<uintptr_t>(d_victims) & 15u)) return KV_ERR_INVALID_ARG;
+  unsigned char* base = nullptr;
+  if (static_scratch(&base) != cudaSuccess) return KV_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left: start the histograms and the
+  // status word from zero (the scalars are reset by the first kernel of the pass).
+  if (cudaMemsetAsync(base + kOffHist, 0, kOffTileCounts, s) != cudaSuccess) return KV_ERR_CUDA;
+  kvt::Workspace ws{};
+  ws.hist = reinterpret_cast<uint32_t*>(base + kOffHist);
+  ws.sel = reinterpret_cast<kvt::SelectScalars*>(base + kOffSel);
+  ws.status = d_status ? d_status : reinterpret_cast<uint32_t*>(base + kOffStatus);
+  ws.tile_counts = reinterpret_cast<uint2*>(base + kOffTileCounts);
+  ws.tile_offsets = reinterpret_cast<uint2*>(base + kOffTileOffsets);
+  ws.n_tiles = (uint32_t)kStaticMaxTiles;
+  kvt::EntryState st{};
+  st.score = const_cast<float*>(d_score);   // selection only reads score and state
+  st.state = const_cast<uint8_t*>(d_state);
+  st.n = n;
+  if (kvt::launch_select(st, k, d_victims, ws, s) != cudaSuccess) return KV_ERR_CUDA;
+  return KV_OK;
+}
