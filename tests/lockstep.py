@@ -38,6 +38,9 @@ class Lockstep:
         self.payload = payload
         self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
                                fill_pattern=True, host_meta=host_meta)
+        # room for any k a test may ask for
+        self.gpu.victims = self.gpu.torch.empty(max(w.N, 4), dtype=self.gpu.torch.int32,
+                                                device=self.gpu.pool.device)
         self.ora = O.OraclePool(oracle_parts(w), w.alpha0, w.beta0, n_tags=w.n_tags, payload=payload)
         oracle_admit(w, self.ora, 0, key=INITIAL_EPOCH_KEY)
         self.compare_state("initial fill")
@@ -145,3 +148,35 @@ class Lockstep:
     def close(self):
         self.gpu.close()
         self.ora.close()
+
+
+def sample_payload(ls, n=256, seed=0):
+    """Checks sampled blocks of a (large) pool against the byte pattern of the tag the
+    oracle says lives there: n resident HBM entries and n live ring slots per partition."""
+    import torch
+    g, o, w = ls.gpu, ls.ora, ls.w
+    g.pool.sync()
+    r = np.random.default_rng(seed)
+    for q, p in enumerate(w.parts):
+        inf = o.info(q)
+        H, cb, nc, eb = inf["H"], inf["chunk_bytes"], inf["n_chunks"], inf["entry_bytes"]
+        ids = np.flatnonzero(o.state[inf["base"]:inf["base"] + inf["n"]] == O.RESIDENT)
+        ids = r.choice(ids, size=min(n, ids.size), replace=False)
+        slab = g.pool.slabs[q]
+        for local in ids:
+            tag = int(o.tag[inf["base"] + local])
+            lb, head = divmod(int(local), H)
+            pieces = []
+            for c in range(nc):
+                off = ((lb * nc + c) * H + head) * cb
+                pieces.append(slab[off:off + cb])
+            got = torch.cat(pieces).cpu().numpy()
+            assert np.array_equal(got, W.pattern_bytes([tag], eb)[0]), (q, int(local), tag)
+        live = np.flatnonzero(o.part_array(q, "r_live"))
+        if live.size:
+            slots = r.choice(live, size=min(n, live.size), replace=False)
+            ring = g.pool.rings[q].numpy()
+            rt = o.part_array(q, "r_tag")
+            for s in slots:
+                got = ring[int(s) * eb:(int(s) + 1) * eb]
+                assert np.array_equal(got, W.pattern_bytes([int(rt[s])], eb)[0]), (q, int(s))
