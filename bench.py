@@ -50,6 +50,8 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-hostlink", action="store_true", help="skip the 1 GiB host-link probe")
+    ap.add_argument("--move-variant", type=int, default=1, choices=[0, 1],
+                    help="pack/unpack kernels: 1 = bulk-copy engine, 0 = register path")
     return ap.parse_args()
 
 
@@ -257,6 +259,8 @@ def main():
                          device=str(dev))
     pool = runner.pool
     pool.kv_timing_enable(True)
+    from paper_2604_26968_b200 import binding as B
+    B.kv_set_move_variant(args.move_variant)
     N, k = w.N, w.k
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     counts = pool.kv_epoch_counts() if world > 1 else None

@@ -307,6 +307,11 @@ typedef struct {
 int32_t kv_timing_enable(kv_pool* pool, int32_t on);
 int32_t kv_timing_read(kv_pool* pool, kv_timing* out);
 
+/* Measurement aid: which pack/unpack kernels kv_demote and kv_promote launch from
+ * now on (process-wide): 1 = shared-memory-staged bulk asynchronous copies
+ * (default), 0 = 16-byte loads and stores through registers. */
+int32_t kv_set_move_variant(int32_t variant);
+
 /* The last CUDA error code seen by a call on this pool (0 = none). */
 int32_t kv_last_cuda_error(const kv_pool* pool);
 

@@ -14,6 +14,8 @@ using namespace kvt;
 namespace kvt {
 std::atomic<uint64_t> g_kernel_launches{0};
 }
+// which pack/unpack kernels run: 1 = bulk-copy engine (default), 0 = register path
+static int g_move_variant = 1;
 
 namespace {
 
@@ -483,8 +485,9 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
       const uint64_t slot0 = (h.cursor + c0) % R;
       {
         TimedScope ts(p, 0, cnt * eb, compute);
-        KV_CUDA(p, launch_pack(g, p->st, p->desc.d_loc, d_victims + off + c0, cnt, slot0, p->staging[b],
-                               meta_off, p->ws, compute));
+        KV_CUDA(p, (g_move_variant ? launch_pack_tma : launch_pack)(
+                       g, p->st, p->desc.d_loc, d_victims + off + c0, cnt, slot0, p->staging[b], meta_off,
+                       p->ws, compute));
       }
       KV_CUDA(p, cudaEventRecord(p->ev_ready[b], compute));
       KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_ready[b], 0));
@@ -579,8 +582,9 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
     KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_ready[b], 0));
     {
       TimedScope ts(p, 1, cnt * eb, compute);
-      KV_CUDA(p, launch_unpack(g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, p->ws.free_list + c0,
-                               cnt, p->staging[b], p->ws, compute));
+      KV_CUDA(p, (g_move_variant ? launch_unpack_tma : launch_unpack)(
+                     g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, p->ws.free_list + c0, cnt,
+                     p->staging[b], p->ws, compute));
     }
     KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], compute));
   }
@@ -646,6 +650,12 @@ int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) 
   KV_CUDA(p, cudaMemsetAsync(p->ws.status, 0, 4, S(stream)));
   KV_CUDA(p, cudaStreamSynchronize(S(stream)));
   *status_bits = *p->h_status;
+  return KV_OK;
+}
+
+int32_t kv_set_move_variant(int32_t variant) {
+  if (variant != 0 && variant != 1) return KV_ERR_INVALID_ARG;
+  g_move_variant = variant;
   return KV_OK;
 }
 

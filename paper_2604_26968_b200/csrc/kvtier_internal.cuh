@@ -102,6 +102,13 @@ cudaError_t launch_pack(const PartGeom& g, const EntryState& st, uint32_t* loc, 
 cudaError_t launch_unpack(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
                           const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
                           const Workspace& ws, cudaStream_t s);
+// ---- kv_move_tma.cu: the same two operations on the bulk asynchronous copy engine ----
+cudaError_t launch_pack_tma(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* victims,
+                            uint64_t count, uint64_t ring_start, uint8_t* staging, uint64_t meta_offset,
+                            const Workspace& ws, cudaStream_t s);
+cudaError_t launch_unpack_tma(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
+                              const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
+                              const Workspace& ws, cudaStream_t s);
 // admits free_list[first .. first+count) of one partition
 cudaError_t launch_admit(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* free_ids,
                          uint64_t first, uint64_t count, uint64_t first_tag, const uint8_t* new_pairs,
