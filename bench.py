@@ -32,9 +32,13 @@ if ROOT not in sys.path:
 METRIC = "KV head-blocks scored+selected/s"
 UNIT = "head-blocks/s"
 
-# DRAM traffic per launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum),
-# keyed by kernel; None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE = {"pack_kernel": None}
+# DRAM traffic from ncu (dram__bytes_read.sum + dram__bytes_write.sum) per payload
+# byte of a launch, keyed by move variant: captured on a 256 MiB launch of a
+# 3 GiB pool (488.7 MB of traffic for 268.4 MB of payload) and scaled to the
+# benchmark's launch size in proportion to the payload.  None = no capture of
+# that kernel as it stands.
+NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE = {1: 488.74 / 268.44, 0: None}
+PACK_KERNEL_NAME = {1: "move_tma_kernel<true> (pack)", 0: "pack_kernel"}
 
 
 def parse():
@@ -46,7 +50,7 @@ def parse():
     ap.add_argument("--config", type=int, default=2, help="pool 1..5")
     ap.add_argument("--scale", type=float, default=1.0, help="shrinks blocks per layer")
     ap.add_argument("--ring-slots", type=int, default=None)
-    ap.add_argument("--batch-mb", type=int, default=64)
+    ap.add_argument("--batch-mb", type=int, default=1024, help="demote/promote chunk (staging buffer) size")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-hostlink", action="store_true", help="skip the 1 GiB host-link probe")
@@ -178,11 +182,11 @@ def oracle_epochs(w, n_epochs, warm=0):
     epoch, epochs timed)."""
     from paper_2604_26968_b200.harness import INITIAL_EPOCH_KEY
     O, pool = oracle_pool(w)
-    n_free = int((pool.state == O.FREE).sum())
-    pool.admit(0, w.decay, w.new_pairs(INITIAL_EPOCH_KEY, n_free), None)
+    fresh = np.flatnonzero(pool.state == O.FREE).astype(np.uint32)
+    pool.admit(0, w.decay, w.new_pairs(INITIAL_EPOCH_KEY, fresh.size), None)
     t_ss, t_all, done = 0.0, 0.0, 0
     for e in range(warm + n_epochs):
-        ev_entry, ev_hit = w.events(e, pool.pair)
+        ev_entry, ev_hit = w.events(e, pool.pair, fresh)
         t0 = time.perf_counter()
         assert pool.epoch_score(e, ev_entry, ev_hit) == O.OK
         rc, v = pool.select_victims(w.k)
@@ -202,8 +206,8 @@ def oracle_epochs(w, n_epochs, warm=0):
             t_ss += t1 - t0
             t_all += (t1 - t0) + t_move
             done += 1
-        n_free = int((pool.state == O.FREE).sum())
-        pool.admit(e, w.decay, w.new_pairs(e, n_free), None)
+        fresh = np.flatnonzero(pool.state == O.FREE).astype(np.uint32)
+        pool.admit(e, w.decay, w.new_pairs(e, fresh.size), None)
     pool.close()
     return t_ss, t_all, done
 
@@ -266,8 +270,7 @@ def main():
     counts = pool.kv_epoch_counts() if world > 1 else None
 
     def gen_events(e):
-        pair = runner.host_array("pair")
-        return w.events(e, pair)
+        return runner.next_events(e)
 
     def one_step(e, d_e, d_h, n, ev):
         """Enqueues one full step; ev = (start, selected, demoted, end) CUDA events."""
@@ -389,7 +392,7 @@ def main():
     pack_gbs = 2 * timing["pack_bytes"] / max(timing["pack_ms"], 1e-9) / 1e6
     unpack_gbs = 2 * timing["unpack_bytes"] / max(timing["unpack_ms"], 1e-9) / 1e6
     ss_bytes = 39 * N + 5 * (tot["events"] / K) + 4 * k
-    tr = NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE["pack_kernel"]
+    tr = NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE[args.move_variant]
     line = {
         "metric": METRIC, "value": N * world / (ss_ms * 1e-3), "unit": UNIT,
         "value_definition": "N / t(kv_epoch_score + kv_select_victims), timed with CUDA events inside full steps",
@@ -413,7 +416,7 @@ def main():
             "pack_launches": timing["pack_launches"], "unpack_launches": timing["unpack_launches"],
         },
         "hostlink": link,
-        "roofline": {"kernel": "pack_kernel", "bound": "hbm", "achieved": pack_gbs, "peak": peak,
+        "roofline": {"kernel": PACK_KERNEL_NAME[args.move_variant], "bound": "hbm", "achieved": pack_gbs, "peak": peak,
                      "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": pack_gbs / peak,
                      "traffic": (tr * timing["pack_bytes"] / max(timing["pack_launches"], 1)) if tr else None,
                      "algorithmic_bytes_per_launch": 2 * timing["pack_bytes"] / max(timing["pack_launches"], 1)},

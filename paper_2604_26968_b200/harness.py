@@ -28,7 +28,12 @@ class EpochRunner:
         self.fill_pattern = fill_pattern
         self.k = workload.k
         self.victims = torch.empty(max(self.k, 4), dtype=torch.int32, device=self.pool.device)
+        self.fresh = None      # entries admitted by the last admit() (input of the next epoch's trace)
         self.check(self.admit(0, key=INITIAL_EPOCH_KEY), "initial kv_admit")
+
+    def next_events(self, epoch):
+        """Draws the epoch's trace from the pool's current pair ids and last admissions."""
+        return self.w.events(epoch, self.host_array("pair"), self.fresh)
 
     def check(self, rc, what):
         if isinstance(rc, tuple):
@@ -52,6 +57,8 @@ class EpochRunner:
 
     def admit(self, epoch, key=None, n_free=None):
         n_free = self.pool.kv_get_stats()["n_free"] if n_free is None else n_free
+        self.fresh = np.flatnonzero(self.host_array("state") == B.KV_STATE_FREE).astype(np.uint32)
+        assert self.fresh.size == n_free
         pairs = self.w.new_pairs(epoch if key is None else key, n_free)
         d_pairs = self.to_device(np.concatenate([pairs, np.zeros(16, np.uint8)]), None)
         rc = self.pool.kv_admit(epoch, self.w.decay, d_pairs, self.fill_pattern)

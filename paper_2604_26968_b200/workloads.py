@@ -133,12 +133,14 @@ class Workload:
             return r.integers(0, 16, size=n, dtype=np.uint8)
         return r.choice(16, size=n, p=self.pair_weights).astype(np.uint8)
 
-    def events(self, epoch: int, pair: np.ndarray):
+    def events(self, epoch: int, pair: np.ndarray, fresh: Optional[np.ndarray] = None):
         """(ev_entry u32[E], ev_hit u8[E]) of one epoch.
 
         pair is the current per-entry pair-id array: the hit flag of a touch is
         Bernoulli(q[pair]) with q[p] = (p + 0.5) / 16, which gives each of the
-        16 posteriors a known limit.
+        16 posteriors a known limit.  fresh lists the entries admitted at the end
+        of the previous epoch: a block that had to be brought in was a cache miss
+        and is being used, so each contributes one touch with a miss flag.
         """
         r = self.rng(epoch, 2)
         chunks = []
@@ -153,6 +155,9 @@ class Workload:
         ev_entry = ids.astype(np.uint32)
         qhit = (pair[ev_entry].astype(np.float64) + 0.5) / 16.0
         ev_hit = (r.random(ev_entry.size) < qhit).astype(np.uint8)
+        if fresh is not None and len(fresh):
+            ev_entry = np.concatenate([ev_entry, np.asarray(fresh, dtype=np.uint32)])
+            ev_hit = np.concatenate([ev_hit, np.zeros(len(fresh), np.uint8)])
         return ev_entry, ev_hit
 
     def promote_list(self, epoch: int, q: int, m: int, cursor: int, live: np.ndarray) -> np.ndarray:
@@ -369,7 +374,7 @@ def config(i: int, scale: float = 1.0, ring_slots: Optional[int] = None) -> Work
                      0.10, 0.05, seed=3, epochs=40)
     elif i == 5:
         blocks = nb(10720)
-        parts = [mha(32, 32, 128, 16, blocks, ring(1 << 20), "mixed"),
+        parts = [mha(32, 32, 128, 16, blocks, ring(3 << 19), "mixed"),
                  gqa(80, 64, 8, 128, 16, blocks, ring(1 << 20), "mixed"),
                  mqa(32, 32, 128, 16, blocks, ring(1 << 17), "mixed"),
                  mla(61, 512, 64, 16, blocks, ring(1 << 17), "mixed")]

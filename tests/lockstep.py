@@ -15,8 +15,10 @@ def oracle_parts(w):
 
 
 def oracle_admit(w, pool, epoch, key=None):
-    """Admits into every FREE slot of the oracle pool; payload = pattern(tag)."""
-    n_free = int((pool.state == O.FREE).sum())
+    """Admits into every FREE slot of the oracle pool; payload = pattern(tag).
+    Returns the ids admitted (ascending)."""
+    fresh = np.flatnonzero(pool.state == O.FREE).astype(np.uint32)
+    n_free = int(fresh.size)
     pairs = w.new_pairs(epoch if key is None else key, n_free)
     payload = None
     if pool.payload and n_free:
@@ -29,7 +31,7 @@ def oracle_admit(w, pool, epoch, key=None):
         payload = np.concatenate(imgs)
     got = pool.admit(epoch, w.decay, pairs, payload)
     assert got == n_free, got
-    return n_free
+    return fresh
 
 
 class Lockstep:
@@ -42,7 +44,8 @@ class Lockstep:
         self.gpu.victims = self.gpu.torch.empty(max(w.N, 4), dtype=self.gpu.torch.int32,
                                                 device=self.gpu.pool.device)
         self.ora = O.OraclePool(oracle_parts(w), w.alpha0, w.beta0, n_tags=w.n_tags, payload=payload)
-        oracle_admit(w, self.ora, 0, key=INITIAL_EPOCH_KEY)
+        self.fresh = oracle_admit(w, self.ora, 0, key=INITIAL_EPOCH_KEY)
+        assert np.array_equal(self.fresh, self.gpu.fresh)
         self.compare_state("initial fill")
         if payload:
             self.compare_payload("initial fill")
@@ -113,7 +116,7 @@ class Lockstep:
     def epoch(self, e, k=None, check_payload=None):
         w, g, o = self.w, self.gpu, self.ora
         k = w.k if k is None else k
-        ev_entry, ev_hit = w.events(e, o.pair)
+        ev_entry, ev_hit = w.events(e, o.pair, self.fresh)
         d_e, d_h, n = g.stage_events(ev_entry, ev_hit)
         assert o.epoch_score(e, ev_entry, ev_hit) == O.OK
         g.check(g.pool.kv_epoch_score(e, d_e, d_h, n), "kv_epoch_score")
@@ -134,8 +137,10 @@ class Lockstep:
             g.check(g.pool.kv_promote(q, lst, g.batch_bytes), "kv_promote")
         self.compare_state("epoch %d promote" % e, scores=False)
         self.compare_ring("epoch %d promote" % e)
-        n_free = oracle_admit(w, o, e)
+        self.fresh = oracle_admit(w, o, e)
+        n_free = int(self.fresh.size)
         g.check(g.admit(e, n_free=n_free), "kv_admit")
+        assert np.array_equal(self.fresh, g.fresh)
         self.compare_state("epoch %d admit" % e, scores=False)
         if self.payload and (check_payload is None or check_payload):
             self.compare_payload("epoch %d" % e)

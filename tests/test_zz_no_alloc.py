@@ -29,7 +29,7 @@ def test_static_selection_matches_pool_selection_on_two_calls_in_a_row():
     N = w.N
     status = torch.zeros(4, dtype=torch.int32, device=pool.device)
     for call, k in enumerate((N // 20, N // 3)):
-        ev_entry, ev_hit = w.events(call, r.host_array("pair"))
+        ev_entry, ev_hit = r.next_events(call)
         d_e, d_h, n = r.stage_events(ev_entry, ev_hit)
         r.check(pool.kv_epoch_score(call, d_e, d_h, n), "kv_epoch_score")
         if call == 1:      # FREE holes: demote the first call's victims
