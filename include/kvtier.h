@@ -312,6 +312,12 @@ int32_t kv_timing_read(kv_pool* pool, kv_timing* out);
  * (default), 0 = 16-byte loads and stores through registers. */
 int32_t kv_set_move_variant(int32_t variant);
 
+/* Measurement aid: how kv_select_victims runs from now on (process-wide): 1 = one
+ * persistent cooperative launch with the keys held in shared memory (default;
+ * falls back to 0 where the device cannot co-schedule it), 0 = one launch per
+ * phase of the radix select. */
+int32_t kv_set_select_variant(int32_t variant);
+
 /* The last CUDA error code seen by a call on this pool (0 = none). */
 int32_t kv_last_cuda_error(const kv_pool* pool);
 

@@ -80,7 +80,7 @@ EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_
            "kv_epoch_update", "kv_select_victims", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
-           "kv_set_move_variant", "kv_last_cuda_error", "kv_status_string",
+           "kv_set_move_variant", "kv_set_select_variant", "kv_last_cuda_error", "kv_status_string",
            "kv_version")
 
 _lib = None
@@ -140,6 +140,8 @@ def load():
     L.kv_timing_enable.argtypes = [vp, i32]
     L.kv_timing_read.restype = i32
     L.kv_timing_read.argtypes = [vp, C.POINTER(kv_timing)]
+    L.kv_set_select_variant.restype = i32
+    L.kv_set_select_variant.argtypes = [i32]
     L.kv_set_move_variant.restype = i32
     L.kv_set_move_variant.argtypes = [i32]
     L.kv_last_cuda_error.restype = i32
@@ -174,6 +176,10 @@ def kv_infer_variant(model: kv_model_desc) -> int:
 
 def kv_entry_bytes(model: kv_model_desc, block_tokens: int) -> int:
     return load().kv_entry_bytes(C.byref(model), block_tokens)
+
+
+def kv_set_select_variant(variant: int) -> int:
+    return load().kv_set_select_variant(int(variant))
 
 
 def kv_set_move_variant(variant: int) -> int:

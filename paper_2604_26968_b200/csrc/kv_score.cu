@@ -1,4 +1,4 @@
-// Scoring kernels: event reduction, Beta posterior, fused EMA + score pass.
+// Scoring kernels: event reduction, and the fused posterior + EMA + score pass.
 //
 // All binary32 arithmetic uses the explicitly rounded intrinsics (__fmul_rn,
 // __fadd_rn, __fsub_rn, __fdiv_rn), which the compiler never contracts into a
@@ -12,9 +12,16 @@ namespace kvt {
 // Each event adds one to the (pair, hit) counter of its entry's pair -- the
 // alpha += 1 / beta += 1 update of the Bayesian reuse section -- and one to the
 // entry's touch count.  Counters are integers, so the order of the atomics does
-// not matter.  Lanes of a warp that hit the same counter are merged first
+// not matter.  A thread takes four consecutive events at a time so that its
+// eight scattered gathers (state and pair of four entries) are in flight
+// together; lanes of a warp that hit the same counter are merged first
 // (match.any), then a 32-counter shared-memory table per block, then one 64-bit
 // global atomic per non-zero counter per block.
+__device__ __forceinline__ void count_event(uint32_t key, uint32_t* s_cnt, unsigned lane) {
+  const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
+  if (key < 32 && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_cnt[key], __popc(peers));
+}
+
 __global__ void __launch_bounds__(kThreads)
 event_reduce_kernel(const uint32_t* __restrict__ ev_entry, const uint8_t* __restrict__ ev_hit,
                     uint64_t n_events, const uint8_t* __restrict__ pair,
@@ -25,26 +32,60 @@ event_reduce_kernel(const uint32_t* __restrict__ ev_entry, const uint8_t* __rest
   __syncthreads();
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
   const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const uint64_t iters = (n_events + stride - 1) / stride;  // same for every thread
+  const uint64_t n4 = n_events / 4;
+  const uint64_t iters = (n4 + stride - 1) / stride;  // same for every thread: the votes need all lanes
   const unsigned lane = threadIdx.x & 31u;
   uint32_t bad = 0;
   for (uint64_t it = 0; it < iters; ++it) {
-    const uint64_t e = it * stride + gtid;
-    uint32_t key = 32;  // 32 = nothing to count
+    const uint64_t v = it * stride + gtid;
+    const bool valid = v < n4;
+    uint4 id4 = make_uint4(0, 0, 0, 0);
+    uchar4 h4 = make_uchar4(0, 0, 0, 0);
+    if (valid) {
+      id4 = reinterpret_cast<const uint4*>(ev_entry)[v];
+      h4 = reinterpret_cast<const uchar4*>(ev_hit)[v];
+    }
+    const uint32_t ids[4] = {id4.x, id4.y, id4.z, id4.w};
+    const uint32_t hit[4] = {h4.x != 0, h4.y != 0, h4.z != 0, h4.w != 0};
+    uint32_t st[4], pr[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {  // all gathers issued before any is used
+      const bool in = valid && ids[j] < n;
+      st[j] = in ? state[ids[j]] : 0xFFu;
+      pr[j] = in ? pair[ids[j]] : 0u;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t key = 32;  // 32 = nothing to count
+      if (valid) {
+        if (ids[j] >= n) {
+          bad |= KV_DEV_EVENT_BAD_ID;
+        } else if (st[j] != KV_STATE_RESIDENT) {
+          bad |= KV_DEV_EVENT_NOT_RESIDENT;
+        } else {
+          key = pr[j] * 2u + hit[j];
+          atomicAdd(&touch[ids[j]], 1u);
+        }
+      }
+      count_event(key, s_cnt, lane);
+    }
+  }
+  // ragged tail (n_events not a multiple of 4): first warp of the grid
+  if (blockIdx.x == 0 && threadIdx.x < 32) {
+    const uint64_t e = n4 * 4 + threadIdx.x;
+    uint32_t key = 32;
     if (e < n_events) {
       const uint32_t i = ev_entry[e];
-      const uint32_t hit = ev_hit[e] != 0;
       if (i >= n) {
         bad |= KV_DEV_EVENT_BAD_ID;
       } else if (state[i] != KV_STATE_RESIDENT) {
         bad |= KV_DEV_EVENT_NOT_RESIDENT;
       } else {
-        key = (uint32_t)pair[i] * 2u + hit;
+        key = (uint32_t)pair[i] * 2u + (ev_hit[e] != 0);
         atomicAdd(&touch[i], 1u);
       }
     }
-    const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
-    if (key < 32 && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_cnt[key], __popc(peers));
+    count_event(key, s_cnt, lane);
   }
   if (bad) atomicOr(status, bad);
   __syncthreads();
@@ -55,40 +96,13 @@ event_reduce_kernel(const uint32_t* __restrict__ ev_entry, const uint8_t* __rest
 cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit, uint64_t n_events,
                                 const EntryState& st, const Workspace& ws, cudaStream_t s) {
   if (n_events == 0) return cudaSuccess;
-  uint64_t blocks = (n_events + kThreads - 1) / kThreads;
+  uint64_t blocks = (n_events / 4 + kThreads - 1) / kThreads;
+  if (blocks == 0) blocks = 1;
   const uint64_t cap = (uint64_t)kSMs * 8;
   if (blocks > cap) blocks = cap;
   event_reduce_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(ev_entry, ev_hit, n_events, st.pair,
                                                             st.state, st.touch, st.n, ws.delta,
                                                             ws.status);
-  count_launches(1);
-  return cudaGetLastError();
-}
-
-// ---- posterior ----------------------------------------------------------------
-// Folds the epoch's counts into the running totals and forms the posterior mean
-// of Eq. "reuse": P = alpha / (alpha + beta) with alpha = alpha0 + hits,
-// beta = beta0 + misses.  The 64-bit counts convert to binary32 with round to
-// nearest even.
-__global__ void posterior_kernel(uint64_t* __restrict__ hits, uint64_t* __restrict__ misses,
-                                 float* __restrict__ P, float alpha0, float beta0,
-                                 unsigned long long* __restrict__ delta) {
-  const unsigned p = threadIdx.x;
-  if (p >= 16) return;
-  const unsigned long long h = hits[p] + delta[2 * p + 1];
-  const unsigned long long m = misses[p] + delta[2 * p];
-  hits[p] = h;
-  misses[p] = m;
-  delta[2 * p] = 0;
-  delta[2 * p + 1] = 0;
-  const float a = __fadd_rn(alpha0, __ull2float_rn(h));
-  const float b = __fadd_rn(beta0, __ull2float_rn(m));
-  P[p] = __fdiv_rn(a, __fadd_rn(a, b));
-}
-
-cudaError_t launch_posterior(uint64_t* hits, uint64_t* misses, float* P, float alpha0, float beta0,
-                             const Workspace& ws, cudaStream_t s) {
-  posterior_kernel<<<1, 32, 0, s>>>(hits, misses, P, alpha0, beta0, ws.delta);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -109,19 +123,45 @@ __device__ __forceinline__ void entry_step(float& ema, float decay, uint32_t tou
   }
 }
 
-// Four entries per thread and iteration: every array is read and written with
-// 16-byte (or, for the byte arrays, 4-byte) accesses, consecutive threads touch
-// consecutive addresses.  touch and last_epoch are only written where an entry
-// was touched, so an idle pool costs reads of 14 bytes and writes of 8 bytes per
-// entry.
+struct Predictor {
+  uint64_t* hits;
+  uint64_t* misses;
+  float* P;
+  float alpha0, beta0;
+  unsigned long long* delta;   // [32] this epoch's counts, index 2*pair + hit
+  unsigned int* ticket;        // blocks that have finished (the last one commits)
+};
+
+// Posterior mean of Eq. "reuse" for pair p from the running totals plus this
+// epoch's counts: P = alpha / (alpha + beta), alpha = alpha0 + hits, beta =
+// beta0 + misses.  The 64-bit counts convert to binary32 with round to nearest
+// even; the division is IEEE.
+__device__ __forceinline__ float posterior(const Predictor& pd, unsigned p, unsigned long long& h,
+                                           unsigned long long& m) {
+  h = pd.hits[p] + pd.delta[2 * p + 1];
+  m = pd.misses[p] + pd.delta[2 * p];
+  const float a = __fadd_rn(pd.alpha0, __ull2float_rn(h));
+  const float b = __fadd_rn(pd.beta0, __ull2float_rn(m));
+  return __fdiv_rn(a, __fadd_rn(a, b));
+}
+
+// Every block forms the 16 posteriors itself (32 counters, read-only here), then
+// streams its share of the entries: four per thread and iteration, every array
+// read and written with 16-byte (for the byte arrays 4-byte) accesses.  touch and
+// last_epoch are only written where an entry was touched.  The last block to
+// finish folds the epoch's counts into the totals, clears them and publishes P;
+// by then every block has read them.
 __global__ void __launch_bounds__(kThreads)
 entry_update_kernel(float* __restrict__ ema, const float* __restrict__ decay,
                     uint32_t* __restrict__ touch, uint32_t* __restrict__ last_epoch,
                     const uint8_t* __restrict__ pair, const uint8_t* __restrict__ state,
-                    float* __restrict__ score, const float* __restrict__ P, uint64_t n,
-                    uint32_t epoch) {
+                    float* __restrict__ score, const Predictor pd, uint64_t n, uint32_t epoch) {
   __shared__ float sP[16];
-  if (threadIdx.x < 16) sP[threadIdx.x] = P[threadIdx.x];
+  __shared__ bool s_last;
+  if (threadIdx.x < 16) {
+    unsigned long long h, m;
+    sP[threadIdx.x] = posterior(pd, threadIdx.x, h, m);
+  }
   __syncthreads();
   const uint64_t n4 = n / 4;
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
@@ -161,16 +201,36 @@ entry_update_kernel(float* __restrict__ ema, const float* __restrict__ decay,
       last_epoch[i] = epoch;
     }
   }
+  // commit by the last block to finish
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    s_last = atomicAdd(pd.ticket, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (s_last && threadIdx.x < 16) {
+    const unsigned p = threadIdx.x;
+    unsigned long long h, m;
+    const float P = posterior(pd, p, h, m);
+    pd.hits[p] = h;
+    pd.misses[p] = m;
+    pd.P[p] = P;
+    pd.delta[2 * p] = 0;
+    pd.delta[2 * p + 1] = 0;
+    if (p == 0) *pd.ticket = 0;
+  }
 }
 
-cudaError_t launch_entry_update(const EntryState& st, const float* P, uint32_t epoch, cudaStream_t s) {
-  if (st.n == 0) return cudaSuccess;
+cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P,
+                                float alpha0, float beta0, const Workspace& ws, uint32_t epoch,
+                                cudaStream_t s) {
   uint64_t blocks = (st.n / 4 + kThreads - 1) / kThreads;
   if (blocks == 0) blocks = 1;
   const uint64_t cap = (uint64_t)kSMs * 8;
   if (blocks > cap) blocks = cap;
+  const Predictor pd{hits, misses, P, alpha0, beta0, ws.delta, &ws.sel->update_ticket};
   entry_update_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(st.ema, st.decay, st.touch, st.last_epoch,
-                                                            st.pair, st.state, st.score, P, st.n, epoch);
+                                                            st.pair, st.state, st.score, pd, st.n, epoch);
   count_launches(1);
   return cudaGetLastError();
 }

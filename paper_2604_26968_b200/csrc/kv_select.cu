@@ -334,6 +334,9 @@ __global__ void select_begin_kernel(SelectScalars* sel, unsigned long long k) {
   sel->need_eq = 0;
 }
 
+// 1 = one persistent cooperative launch (default), 0 = one launch per phase
+int g_select_variant = 1;
+
 static unsigned hist_grid(uint64_t n) {
   uint64_t blocks = (n / 4 + kThreads - 1) / kThreads;
   if (blocks == 0) blocks = 1;
@@ -344,6 +347,11 @@ static unsigned hist_grid(uint64_t n) {
 cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims, const Workspace& ws,
                           cudaStream_t s) {
   if (k == 0 || st.n == 0) return cudaSuccess;
+  if (g_select_variant == 1) {
+    bool used = false;
+    const cudaError_t e = launch_select_persistent(st, k, d_victims, ws, s, &used);
+    if (e != cudaSuccess || used) return e;
+  }
   const unsigned g = hist_grid(st.n);
   select_begin_kernel<<<1, 1, 0, s>>>(ws.sel, k);
   select_hist_kernel<0><<<g, kThreads, 0, s>>>(st.score, st.state, st.n, ws.sel, ws.hist);

@@ -1,0 +1,427 @@
+// k-lowest selection as ONE cooperative, persistent launch.
+//
+// The multi-launch selection in kv_select.cu spends most of its time between
+// kernels when the pool has a few million entries: ten dependent launches of
+// 3-10 us each.  Here one CTA per SM stays resident for the whole selection.
+// Each CTA owns a contiguous slice of the entries, converts its slice's scores
+// to order-preserving keys ONCE and keeps them in shared memory (up to 48 K keys
+// per SM, i.e. 7.2 M entries on 148 SMs; the rest of a larger slice is re-read
+// from the score array, which then sits in L2), and the phases of the radix
+// select -- three digit histograms, the count, the ordered write -- are separated
+// by grid-wide barriers instead of kernel boundaries.
+//
+// The grid barrier is a counter in global memory that every CTA increments and
+// then polls.  A cooperative launch guarantees that all CTAs are resident, so
+// the wait ends; it is nevertheless bounded, and a CTA that gives up sets
+// KV_DEV_WAIT_EXPIRED and leaves (every other CTA then runs into the same limit).
+#include "kvtier_internal.cuh"
+
+namespace kvt {
+
+constexpr uint32_t kPThreads = 1024;
+constexpr uint32_t kPChunk = kPThreads * 4;             // 4096 entries: one 16-byte vector per thread
+constexpr uint32_t kPKeyCap = 49152;                    // keys kept in shared memory per CTA (192 KB)
+constexpr uint32_t kPHistBins = 2048;
+constexpr uint32_t kExcluded = 0xFFFFFFFFu;             // key of a non-candidate (FREE) entry
+constexpr uint32_t kBarrierSpins = 1u << 22;
+
+static_assert(kPKeyCap % kPChunk == 0, "the cached part of a slice is a whole number of chunks");
+static_assert(kPKeyCap < 65536, "per-CTA counts of the cached part are packed in 16 bits");
+
+__device__ __forceinline__ uint32_t p_score_key(float s) {
+  uint32_t b = __float_as_uint(s);
+  if (b == 0x80000000u) b = 0u;  // -0.0 orders with +0.0
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Adds one to s_hist[bin] for every active lane; one atomic when the warp agrees
+// on the bin (the common case while most scores are equal).
+__device__ __forceinline__ void p_warp_hist_add(uint32_t* s_hist, bool active, uint32_t bin) {
+  const unsigned m = __ballot_sync(0xFFFFFFFFu, active);
+  if (m == 0) return;
+  const int leader = __ffs(m) - 1;
+  const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, bin, leader);
+  const bool same = !active || bin == b0;
+  if (__all_sync(0xFFFFFFFFu, same)) {
+    if ((int)(threadIdx.x & 31u) == leader) atomicAdd(&s_hist[b0], (uint32_t)__popc(m));
+  } else if (active) {
+    atomicAdd(&s_hist[bin], 1u);
+  }
+}
+
+struct PArgs {
+  const float* score;
+  const uint8_t* state;
+  unsigned long long n;
+  unsigned long long k;
+  uint32_t* victims;
+  uint32_t* hist;         // [3][2048], zero on entry, zero again on exit
+  SelectScalars* sel;
+  uint2* cta_counts;      // [gridDim.x]
+  uint32_t* status;
+  unsigned long long per; // entries per CTA slice (multiple of 4)
+};
+
+// Bounded grid-wide barrier; false if the wait ran out.
+__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int target) {
+  __shared__ int s_ok;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(counter, 1u);
+    int ok = 0;
+    for (uint32_t it = 0; it < kBarrierSpins; ++it) {
+      unsigned int v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+      if (v >= target) { ok = 1; break; }
+      __nanosleep(32);
+    }
+    s_ok = ok;
+    __threadfence();
+  }
+  __syncthreads();
+  return s_ok != 0;
+}
+
+// Block-wide exclusive scan over the 1024 threads; also returns the block total.
+__device__ __forceinline__ uint32_t block_scan_excl(uint32_t v, uint32_t* s_warp, uint32_t& total) {
+  const uint32_t t = threadIdx.x;
+  uint32_t incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if ((t & 31u) >= (uint32_t)o) incl += y;
+  }
+  __syncthreads();  // s_warp may still be read by the previous call's consumers
+  if ((t & 31u) == 31u) s_warp[t >> 5] = incl;
+  __syncthreads();
+  if (t < 32) {
+    uint32_t w = s_warp[t];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, w, o);
+      if (t >= (uint32_t)o) w += y;
+    }
+    s_warp[t] = w;
+  }
+  __syncthreads();
+  total = s_warp[31];
+  return incl - v + ((t >> 5) ? s_warp[(t >> 5) - 1] : 0u);
+}
+
+// Finds the bin of a global histogram (nbins <= 2048) that contains rank k_rem
+// (1-based) and returns (bin, ranks before the bin) to every thread; bin is
+// 0xFFFFFFFF when k_rem exceeds the histogram's total.
+__device__ __forceinline__ void pick_bin(const uint32_t* __restrict__ hist, uint32_t nbins,
+                                         unsigned long long k_rem, uint32_t* s_warp, uint32_t* s_pick,
+                                         uint32_t& bin, uint32_t& before_bin) {
+  const uint32_t t = threadIdx.x;
+  const uint32_t b0 = 2 * t, b1 = 2 * t + 1;
+  const uint32_t c0 = b0 < nbins ? __ldcg(&hist[b0]) : 0u;
+  const uint32_t c1 = b1 < nbins ? __ldcg(&hist[b1]) : 0u;
+  if (t == 0) { s_pick[0] = 0xFFFFFFFFu; s_pick[1] = 0; }
+  uint32_t total;
+  const uint32_t before = block_scan_excl(c0 + c1, s_warp, total);  // contains block barriers
+  if (c0 && (unsigned long long)before < k_rem && k_rem <= (unsigned long long)before + c0) {
+    s_pick[0] = b0; s_pick[1] = before;
+  }
+  const uint32_t before1 = before + c0;
+  if (c1 && (unsigned long long)before1 < k_rem && k_rem <= (unsigned long long)before1 + c1) {
+    s_pick[0] = b1; s_pick[1] = before1;
+  }
+  __syncthreads();
+  bin = s_pick[0];
+  before_bin = s_pick[1];
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const PArgs a) {
+  extern __shared__ __align__(16) uint32_t s_keys[];  // kPKeyCap keys
+  __shared__ uint32_t s_hist[kPHistBins];
+  __shared__ uint32_t s_warp[32];
+  __shared__ uint32_t s_pick[2];
+  const uint32_t t = threadIdx.x;
+  unsigned int* bar = &a.sel->bar_arrive;
+  const unsigned int G = gridDim.x;
+  const unsigned long long s0 = (unsigned long long)blockIdx.x * a.per;
+  const unsigned long long s1 = (s0 + a.per < a.n) ? s0 + a.per : a.n;
+  const uint32_t len = s1 > s0 ? (uint32_t)(s1 - s0) : 0u;
+  const uint32_t cached = len < kPKeyCap ? len : kPKeyCap;        // local [0, cached) lives in s_keys
+  const uint32_t first_far = kPKeyCap / kPChunk;                   // first chunk beyond the cache
+  const uint32_t n_chunks = (len + kPChunk - 1) / kPChunk;
+  bool ok = true;
+  auto stamp = [&](int i) {
+    if (blockIdx.x == 0 && t == 0) {
+      unsigned long long ns;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns));
+      a.sel->phase_ns[i] = ns;
+    }
+  };
+  stamp(0);
+
+  // keys of the thread's vector (4 entries) of chunk c, computed from the arrays;
+  // entries past the slice or not RESIDENT give kExcluded
+  auto keys_from_arrays = [&](uint32_t c, uint32_t key[4]) {
+    const uint32_t j0 = c * kPChunk + 4u * t;
+    const unsigned long long i0 = s0 + j0;
+    if (j0 + 4 <= len) {
+      const float4 sc = __ldcg(reinterpret_cast<const float4*>(a.score + i0));
+      const uchar4 st = __ldcg(reinterpret_cast<const uchar4*>(a.state + i0));
+      key[0] = st.x == KV_STATE_RESIDENT ? p_score_key(sc.x) : kExcluded;
+      key[1] = st.y == KV_STATE_RESIDENT ? p_score_key(sc.y) : kExcluded;
+      key[2] = st.z == KV_STATE_RESIDENT ? p_score_key(sc.z) : kExcluded;
+      key[3] = st.w == KV_STATE_RESIDENT ? p_score_key(sc.w) : kExcluded;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        key[j] = (j0 + j < len && a.state[i0 + j] == KV_STATE_RESIDENT) ? p_score_key(a.score[i0 + j])
+                                                                        : kExcluded;
+    }
+  };
+
+  // Applies f(key) to every key of the slice, all threads in lock step (f may
+  // vote across the warp): the cached part with a stride of one block, the far
+  // part chunk by chunk from the arrays.
+  auto for_each_key = [&](auto f) {
+    const uint32_t iters = (cached + kPThreads - 1) / kPThreads;
+    for (uint32_t i = 0; i < iters; ++i) {
+      const uint32_t j = i * kPThreads + t;
+      f(j < cached ? s_keys[j] : kExcluded);
+    }
+    for (uint32_t c = first_far; c < n_chunks; ++c) {
+      uint32_t key[4];
+      keys_from_arrays(c, key);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) f(key[j]);
+    }
+  };
+  auto clear_hist = [&]() {
+    for (uint32_t b = t; b < kPHistBins; b += kPThreads) s_hist[b] = 0;
+    __syncthreads();
+  };
+  auto flush_hist = [&](uint32_t* g_hist, uint32_t nbins) {
+    __syncthreads();
+    for (uint32_t b = t; b < nbins; b += kPThreads) {
+      const uint32_t c = s_hist[b];
+      if (c) atomicAdd(&g_hist[b], c);
+    }
+  };
+
+  // ---- phase A: keys into shared memory, then the histogram of digit 0 (bits 31..21) ----
+  clear_hist();
+  {
+    const uint32_t cached_chunks = (cached + kPChunk - 1) / kPChunk;
+#pragma unroll 4
+    for (uint32_t c = 0; c < cached_chunks; ++c) {
+      uint32_t key[4];
+      keys_from_arrays(c, key);
+      reinterpret_cast<uint4*>(s_keys)[c * kPThreads + t] = make_uint4(key[0], key[1], key[2], key[3]);
+    }
+    __syncthreads();
+  }
+  for_each_key([&](uint32_t key) { p_warp_hist_add(s_hist, key != kExcluded, key >> 21); });
+  flush_hist(a.hist, 2048);
+  stamp(1);
+  ok = grid_barrier(bar, G);
+  stamp(2);
+  if (!ok) goto fail;
+
+  {
+    // ---- phase B: fix digit 0, histogram of digit 1 (bits 20..10) ----
+    uint32_t bin, before;
+    unsigned long long k_rem = a.k;
+    pick_bin(a.hist, 2048, k_rem, s_warp, s_pick, bin, before);
+    const bool found0 = bin != 0xFFFFFFFFu;
+    uint32_t prefix = bin << 21;
+    k_rem -= before;
+    clear_hist();
+    for_each_key([&](uint32_t key) {
+      p_warp_hist_add(s_hist, key != kExcluded && (key & 0xFFE00000u) == prefix, (key >> 10) & 2047u);
+    });
+    flush_hist(a.hist + kPHistBins, 2048);
+    ok = grid_barrier(bar, 2 * G);
+    stamp(3);
+    if (!ok) goto fail;
+    if (blockIdx.x == 0)
+      for (uint32_t b = t; b < 2048; b += kPThreads) a.hist[b] = 0;  // nobody reads digit 0 any more
+
+    // ---- phase C: fix digit 1, histogram of digit 2 (bits 9..0) ----
+    pick_bin(a.hist + kPHistBins, 2048, k_rem, s_warp, s_pick, bin, before);
+    const bool found1 = bin != 0xFFFFFFFFu;
+    prefix |= (bin & 2047u) << 10;
+    k_rem -= before;
+    clear_hist();
+    for_each_key([&](uint32_t key) {
+      p_warp_hist_add(s_hist, key != kExcluded && (key & 0xFFFFFC00u) == prefix, key & 1023u);
+    });
+    flush_hist(a.hist + 2 * kPHistBins, 1024);
+    ok = grid_barrier(bar, 3 * G);
+    stamp(4);
+    if (!ok) goto fail;
+    if (blockIdx.x == 0)
+      for (uint32_t b = t; b < 2048; b += kPThreads) a.hist[kPHistBins + b] = 0;
+
+    // ---- phase D: fix digit 2 -> tau; count (key < tau, key == tau) in the slice ----
+    pick_bin(a.hist + 2 * kPHistBins, 1024, k_rem, s_warp, s_pick, bin, before);
+    const bool found = found0 && found1 && bin != 0xFFFFFFFFu;
+    const uint32_t tau = prefix | (bin & 1023u);
+    const unsigned long long need_eq = k_rem - before;
+    {
+      uint32_t n_less = 0, n_eq = 0;
+      for_each_key([&](uint32_t key) {
+        n_less += (key != kExcluded && key < tau);
+        n_eq += (key != kExcluded && key == tau);
+      });
+      uint32_t tot_less, tot_eq;
+      (void)block_scan_excl(n_less, s_warp, tot_less);
+      (void)block_scan_excl(n_eq, s_warp, tot_eq);
+      if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(tot_less, tot_eq);
+    }
+    stamp(5);
+    ok = grid_barrier(bar, 4 * G);
+    stamp(6);
+    if (!ok) goto fail;
+    if (blockIdx.x == 0)
+      for (uint32_t b = t; b < 2048; b += kPThreads) a.hist[2 * kPHistBins + b] = 0;
+
+    // ---- phase E: ordered write ----
+    unsigned long long less_before, eq_before;
+    {
+      uint32_t la = 0, ea = 0;  // partial sums over the CTAs before this one
+      for (uint32_t g = t; g < blockIdx.x; g += kPThreads) {
+        const uint2 cc = __ldcg(&a.cta_counts[g]);
+        la += cc.x; ea += cc.y;
+      }
+      uint32_t tl, te;
+      (void)block_scan_excl(la, s_warp, tl);
+      (void)block_scan_excl(ea, s_warp, te);
+      less_before = tl; eq_before = te;
+    }
+    auto emit = [&](uint32_t key, unsigned long long id, unsigned long long& n1, unsigned long long& n2) {
+      if (key == kExcluded) return;
+      if (key < tau) {
+        const unsigned long long pos = n1 + (n2 < need_eq ? n2 : need_eq);
+        if (pos < a.k) a.victims[pos] = (uint32_t)id;
+        ++n1;
+      } else if (key == tau) {
+        if (n2 < need_eq) {
+          const unsigned long long pos = n1 + n2;
+          if (pos < a.k) a.victims[pos] = (uint32_t)id;
+        }
+        ++n2;
+      }
+    };
+    if (found) {
+      // cached part: every thread owns a contiguous run of L keys (L odd: the
+      // strided shared-memory reads of a warp then fall into distinct banks)
+      {
+        uint32_t L = (cached + kPThreads - 1) / kPThreads;
+        L |= 1u;
+        const uint32_t j0 = t * L;
+        const uint32_t j1 = (j0 + L < cached) ? j0 + L : cached;
+        uint32_t v = 0;
+        for (uint32_t j = j0; j < j1; ++j) {
+          const uint32_t key = s_keys[j];
+          v += (key != kExcluded && key < tau) + ((uint32_t)(key != kExcluded && key == tau) << 16);
+        }
+        uint32_t total;
+        const uint32_t excl = block_scan_excl(v, s_warp, total);
+        unsigned long long n1 = less_before + (excl & 0xFFFFu), n2 = eq_before + (excl >> 16);
+        for (uint32_t j = j0; j < j1; ++j) emit(s_keys[j], s0 + j, n1, n2);
+        less_before += total & 0xFFFFu;
+        eq_before += total >> 16;
+      }
+      // far part: chunk by chunk, a vector per thread
+      for (uint32_t c = first_far; c < n_chunks; ++c) {
+        uint32_t key[4];
+        keys_from_arrays(c, key);
+        uint32_t v = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          v += (key[j] != kExcluded && key[j] < tau) + ((uint32_t)(key[j] != kExcluded && key[j] == tau) << 16);
+        uint32_t total;
+        const uint32_t excl = block_scan_excl(v, s_warp, total);
+        unsigned long long n1 = less_before + (excl & 0xFFFFu), n2 = eq_before + (excl >> 16);
+        const unsigned long long i0 = s0 + (unsigned long long)c * kPChunk + 4ull * t;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) emit(key[j], i0 + j, n1, n2);
+        less_before += total & 0xFFFFu;
+        eq_before += total >> 16;
+      }
+    }
+    if (blockIdx.x == G - 1 && t == 0) {
+      // every entry has been counted: the selection must hold exactly k ids
+      unsigned long long tl = 0, te = 0;
+      for (uint32_t g = 0; g < G; ++g) { const uint2 cc = __ldcg(&a.cta_counts[g]); tl += cc.x; te += cc.y; }
+      const unsigned long long got = tl + (te < need_eq ? te : need_eq);
+      if (!found || got != a.k) atomicOr(a.status, KV_DEV_SELECT_MISMATCH);
+      a.sel->tau = tau;
+      a.sel->need_eq = need_eq;
+    }
+  }
+  stamp(7);
+  goto done;
+
+fail:
+  if (t == 0) atomicOr(a.status, KV_DEV_WAIT_EXPIRED);
+done:
+  // the last CTA to leave resets the barrier for the next launch
+  __syncthreads();
+  if (t == 0) {
+    __threadfence();
+    const unsigned int old = atomicAdd(&a.sel->bar_done, 1u);
+    if (old == G - 1) {
+      a.sel->bar_arrive = 0;
+      a.sel->bar_done = 0;
+      __threadfence();
+    }
+  }
+}
+
+// Launches the persistent selection if the device can hold one CTA per SM of it
+// co-resident; *used = false (and nothing launched) otherwise.
+cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
+                                     const Workspace& ws, cudaStream_t s, bool* used) {
+  *used = false;
+  static int state = 0;  // 0 = not probed, 1 = usable, -1 = not usable
+  static int n_sm = 0;
+  const size_t smem = (size_t)kPKeyCap * 4;
+  if (state == 0) {
+    int dev = 0, coop = 0, blocks = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t e = cudaFuncSetAttribute(select_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e == cudaSuccess)
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, select_persistent_kernel, (int)kPThreads, smem);
+    state = (e == cudaSuccess && coop && blocks >= 1 && n_sm > 0) ? 1 : -1;
+    (void)cudaGetLastError();
+  }
+  if (state != 1) return cudaSuccess;
+  unsigned int G = (unsigned int)n_sm;
+  const uint64_t min_per = kPChunk;  // do not spread tiny pools over more CTAs than they have chunks
+  if ((st.n + min_per - 1) / min_per < G) G = (unsigned int)((st.n + min_per - 1) / min_per);
+  if (G == 0) G = 1;
+  if (G + 2 > ws.n_tiles) return cudaSuccess;  // cta_counts live in the tile-count scratch
+  PArgs a;
+  a.score = st.score;
+  a.state = st.state;
+  a.n = st.n;
+  a.k = k;
+  a.victims = d_victims;
+  a.hist = ws.hist;
+  a.sel = ws.sel;
+  a.cta_counts = ws.tile_counts;
+  a.status = ws.status;
+  a.per = ((st.n + G - 1) / G + 3) / 4 * 4;
+  void* args[] = {&a};
+  cudaError_t e = cudaLaunchCooperativeKernel((void*)select_persistent_kernel, dim3(G), dim3(kPThreads), args,
+                                              smem, s);
+  if (e != cudaSuccess) return e;
+  count_launches(1);
+  *used = true;
+  return cudaSuccess;
+}
+
+}  // namespace kvt

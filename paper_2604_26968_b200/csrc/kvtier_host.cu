@@ -410,9 +410,8 @@ uint64_t* kv_epoch_counts(kv_pool* p) {
 
 int32_t kv_epoch_update(kv_pool* p, uint32_t epoch, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
-  KV_CUDA(p, launch_posterior(p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
-                              p->desc.beta0, p->ws, S(stream)));
-  KV_CUDA(p, launch_entry_update(p->st, p->desc.d_P, epoch, S(stream)));
+  KV_CUDA(p, launch_entry_update(p->st, p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
+                                 p->desc.beta0, p->ws, epoch, S(stream)));
   p->stats.epochs += 1;
   return KV_OK;
 }
@@ -656,6 +655,12 @@ int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) 
 int32_t kv_set_move_variant(int32_t variant) {
   if (variant != 0 && variant != 1) return KV_ERR_INVALID_ARG;
   g_move_variant = variant;
+  return KV_OK;
+}
+
+int32_t kv_set_select_variant(int32_t variant) {
+  if (variant != 0 && variant != 1) return KV_ERR_INVALID_ARG;
+  kvt::g_select_variant = variant;
   return KV_OK;
 }
 

@@ -56,8 +56,11 @@ struct SelectScalars {
   uint32_t tau;           // key of the k-th smallest entry
   unsigned long long k_rem;    // rank still to resolve inside the current bucket
   unsigned long long need_eq;  // how many entries with key == tau are taken
-  unsigned long long written;  // entries written by the last compaction
-  unsigned long long pad;
+  unsigned int bar_arrive;     // grid barrier of the persistent selection: arrivals
+  unsigned int bar_done;       // ... and CTAs that have left (the last one resets both)
+  unsigned int update_ticket;  // blocks of the entry pass that have finished (the last one commits)
+  unsigned int pad;
+  unsigned long long phase_ns[8];  // %globaltimer at the phase boundaries of the last persistent selection (CTA 0)
 };
 
 struct Workspace {
@@ -76,13 +79,20 @@ struct Workspace {
 // ---- kv_score.cu ----
 cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit, uint64_t n_events,
                                 const EntryState& st, const Workspace& ws, cudaStream_t s);
-cudaError_t launch_posterior(uint64_t* hits, uint64_t* misses, float* P, float alpha0, float beta0,
-                             const Workspace& ws, cudaStream_t s);
-cudaError_t launch_entry_update(const EntryState& st, const float* P, uint32_t epoch, cudaStream_t s);
+// posterior (from hits/misses plus the epoch counters in ws.delta) + EMA + score in one launch;
+// folds ws.delta into hits/misses, clears it and writes P
+cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P,
+                                float alpha0, float beta0, const Workspace& ws, uint32_t epoch,
+                                cudaStream_t s);
 
 // ---- kv_select.cu ----
 cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims, const Workspace& ws,
                           cudaStream_t s);
+extern int g_select_variant;  // which selection launch_select uses (see kv_select.cu)
+// kv_select_persist.cu: the same selection as one cooperative launch; *used tells
+// whether it was launched (false: the device cannot co-schedule it, nothing was enqueued)
+cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
+                                     const Workspace& ws, cudaStream_t s, bool* used);
 // ascending ids of FREE entries in [lo, hi), at most `limit` of them, into ws.free_list
 cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uint64_t limit,
                              const Workspace& ws, cudaStream_t s);
