@@ -21,8 +21,12 @@
  *   - the caller allocates ALL memory (device, pinned host) and the streams;
  *     the library allocates no device memory and never synchronises the device;
  *     GPU work is enqueued on the given streams and results are valid once the
- *     caller has synchronised them.  Use the same compute and copy streams for
- *     every call on one pool (or order differing streams yourself);
+ *     caller has synchronised them.  Use ONE compute stream for every call on a
+ *     pool.  kv_demote and kv_promote each take a copy stream; give kv_promote a
+ *     different one than kv_demote and the H2D copies of a promotion overlap the
+ *     D2H copies of the demotion before it (the library orders the two streams
+ *     wherever a promotion reads ring slots that a demotion is still writing,
+ *     and the other way round); keep each call's copy stream the same over time;
  *   - device and pinned pointers must be 16-byte aligned;
  *   - functions return KV_OK (0) or a negative kv_status; on a negative status
  *     detected by the host nothing has been enqueued and no state has changed;
@@ -149,8 +153,9 @@ typedef struct {
   /* block table (device): d_loc[tag] = entry id, KV_LOC_HOST|ring slot, or KV_NONE */
   uint32_t* d_loc;
   uint64_t n_tags;
-  /* two device staging buffers of staging_bytes each */
-  void* d_staging[2];
+  /* four device staging buffers of staging_bytes each: [0],[1] double-buffer the
+   * demotions, [2],[3] the promotions */
+  void* d_staging[4];
   uint64_t staging_bytes;
   uint64_t max_promote; /* longest promote list this pool will be given */
   /* scratch of the sizes kv_workspace_bytes reports */

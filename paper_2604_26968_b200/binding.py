@@ -49,7 +49,7 @@ class kv_pool_desc(C.Structure):
                 ("d_hits", C.c_void_p), ("d_misses", C.c_void_p), ("d_P", C.c_void_p),
                 ("alpha0", C.c_float), ("beta0", C.c_float),
                 ("d_loc", C.c_void_p), ("n_tags", C.c_uint64),
-                ("d_staging", C.c_void_p * 2), ("staging_bytes", C.c_uint64),
+                ("d_staging", C.c_void_p * 4), ("staging_bytes", C.c_uint64),
                 ("max_promote", C.c_uint64),
                 ("d_workspace", C.c_void_p), ("workspace_bytes", C.c_uint64),
                 ("h_workspace", C.c_void_p), ("h_workspace_bytes", C.c_uint64)]
@@ -232,7 +232,7 @@ class Pool:
         self.misses = dz(16, torch.int64)
         self.P = dz(16, torch.float32)
         self.loc = dz(self.n_tags, torch.int32)
-        self.staging = [torch.empty(self.staging_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+        self.staging = [torch.empty(self.staging_bytes, dtype=torch.uint8, device=dev) for _ in range(4)]
         self.slabs, self.rings, self.metas = [], [], []
         d = kv_pool_desc()
         d.n_partitions = len(self.parts)
@@ -254,7 +254,8 @@ class Pool:
         d.d_hits, d.d_misses, d.d_P = self.hits.data_ptr(), self.misses.data_ptr(), self.P.data_ptr()
         d.alpha0, d.beta0 = alpha0, beta0
         d.d_loc, d.n_tags = self.loc.data_ptr(), self.n_tags
-        d.d_staging[0], d.d_staging[1] = self.staging[0].data_ptr(), self.staging[1].data_ptr()
+        for b in range(4):
+            d.d_staging[b] = self.staging[b].data_ptr()
         d.staging_bytes = self.staging_bytes
         d.max_promote = self.max_promote
         dev_b, host_b = C.c_uint64(0), C.c_uint64(0)
@@ -267,7 +268,8 @@ class Pool:
         d.h_workspace, d.h_workspace_bytes = self.h_workspace.data_ptr(), host_b.value
         self.desc = d
         self.compute = stream if stream is not None else torch.cuda.Stream(device=dev)
-        self.copy = torch.cuda.Stream(device=dev)
+        self.copy = torch.cuda.Stream(device=dev)        # D2H copies of demotions
+        self.copy_h2d = torch.cuda.Stream(device=dev)    # H2D copies of promotions (overlap the D2H ones)
         self._h = C.c_void_p()
         with torch.cuda.device(dev):
             rc = self.lib.kv_pool_create(C.byref(d), _stream_ptr(self.compute), C.byref(self._h))
@@ -289,6 +291,7 @@ class Pool:
     def sync(self):
         self.compute.synchronize()
         self.copy.synchronize()
+        self.copy_h2d.synchronize()
 
     # -- the five calls, plus the harness extras; each returns the status --------
     def kv_epoch_score(self, epoch, d_ev_entry, d_ev_hit, n_events=None):
@@ -323,7 +326,7 @@ class Pool:
         h_slots = np.ascontiguousarray(h_slots, dtype=np.uint64)
         return self.lib.kv_promote(self._h, partition, h_slots.ctypes.data_as(C.c_void_p) if h_slots.size else None,
                                    h_slots.size, int(batch_bytes), _stream_ptr(self.compute),
-                                   _stream_ptr(self.copy))
+                                   _stream_ptr(self.copy_h2d))
 
     def kv_admit(self, epoch, decay, d_new_pairs, fill_pattern=True):
         n = C.c_uint64(0)

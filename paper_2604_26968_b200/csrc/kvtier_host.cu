@@ -80,7 +80,7 @@ struct kv_pool {
   uint64_t bases[5] = {0, 0, 0, 0, 0};
   EntryState st;
   Workspace ws;
-  uint8_t* staging[2] = {nullptr, nullptr};
+  uint8_t* staging[4] = {nullptr, nullptr, nullptr, nullptr};  // [0,1] demotion, [2,3] promotion
   uint64_t staging_bytes = 0;
   uint64_t max_promote = 0;
   uint32_t* h_list[2] = {nullptr, nullptr};
@@ -89,9 +89,15 @@ struct kv_pool {
   uint64_t next_tag = 0;
   kv_stats stats;
   uint64_t last_counts[4] = {0, 0, 0, 0};
-  cudaEvent_t ev_staging_free[2], ev_ready[2], ev_list_copied[2], ev_list_free[2], ev_counts;
+  cudaEvent_t ev_staging_free[4], ev_ready[4], ev_list_copied[2], ev_list_free[2], ev_counts;
+  // copies in flight: the last two demotions per partition (ring slot range + completion event of
+  // their D2H copies) and the last promotion's H2D copies
+  struct D2H { cudaEvent_t ev; uint64_t start = 0, count = 0; bool valid = false; };
+  D2H d2h[4][2];
+  cudaEvent_t ev_h2d_done;
+  bool h2d_valid = false;
   bool events_made = false;
-  int staging_turn = 0, list_turn = 0;
+  int demote_turn = 0, promote_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
   // optional per-launch timing of the pack / unpack kernels
   struct Timed { cudaEvent_t a, b; int kind; uint64_t bytes; bool pending; };
@@ -283,7 +289,8 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
   if (!(desc->alpha0 > 0.0f) || !(desc->beta0 > 0.0f)) return KV_ERR_INVALID_ARG;
   const void* need[] = {desc->d_ema, desc->d_decay, desc->d_touch, desc->d_last_epoch, desc->d_pair,
                         desc->d_state, desc->d_tag, desc->d_score, desc->d_hits, desc->d_misses,
-                        desc->d_P, desc->d_staging[0], desc->d_staging[1], desc->d_workspace,
+                        desc->d_P, desc->d_staging[0], desc->d_staging[1], desc->d_staging[2], desc->d_staging[3],
+                        desc->d_workspace,
                         desc->h_workspace};
   for (const void* p : need)
     if (!p || !aligned16(p)) return KV_ERR_INVALID_ARG;
@@ -349,14 +356,17 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
     ph.h_ring = static_cast<uint8_t*>(desc->part[q].h_ring);
     ph.h_meta = static_cast<uint8_t*>(desc->part[q].h_meta);
   }
-  p->staging[0] = static_cast<uint8_t*>(desc->d_staging[0]);
-  p->staging[1] = static_cast<uint8_t*>(desc->d_staging[1]);
+  for (int b = 0; b < 4; ++b) p->staging[b] = static_cast<uint8_t*>(desc->d_staging[b]);
   p->staging_bytes = desc->staging_bytes;
   p->max_promote = desc->max_promote;
   p->stats.n_entries = g.N;
   p->stats.n_free = g.N;
 
   cudaEvent_t* evs[] = {&p->ev_staging_free[0], &p->ev_staging_free[1], &p->ev_ready[0], &p->ev_ready[1],
+                        &p->ev_staging_free[2], &p->ev_staging_free[3], &p->ev_ready[2], &p->ev_ready[3],
+                        &p->d2h[0][0].ev, &p->d2h[0][1].ev, &p->d2h[1][0].ev, &p->d2h[1][1].ev,
+                        &p->d2h[2][0].ev, &p->d2h[2][1].ev, &p->d2h[3][0].ev, &p->d2h[3][1].ev,
+                        &p->ev_h2d_done,
                         &p->ev_list_copied[0], &p->ev_list_copied[1], &p->ev_list_free[0],
                         &p->ev_list_free[1], &p->ev_counts};
   int made = 0;
@@ -385,6 +395,10 @@ int32_t kv_pool_destroy(kv_pool* p) {
   if (!p) return KV_ERR_INVALID_ARG;
   if (p->events_made) {
     cudaEvent_t evs[] = {p->ev_staging_free[0], p->ev_staging_free[1], p->ev_ready[0], p->ev_ready[1],
+                         p->ev_staging_free[2], p->ev_staging_free[3], p->ev_ready[2], p->ev_ready[3],
+                         p->d2h[0][0].ev, p->d2h[0][1].ev, p->d2h[1][0].ev, p->d2h[1][1].ev,
+                         p->d2h[2][0].ev, p->d2h[2][1].ev, p->d2h[3][0].ev, p->d2h[3][1].ev,
+                         p->ev_h2d_done,
                          p->ev_list_copied[0], p->ev_list_copied[1], p->ev_list_free[0],
                          p->ev_list_free[1], p->ev_counts};
     for (cudaEvent_t ev : evs) cudaEventDestroy(ev);
@@ -470,6 +484,8 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
     per[q] = entries_per_batch(p, q, batch_bytes);
     if (per[q] == 0 || batch_bytes > p->staging_bytes) return KV_ERR_INVALID_ARG;
   }
+  // ring slots written below may have been read by the last promotion's H2D copies
+  if (p->h2d_valid) KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_h2d_done, 0));
   uint64_t off = 0;
   for (int q = 0; q < p->n_parts; ++q) {
     const PartGeom& g = p->geom[q];
@@ -477,8 +493,8 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
     const uint64_t eb = g.entry_bytes, R = g.ring_slots;
     for (uint64_t c0 = 0; c0 < kq[q]; c0 += per[q]) {
       const uint64_t cnt = (kq[q] - c0 < per[q]) ? kq[q] - c0 : per[q];
-      const int b = p->staging_turn;
-      p->staging_turn ^= 1;
+      const int b = p->demote_turn;
+      p->demote_turn ^= 1;
       KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_staging_free[b], 0));
       const uint64_t meta_off = h.h_meta ? align_up(cnt * eb, 16) : ~0ull;
       const uint64_t slot0 = (h.cursor + c0) % R;
@@ -505,6 +521,15 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
                                      (cnt - first) * mb, cudaMemcpyDeviceToHost, copy));
       }
       KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], copy));
+    }
+    if (kq[q] > 0) {  // remember which slots this demotion's copies are writing, and when they are done
+      kv_pool::D2H older = p->d2h[q][1];
+      p->d2h[q][1] = p->d2h[q][0];
+      p->d2h[q][0] = older;  // reuse the older record's event object
+      p->d2h[q][0].start = h.cursor;
+      p->d2h[q][0].count = kq[q];
+      p->d2h[q][0].valid = true;
+      KV_CUDA(p, cudaEventRecord(p->d2h[q][0].ev, copy));
     }
     // host mirror of the ring: overwritten live slots are dropped
     for (uint64_t j = 0; j < kq[q]; ++j) {
@@ -555,8 +580,17 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
   auto restore = [&]() { for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 1; };
   cudaError_t e = cudaEventSynchronize(p->ev_list_copied[li]);  // the pinned list buffer is ours again
   if (e != cudaSuccess) { restore(); return cuda_fail(p, e); }
-  for (uint64_t j = 0; j < m; ++j) p->h_list[li][j] = (uint32_t)h_slots[j];
-  e = cudaStreamWaitEvent(copy, p->ev_list_free[li], 0);  // older kernels are done reading the device list
+  bool newest = false;  // does the list name a slot that the newest demotion's copies are still writing?
+  const kv_pool::D2H& d0 = p->d2h[q][0];
+  for (uint64_t j = 0; j < m; ++j) {
+    p->h_list[li][j] = (uint32_t)h_slots[j];
+    if (d0.valid && (h_slots[j] + R - d0.start) % R < d0.count) newest = true;
+  }
+  // the H2D copies below may run on another stream than the D2H copies that filled the slots
+  if (e == cudaSuccess && newest) e = cudaStreamWaitEvent(copy, d0.ev, 0);
+  if (e == cudaSuccess && !newest && p->d2h[q][1].valid) e = cudaStreamWaitEvent(copy, p->d2h[q][1].ev, 0);
+  if (e == cudaSuccess)
+    e = cudaStreamWaitEvent(copy, p->ev_list_free[li], 0);  // older kernels are done reading the device list
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(p->ws.slot_list[li], p->h_list[li], m * 4, cudaMemcpyHostToDevice, copy);
   if (e == cudaSuccess) e = cudaEventRecord(p->ev_list_copied[li], copy);
@@ -564,8 +598,8 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
   if (e != cudaSuccess) { restore(); return cuda_fail(p, e); }
   for (uint64_t c0 = 0; c0 < m; c0 += per) {
     const uint64_t cnt = (m - c0 < per) ? m - c0 : per;
-    const int b = p->staging_turn;
-    p->staging_turn ^= 1;
+    const int b = 2 + p->promote_turn;
+    p->promote_turn ^= 1;
     KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_staging_free[b], 0));
     // runs of consecutive ring slots become single copies
     uint64_t j = 0;
@@ -588,6 +622,8 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
     KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], compute));
   }
   KV_CUDA(p, cudaEventRecord(p->ev_list_free[li], compute));
+  KV_CUDA(p, cudaEventRecord(p->ev_h2d_done, copy));
+  p->h2d_valid = true;
   for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 0;
   h.n_live -= m;
   h.n_free -= m;

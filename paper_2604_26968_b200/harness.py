@@ -72,7 +72,7 @@ class EpochRunner:
         for q, p in enumerate(self.w.parts):
             cur, n_live, live = self.pool.kv_ring_query(q)
             m_q = min(int(self.w.promote_frac * p.n_entries), counts[q], int(n_live))
-            out.append(self.w.promote_list(epoch, q, m_q, cur, live))
+            out.append(self.w.promote_list(epoch, q, m_q, cur, live, just_written=counts[q]))
         return out
 
     def step(self, epoch, d_ev_entry, d_ev_hit, n_events, promote_lists=None, admit=True):

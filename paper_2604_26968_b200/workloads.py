@@ -160,12 +160,22 @@ class Workload:
             ev_hit = np.concatenate([ev_hit, np.zeros(len(fresh), np.uint8)])
         return ev_entry, ev_hit
 
-    def promote_list(self, epoch: int, q: int, m: int, cursor: int, live: np.ndarray) -> np.ndarray:
-        """Host ring slots (u64) to promote into partition q; all live, distinct."""
+    def promote_list(self, epoch: int, q: int, m: int, cursor: int, live: np.ndarray,
+                     just_written: int = 0) -> np.ndarray:
+        """Host ring slots (u64) to promote into partition q; all live, distinct.
+
+        just_written is the number of slots, ending at the cursor, that this epoch's
+        demotion wrote: a prefetcher does not ask back what was evicted a moment ago,
+        so the "runs" style leaves them out when enough older slots are live."""
         m = int(min(m, int(live.sum())))
         if m <= 0:
             return np.zeros(0, np.uint64)
         R = live.size
+        if self.promote_style != "recent" and just_written > 0:
+            idx = (cursor - 1 - np.arange(min(just_written, R))) % R
+            if int(live.sum()) - int(live[idx].sum()) >= m:
+                live = live.copy()
+                live[idx] = 0
         if self.promote_style == "recent":
             # the m most recently written live slots, oldest first
             order = (cursor - 1 - np.arange(R)) % R

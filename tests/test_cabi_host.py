@@ -108,7 +108,7 @@ def test_bad_descriptions_are_refused_without_cuda():
     for f in ("d_ema", "d_decay", "d_touch", "d_last_epoch", "d_pair", "d_state", "d_tag", "d_score",
               "d_hits", "d_misses", "d_P", "d_workspace", "h_workspace"):
         setattr(d, f, 0x1000)
-    d.d_staging[0] = d.d_staging[1] = 0x1000
+    d.d_staging[0] = d.d_staging[1] = d.d_staging[2] = d.d_staging[3] = 0x1000
     d.part[0].d_slab = 0x1008                     # not 16-byte aligned
     d.part[0].h_ring = 0x1000
     d.staging_bytes = 1 << 20
