@@ -160,6 +160,13 @@ struct Pool {
   int64_t N = 0;
   int payload = 0;
   float alpha0 = 1.0f, beta0 = 1.0f;
+  int policy = 0;                 // 0 Bayesian, 1 EMA only, 2 LRU
+  float kappa = 0.0f;             // confidence saturation constant
+  int window = 0;                 // epochs in the sliding window; 0 = no blending
+  int win_head = 0;
+  std::vector<uint64_t> win;      // [window][32] per-epoch counts, index 2*pair + hit
+  uint64_t wsum[32] = {0};        // sums over the window
+  float estimate[16] = {0};       // reuse estimate used for scoring
   std::vector<float> ema, decay, score;
   std::vector<uint32_t> touch, last_epoch, tag;
   std::vector<uint8_t> pair, state;
@@ -289,6 +296,7 @@ void* okv_create(int32_t n_parts, const PartDesc* parts, float alpha0, float bet
   for (int i = 0; i < 16; ++i) {
     p->hits[i] = p->misses[i] = 0;
     p->P[i] = alpha0 / (alpha0 + beta0);
+    p->estimate[i] = p->P[i];
   }
   p->loc.assign((size_t)n_tags, NONE);
   return p;
@@ -372,6 +380,28 @@ void okv_get_stats(void* h, uint64_t* out8) {
 
 uint64_t okv_next_tag(void* h) { return static_cast<Pool*>(h)->next_tag; }
 
+// Eviction policy: 0 Bayesian (default), 1 EMA only, 2 LRU.
+int32_t okv_set_policy(void* h, int32_t policy) {
+  if (policy < 0 || policy > 2) return ERR_INVALID_ARG;
+  static_cast<Pool*>(h)->policy = policy;
+  return OK;
+}
+
+// Confidence-weighted blend; window == 0 switches it off.  Resets the window.
+int32_t okv_set_confidence_blend(void* h, float kappa, int32_t window) {
+  Pool* p = static_cast<Pool*>(h);
+  if (window < 0 || window > 64 || (window > 0 && !(kappa > 0.0f))) return ERR_INVALID_ARG;
+  p->kappa = kappa;
+  p->window = window;
+  p->win_head = 0;
+  p->win.assign((size_t)window * 32, 0);
+  for (int i = 0; i < 32; ++i) p->wsum[i] = 0;
+  return OK;
+}
+
+// The 16 reuse estimates used by the Bayesian score (the posterior, or its blend).
+float* okv_estimate(void* h) { return static_cast<Pool*>(h)->estimate; }
+
 // One epoch of scoring, in the order update-then-decide:
 //   1. every observed event adds one to alpha (reuse) or beta (miss) of the
 //      entry's (block-type, transition-type) pair, and counts a touch;
@@ -390,10 +420,11 @@ int32_t okv_epoch_score(void* h, uint32_t epoch, const uint32_t* ev_entry, const
       return ERR_INVALID_ARG;
   }
   // step 1
+  uint64_t epoch_hits[16] = {0}, epoch_misses[16] = {0};
   for (uint64_t e = 0; e < n_events; ++e) {
     uint32_t i = ev_entry[e];
     uint8_t pr = p->pair[i];
-    if (ev_hit[e]) p->hits[pr] += 1; else p->misses[pr] += 1;
+    if (ev_hit[e]) { p->hits[pr] += 1; epoch_hits[pr] += 1; } else { p->misses[pr] += 1; epoch_misses[pr] += 1; }
     p->touch[i] += 1;
   }
   // step 2
@@ -414,12 +445,48 @@ int32_t okv_epoch_score(void* h, uint32_t epoch, const uint32_t* ev_entry, const
     float b = p->beta0 + (float)p->misses[pr];
     p->P[pr] = a / (a + b);
   }
-  // step 4
+  // step 3b (optional): confidence-weighted blend of the posterior with the
+  // empirical hit frequency of the last `window` epochs (this one included).
+  // The paper describes it in words only (confidence saturates toward 1 with
+  // observations; well-observed pairs rely on the posterior, young ones on the
+  // windowed frequency) [reading]: c = n/(n+kappa), n = hits+misses;
+  // f = window hits / window observations (the posterior itself if the window
+  // is empty); estimate = c*P + (1-c)*f.
+  if (p->window > 0) {
+    uint64_t* slot = &p->win[(size_t)p->win_head * 32];
+    for (int pr = 0; pr < 16; ++pr) {
+      p->wsum[2 * pr] = p->wsum[2 * pr] - slot[2 * pr] + epoch_misses[pr];
+      p->wsum[2 * pr + 1] = p->wsum[2 * pr + 1] - slot[2 * pr + 1] + epoch_hits[pr];
+      slot[2 * pr] = epoch_misses[pr];
+      slot[2 * pr + 1] = epoch_hits[pr];
+    }
+    p->win_head = (p->win_head + 1) % p->window;
+  }
+  for (int pr = 0; pr < 16; ++pr) {
+    if (p->window == 0) { p->estimate[pr] = p->P[pr]; continue; }
+    float n = (float)(p->hits[pr] + p->misses[pr]);
+    float c = n / (n + p->kappa);
+    float wh = (float)p->wsum[2 * pr + 1];
+    float wn = (float)(p->wsum[2 * pr + 1] + p->wsum[2 * pr]);
+    float f = wn > 0.0f ? wh / wn : p->P[pr];
+    float t1 = c * p->P[pr];
+    float t2 = 1.0f - c;
+    float t3 = t2 * f;
+    p->estimate[pr] = t1 + t3;
+  }
+  // step 4: the policy's score.  0 = Bayesian (reuse estimate x EMA importance),
+  // 1 = EMA only, 2 = LRU (epoch of the last touch): the paper's three-way
+  // comparison of eviction policies.
   for (int64_t i = 0; i < p->N; ++i) {
-    if (p->state[i] == ST_RESIDENT)
-      p->score[i] = p->P[p->pair[i]] * p->ema[i];
-    else
+    if (p->state[i] != ST_RESIDENT) {
       p->score[i] = std::numeric_limits<float>::infinity();
+    } else if (p->policy == 1) {
+      p->score[i] = p->ema[i];
+    } else if (p->policy == 2) {
+      p->score[i] = (float)p->last_epoch[i];
+    } else {
+      p->score[i] = p->estimate[p->pair[i]] * p->ema[i];
+    }
   }
   p->st.epochs += 1;
   p->st.events += n_events;

@@ -68,6 +68,12 @@ def lib():
         L.okv_get_stats.argtypes = [C.c_void_p, C.c_void_p]
         L.okv_next_tag.restype = C.c_uint64
         L.okv_next_tag.argtypes = [C.c_void_p]
+        L.okv_set_policy.restype = C.c_int32
+        L.okv_set_policy.argtypes = [C.c_void_p, C.c_int32]
+        L.okv_set_confidence_blend.restype = C.c_int32
+        L.okv_set_confidence_blend.argtypes = [C.c_void_p, C.c_float, C.c_int32]
+        L.okv_estimate.restype = C.c_void_p
+        L.okv_estimate.argtypes = [C.c_void_p]
         L.okv_epoch_score.restype = C.c_int32
         L.okv_epoch_score.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64]
         L.okv_select_victims.restype = C.c_int32
@@ -175,6 +181,17 @@ class OraclePool:
     @property
     def next_tag(self):
         return int(lib().okv_next_tag(self._h))
+
+    @property
+    def estimate(self):
+        """The 16 reuse estimates the Bayesian score uses (posterior, or its blend)."""
+        return _view(lib().okv_estimate(self._h), np.float32, 16)
+
+    def set_policy(self, policy):
+        return lib().okv_set_policy(self._h, policy)
+
+    def set_confidence_blend(self, kappa, window):
+        return lib().okv_set_confidence_blend(self._h, kappa, window)
 
     def info(self, q):
         L = lib()
