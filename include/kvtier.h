@@ -209,6 +209,31 @@ int32_t kv_epoch_events(kv_pool* pool, const uint32_t* d_ev_entry, const uint8_t
 uint64_t* kv_epoch_counts(kv_pool* pool);
 int32_t kv_epoch_update(kv_pool* pool, uint32_t epoch, kv_stream_t stream);
 
+/* Eviction policy used by step 4 of kv_epoch_score from the next call on: the
+ * three policies the paper compares in its table of cache hit rates.
+ *   KV_POLICY_BAYESIAN  score = reuse estimate of the pair x EMA importance (default)
+ *   KV_POLICY_EMA       score = EMA importance alone ("pattern-aware")
+ *   KV_POLICY_LRU       score = epoch of the last touch ("reactive") */
+typedef enum { KV_POLICY_BAYESIAN = 0, KV_POLICY_EMA = 1, KV_POLICY_LRU = 2 } kv_policy_t;
+int32_t kv_set_policy(kv_pool* pool, int32_t policy);
+
+/* Confidence-weighted reuse estimate (Bayesian reuse section: a confidence score
+ * that saturates toward 1 as observations accumulate weighs the posterior
+ * against an empirical frequency over a sliding window of recent observations;
+ * the paper gives no formula, the one used here is):
+ *   n = hits + misses of the pair,  c = n / (n + kappa),
+ *   f = hits / observations of the pair over the last `window` epochs (this
+ *       epoch included; the posterior itself while the window is empty),
+ *   estimate = c * P + (1 - c) * f          (binary32, each operation rounded once)
+ * and the Bayesian score uses `estimate` in place of P.  window is 1..64 epochs;
+ * window = 0 switches the blend off (default; estimate = P).  The call empties
+ * the window (enqueued on `stream`) and takes effect from the next
+ * kv_epoch_score.  d_P keeps holding the plain posterior of Eq. "reuse". */
+int32_t kv_set_confidence_blend(kv_pool* pool, float kappa, int32_t window, kv_stream_t stream);
+
+/* Device address of the 16 reuse estimates (f32) the Bayesian score used last. */
+const float* kv_reuse_estimate(kv_pool* pool);
+
 /* Writes to d_victims (device, u32[k]) the k RESIDENT entries that come first in
  * the total order (score, global id), in ascending id order: the k lowest
  * scores, ties broken by lowest (partition, layer, block, head).

@@ -24,6 +24,7 @@ KV_ERR_UNIMPLEMENTED = -9
 KV_ERR_TAGS_EXHAUSTED = -10
 KV_AUTO, KV_MHA, KV_GQA, KV_MQA, KV_MLA = -1, 0, 1, 2, 3
 KV_STATE_FREE, KV_STATE_RESIDENT = 0, 1
+KV_POLICY_BAYESIAN, KV_POLICY_EMA, KV_POLICY_LRU = 0, 1, 2
 KV_NONE = 0xFFFFFFFF
 KV_LOC_HOST = 0x80000000
 
@@ -77,7 +78,7 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
            "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_events", "kv_epoch_counts",
-           "kv_epoch_update", "kv_select_victims", "kv_select_victims_static", "kv_demote",
+           "kv_epoch_update", "kv_set_policy", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_select_victims", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
            "kv_set_move_variant", "kv_set_select_variant", "kv_last_cuda_error", "kv_status_string",
@@ -116,6 +117,12 @@ def load():
     L.kv_epoch_counts.argtypes = [vp]
     L.kv_epoch_update.restype = i32
     L.kv_epoch_update.argtypes = [vp, u32, vp]
+    L.kv_set_policy.restype = i32
+    L.kv_set_policy.argtypes = [vp, i32]
+    L.kv_set_confidence_blend.restype = i32
+    L.kv_set_confidence_blend.argtypes = [vp, C.c_float, i32, vp]
+    L.kv_reuse_estimate.restype = vp
+    L.kv_reuse_estimate.argtypes = [vp]
     L.kv_select_victims.restype = i32
     L.kv_select_victims.argtypes = [vp, u64, vp, vp]
     L.kv_select_victims_static.restype = i32
@@ -313,6 +320,17 @@ class Pool:
 
     def kv_epoch_update(self, epoch):
         return self.lib.kv_epoch_update(self._h, epoch, _stream_ptr(self.compute))
+
+    def kv_set_policy(self, policy):
+        return self.lib.kv_set_policy(self._h, int(policy))
+
+    def kv_set_confidence_blend(self, kappa, window):
+        return self.lib.kv_set_confidence_blend(self._h, float(kappa), int(window), _stream_ptr(self.compute))
+
+    def kv_reuse_estimate(self):
+        """The 16 reuse estimates as a float32 tensor aliasing the library's device memory."""
+        off = self.lib.kv_reuse_estimate(self._h) - self.workspace.data_ptr()
+        return self.workspace[off:off + 64].view(self.torch.float32)
 
     def kv_select_victims(self, k, d_victims):
         return self.lib.kv_select_victims(self._h, int(k), d_victims.data_ptr() if k else None,

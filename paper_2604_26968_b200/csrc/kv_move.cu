@@ -284,8 +284,10 @@ __global__ void __launch_bounds__(kThreads) init_ring_kernel(const PartGeom g) {
 __global__ void init_scalars_kernel(uint64_t* hits, uint64_t* misses, float* P, float p0,
                                     const Workspace ws) {
   const uint32_t t = threadIdx.x;
-  if (t < 16) { hits[t] = 0; misses[t] = 0; P[t] = p0; }
-  if (t < 32) ws.delta[t] = 0;
+  if (t < 16) { hits[t] = 0; misses[t] = 0; P[t] = p0; ws.blend->estimate[t] = p0; }
+  if (t < 32) { ws.delta[t] = 0; ws.blend->wsum[t] = 0; }
+  for (uint32_t i = t; i < kMaxWindow * 32; i += blockDim.x) ws.blend->win[i] = 0;
+  if (t == 0) { ws.blend->head = 0; ws.blend->pad = 0; }
   for (uint32_t b = t; b < 3 * kHistBins; b += blockDim.x) ws.hist[b] = 0;
   if (t < 4) ws.part_counts[t] = 0;
   if (t == 0) {

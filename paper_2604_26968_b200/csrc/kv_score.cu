@@ -108,16 +108,21 @@ cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit,
 }
 
 // ---- fused entry pass ------------------------------------------------------------
-// One step of the per-entry EMA, then the eviction score.
+// One step of the per-entry EMA, then the eviction score of the chosen policy:
+// 0 = reuse estimate x EMA importance, 1 = EMA only, 2 = LRU (epoch of the last
+// touch, this epoch's touches included) -- the three policies the paper compares.
 __device__ __forceinline__ void entry_step(float& ema, float decay, uint32_t touch, uint32_t pair,
-                                           uint32_t state, const float* sP, float& score) {
+                                           uint32_t state, const float* sP, int policy,
+                                           uint32_t last_epoch, uint32_t epoch, float& score) {
   if (state == KV_STATE_RESIDENT) {
     const float x = __uint2float_rn(touch);
     const float t1 = __fmul_rn(decay, ema);
     const float t2 = __fsub_rn(1.0f, decay);
     const float t3 = __fmul_rn(t2, x);
     ema = __fadd_rn(t1, t3);
-    score = __fmul_rn(sP[pair & 15u], ema);
+    if (policy == 0) score = __fmul_rn(sP[pair & 15u], ema);
+    else if (policy == 1) score = ema;
+    else score = __uint2float_rn(touch ? epoch : last_epoch);
   } else {
     score = __int_as_float(0x7F800000);  // +inf: not a candidate
   }
@@ -130,7 +135,37 @@ struct Predictor {
   float alpha0, beta0;
   unsigned long long* delta;   // [32] this epoch's counts, index 2*pair + hit
   unsigned int* ticket;        // blocks that have finished (the last one commits)
+  int policy;
+  float kappa;                 // confidence saturation constant of the blend
+  uint32_t window;             // epochs in the sliding window; 0 = no blending
+  BlendState* blend;
 };
+
+// Reuse estimate of pair p: the posterior P, or -- when a window is set -- its
+// confidence-weighted blend with the hit frequency of the last `window` epochs
+// (the current one included).  The paper describes the blend in words (Bayesian
+// reuse section: confidence saturates toward 1 as observations accumulate; young
+// pairs lean on the windowed frequency); the form used is c = n/(n+kappa),
+// estimate = c*P + (1-c)*f, every operation rounded once.  wm/wh receive the
+// window's new sums.
+__device__ __forceinline__ float reuse_estimate(const Predictor& pd, unsigned p, float P,
+                                                unsigned long long h, unsigned long long m,
+                                                unsigned long long& wh, unsigned long long& wm) {
+  wh = wm = 0;
+  if (pd.window == 0) return P;
+  const uint32_t head = pd.blend->head;
+  wm = pd.blend->wsum[2 * p] - pd.blend->win[head * 32 + 2 * p] + pd.delta[2 * p];
+  wh = pd.blend->wsum[2 * p + 1] - pd.blend->win[head * 32 + 2 * p + 1] + pd.delta[2 * p + 1];
+  const float n = __ull2float_rn(h + m);
+  const float c = __fdiv_rn(n, __fadd_rn(n, pd.kappa));
+  const float fh = __ull2float_rn(wh);
+  const float fn = __ull2float_rn(wh + wm);
+  const float f = fn > 0.0f ? __fdiv_rn(fh, fn) : P;
+  const float t1 = __fmul_rn(c, P);
+  const float t2 = __fsub_rn(1.0f, c);
+  const float t3 = __fmul_rn(t2, f);
+  return __fadd_rn(t1, t3);
+}
 
 // Posterior mean of Eq. "reuse" for pair p from the running totals plus this
 // epoch's counts: P = alpha / (alpha + beta), alpha = alpha0 + hits, beta =
@@ -158,9 +193,11 @@ entry_update_kernel(float* __restrict__ ema, const float* __restrict__ decay,
                     float* __restrict__ score, const Predictor pd, uint64_t n, uint32_t epoch) {
   __shared__ float sP[16];
   __shared__ bool s_last;
+  const int policy = pd.policy;
   if (threadIdx.x < 16) {
-    unsigned long long h, m;
-    sP[threadIdx.x] = posterior(pd, threadIdx.x, h, m);
+    unsigned long long h, m, wh, wm;
+    const float P = posterior(pd, threadIdx.x, h, m);
+    sP[threadIdx.x] = reuse_estimate(pd, threadIdx.x, P, h, m, wh, wm);
   }
   __syncthreads();
   const uint64_t n4 = n / 4;
@@ -171,11 +208,13 @@ entry_update_kernel(float* __restrict__ ema, const float* __restrict__ decay,
     const uint4 t = reinterpret_cast<const uint4*>(touch)[v];
     const uchar4 pr = reinterpret_cast<const uchar4*>(pair)[v];
     const uchar4 st = reinterpret_cast<const uchar4*>(state)[v];
+    uint4 le = make_uint4(0, 0, 0, 0);
+    if (policy == 2) le = reinterpret_cast<const uint4*>(last_epoch)[v];  // only LRU reads it
     float4 sc;
-    entry_step(e.x, d.x, t.x, pr.x, st.x, sP, sc.x);
-    entry_step(e.y, d.y, t.y, pr.y, st.y, sP, sc.y);
-    entry_step(e.z, d.z, t.z, pr.z, st.z, sP, sc.z);
-    entry_step(e.w, d.w, t.w, pr.w, st.w, sP, sc.w);
+    entry_step(e.x, d.x, t.x, pr.x, st.x, sP, policy, le.x, epoch, sc.x);
+    entry_step(e.y, d.y, t.y, pr.y, st.y, sP, policy, le.y, epoch, sc.y);
+    entry_step(e.z, d.z, t.z, pr.z, st.z, sP, policy, le.z, epoch, sc.z);
+    entry_step(e.w, d.w, t.w, pr.w, st.w, sP, policy, le.w, epoch, sc.w);
     reinterpret_cast<float4*>(ema)[v] = e;
     reinterpret_cast<float4*>(score)[v] = sc;
     // touch counts of FREE entries are always zero (events on them are refused)
@@ -193,7 +232,7 @@ entry_update_kernel(float* __restrict__ ema, const float* __restrict__ decay,
     float e = ema[i];
     float sc;
     const uint32_t t = touch[i];
-    entry_step(e, decay[i], t, pair[i], state[i], sP, sc);
+    entry_step(e, decay[i], t, pair[i], state[i], sP, policy, policy == 2 ? last_epoch[i] : 0u, epoch, sc);
     ema[i] = e;
     score[i] = sc;
     if (t) {
@@ -210,25 +249,49 @@ entry_update_kernel(float* __restrict__ ema, const float* __restrict__ decay,
   __syncthreads();
   if (s_last && threadIdx.x < 16) {
     const unsigned p = threadIdx.x;
-    unsigned long long h, m;
+    unsigned long long h, m, wh, wm;
     const float P = posterior(pd, p, h, m);
+    const float est = reuse_estimate(pd, p, P, h, m, wh, wm);
     pd.hits[p] = h;
     pd.misses[p] = m;
     pd.P[p] = P;
+    pd.blend->estimate[p] = est;
+    const uint32_t head = pd.blend->head;
+    __syncwarp(0xFFFFu);  // all 16 lanes have read the head and the expiring window slot
+    if (pd.window > 0) {   // this epoch's counts replace the oldest slot of the window
+      pd.blend->win[head * 32 + 2 * p] = pd.delta[2 * p];
+      pd.blend->win[head * 32 + 2 * p + 1] = pd.delta[2 * p + 1];
+      pd.blend->wsum[2 * p] = wm;
+      pd.blend->wsum[2 * p + 1] = wh;
+      if (p == 0) pd.blend->head = (head + 1) % pd.window;
+    }
     pd.delta[2 * p] = 0;
     pd.delta[2 * p + 1] = 0;
     if (p == 0) *pd.ticket = 0;
   }
 }
 
+__global__ void blend_reset_kernel(BlendState* b) {
+  for (uint32_t i = threadIdx.x; i < kMaxWindow * 32; i += blockDim.x) b->win[i] = 0;
+  if (threadIdx.x < 32) b->wsum[threadIdx.x] = 0;
+  if (threadIdx.x == 0) b->head = 0;
+}
+
+cudaError_t launch_blend_reset(const Workspace& ws, cudaStream_t s) {
+  blend_reset_kernel<<<1, 256, 0, s>>>(ws.blend);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P,
                                 float alpha0, float beta0, const Workspace& ws, uint32_t epoch,
-                                cudaStream_t s) {
+                                const ScoreOptions& opt, cudaStream_t s) {
   uint64_t blocks = (st.n / 4 + kThreads - 1) / kThreads;
   if (blocks == 0) blocks = 1;
   const uint64_t cap = (uint64_t)kSMs * 8;
   if (blocks > cap) blocks = cap;
-  const Predictor pd{hits, misses, P, alpha0, beta0, ws.delta, &ws.sel->update_ticket};
+  const Predictor pd{hits,       misses,    P,          alpha0, beta0, ws.delta, &ws.sel->update_ticket,
+                     opt.policy, opt.kappa, opt.window, ws.blend};
   entry_update_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(st.ema, st.decay, st.touch, st.last_epoch,
                                                             st.pair, st.state, st.score, pd, st.n, epoch);
   count_launches(1);

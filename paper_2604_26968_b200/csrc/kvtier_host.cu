@@ -99,6 +99,7 @@ struct kv_pool {
   bool events_made = false;
   int demote_turn = 0, promote_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
+  ScoreOptions score_opt;   // eviction policy and confidence blend
   // optional per-launch timing of the pack / unpack kernels
   struct Timed { cudaEvent_t a, b; int kind; uint64_t bytes; bool pending; };
   bool timing = false;
@@ -110,7 +111,7 @@ struct kv_pool {
 namespace {
 
 struct Layout {
-  uint64_t delta, hist, sel, status, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
+  uint64_t delta, hist, sel, status, blend, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
   uint64_t ring[4][5];
   uint64_t dev_total;
   uint64_t h_list[2], h_counts, h_status, host_total;
@@ -161,6 +162,7 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
   L->hist = take(3 * kHistBins * 4);
   L->sel = take(sizeof(SelectScalars));
   L->status = take(4);
+  L->blend = take(sizeof(BlendState));
   L->part_counts = take(4 * 8);
   L->tile_counts = take((uint64_t)L->n_tiles * 8);
   L->tile_offsets = take((uint64_t)L->n_tiles * 8);
@@ -320,6 +322,7 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
   p->ws.hist = reinterpret_cast<uint32_t*>(w + L.hist);
   p->ws.sel = reinterpret_cast<SelectScalars*>(w + L.sel);
   p->ws.status = reinterpret_cast<uint32_t*>(w + L.status);
+  p->ws.blend = reinterpret_cast<BlendState*>(w + L.blend);
   p->ws.part_counts = reinterpret_cast<unsigned long long*>(w + L.part_counts);
   p->ws.tile_counts = reinterpret_cast<uint2*>(w + L.tile_counts);
   p->ws.tile_offsets = reinterpret_cast<uint2*>(w + L.tile_offsets);
@@ -425,7 +428,7 @@ uint64_t* kv_epoch_counts(kv_pool* p) {
 int32_t kv_epoch_update(kv_pool* p, uint32_t epoch, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
   KV_CUDA(p, launch_entry_update(p->st, p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
-                                 p->desc.beta0, p->ws, epoch, S(stream)));
+                                 p->desc.beta0, p->ws, epoch, p->score_opt, S(stream)));
   p->stats.epochs += 1;
   return KV_OK;
 }
@@ -687,6 +690,23 @@ int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) 
   *status_bits = *p->h_status;
   return KV_OK;
 }
+
+int32_t kv_set_policy(kv_pool* p, int32_t policy) {
+  if (!p || policy < KV_POLICY_BAYESIAN || policy > KV_POLICY_LRU) return KV_ERR_INVALID_ARG;
+  p->score_opt.policy = policy;
+  return KV_OK;
+}
+
+int32_t kv_set_confidence_blend(kv_pool* p, float kappa, int32_t window, kv_stream_t stream) {
+  if (!p || window < 0 || window > (int32_t)kMaxWindow || (window > 0 && !(kappa > 0.0f)))
+    return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_blend_reset(p->ws, S(stream)));
+  p->score_opt.kappa = kappa;
+  p->score_opt.window = (uint32_t)window;
+  return KV_OK;
+}
+
+const float* kv_reuse_estimate(kv_pool* p) { return p ? p->ws.blend->estimate : nullptr; }
 
 int32_t kv_set_move_variant(int32_t variant) {
   if (variant != 0 && variant != 1) return KV_ERR_INVALID_ARG;

@@ -63,7 +63,26 @@ struct SelectScalars {
   unsigned long long phase_ns[8];  // %globaltimer at the phase boundaries of the last persistent selection (CTA 0)
 };
 
+// Sliding window of per-epoch (pair, hit) counts for the confidence-weighted
+// blend of the reuse estimate, and the estimates themselves.
+constexpr uint32_t kMaxWindow = 64;
+struct BlendState {
+  unsigned long long wsum[32];              // sums over the window, index 2*pair + hit
+  unsigned long long win[kMaxWindow * 32];  // ring of per-epoch counts
+  float estimate[16];                       // reuse estimate used by the Bayesian score
+  uint32_t head;                            // ring slot the next epoch overwrites
+  uint32_t pad;
+};
+
+// Host-chosen options of the scoring pass.
+struct ScoreOptions {
+  int policy = 0;       // 0 Bayesian, 1 EMA only, 2 LRU
+  float kappa = 0.0f;   // confidence saturation constant
+  uint32_t window = 0;  // epochs in the sliding window; 0 = no blending
+};
+
 struct Workspace {
+  BlendState* blend;
   unsigned long long* delta;   // [32] per-epoch (pair, hit) counts: index pair*2+hit
   uint32_t* hist;              // [3][kHistBins]
   SelectScalars* sel;
@@ -83,7 +102,9 @@ cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit,
 // folds ws.delta into hits/misses, clears it and writes P
 cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P,
                                 float alpha0, float beta0, const Workspace& ws, uint32_t epoch,
-                                cudaStream_t s);
+                                const ScoreOptions& opt, cudaStream_t s);
+// empties the sliding window of the blend (the estimates stay as they are)
+cudaError_t launch_blend_reset(const Workspace& ws, cudaStream_t s);
 
 // ---- kv_select.cu ----
 cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims, const Workspace& ws,

@@ -35,17 +35,23 @@ def oracle_admit(w, pool, epoch, key=None):
 
 
 class Lockstep:
-    def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True):
+    def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True,
+                 policy=0, blend=None):
         self.w = w
         self.payload = payload
         self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
                                fill_pattern=True, host_meta=host_meta)
+        self.options = (policy, blend)
         # room for any k a test may ask for
         self.gpu.victims = self.gpu.torch.empty(max(w.N, 4), dtype=self.gpu.torch.int32,
                                                 device=self.gpu.pool.device)
         self.ora = O.OraclePool(oracle_parts(w), w.alpha0, w.beta0, n_tags=w.n_tags, payload=payload)
         self.fresh = oracle_admit(w, self.ora, 0, key=INITIAL_EPOCH_KEY)
         assert np.array_equal(self.fresh, self.gpu.fresh)
+        assert self.ora.set_policy(policy) == O.OK and self.gpu.pool.kv_set_policy(policy) == 0
+        if blend is not None:
+            assert self.ora.set_confidence_blend(*blend) == O.OK
+            assert self.gpu.pool.kv_set_confidence_blend(*blend) == 0
         self.compare_state("initial fill")
         if payload:
             self.compare_payload("initial fill")
@@ -68,6 +74,9 @@ class Lockstep:
         assert np.array_equal(g.host_array("hits"), o.hits), where
         assert np.array_equal(g.host_array("misses"), o.misses), where
         assert np.array_equal(g.host_array("P").view(np.uint32), o.P.view(np.uint32)), where
+        g.pool.sync()
+        est = g.pool.kv_reuse_estimate().cpu().numpy()
+        assert np.array_equal(est.view(np.uint32), o.estimate.view(np.uint32)), where
         assert np.array_equal(g.host_array("loc"), o.loc), where
         assert g.pool.kv_device_status() == 0, where
 
