@@ -56,6 +56,8 @@ def parse():
     ap.add_argument("--no-hostlink", action="store_true", help="skip the 1 GiB host-link probe")
     ap.add_argument("--move-variant", type=int, default=1, choices=[0, 1],
                     help="pack/unpack kernels: 1 = bulk-copy engine, 0 = register path")
+    ap.add_argument("--tiny-entries", action="store_true",
+                    help="32-64 byte blocks (same entry count and traces): for profiling scoring/selection")
     ap.add_argument("--select-variant", type=int, default=1, choices=[0, 1],
                     help="selection: 1 = one persistent cooperative launch, 0 = one launch per phase")
     return ap.parse_args()
@@ -220,7 +222,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2604_26968_b200 import workloads as W
-    w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots)
+    w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries)
     t_ss, t_all, done = oracle_epochs(w, args.steps, warm=args.warmup)
     value = w.N * done / t_ss
     sample = "%d full epochs of pool %d (N=%d) in metadata mode (no payload bytes), 1 thread" % (
@@ -258,7 +260,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots)
+    w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries)
     w.seed = w.seed + 1000 * rank     # every rank owns its own pool and trace (weak scaling)
     link = hostlink_probe(torch, dev) if rank == 0 and not args.no_hostlink else None
     runner = EpochRunner(w, batch_bytes=args.batch_mb << 20, fill_pattern=True, host_meta=True,

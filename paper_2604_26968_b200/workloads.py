@@ -360,7 +360,8 @@ def pattern_bytes(tags: np.ndarray, entry_bytes: int) -> np.ndarray:
 
 # ---- the five pools ---------------------------------------------------------
 
-def config(i: int, scale: float = 1.0, ring_slots: Optional[int] = None) -> Workload:
+def config(i: int, scale: float = 1.0, ring_slots: Optional[int] = None,
+           tiny_entries: bool = False) -> Workload:
     """Pool i (1..5).  scale < 1 shrinks blocks_per_layer (for tests and for
     devices with less free memory); ring_slots overrides the host ring size of
     every partition."""
@@ -392,4 +393,12 @@ def config(i: int, scale: float = 1.0, ring_slots: Optional[int] = None) -> Work
         w.pair_weights = np.random.default_rng([4, 77]).dirichlet(np.full(16, 0.5))
     else:
         raise ValueError("config index must be 1..5")
+    if tiny_entries:
+        # same entries, states and traces, but 32-64 byte blocks: for profiling the scoring
+        # and selection kernels at full entry count without holding the payload
+        for p in w.parts:
+            if p.variant == MLA:
+                p.d_latent, p.d_rope = 8, 0
+            else:
+                p.head_dim = 1
     return w
