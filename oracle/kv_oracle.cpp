@@ -512,6 +512,49 @@ int32_t okv_select_victims(void* h, uint64_t k, uint32_t* out_victims) {
   return OK;
 }
 
+// Block-granular selection (head-granular eviction section: "eviction selects
+// the block with the lowest weighted aggregate importance score across heads,
+// using architecture-dependent head weights (uniform for MHA, proportional to
+// group size for GQA)").  Reading: the aggregate of block (layer, block) is
+// w * (s_0 + s_1 + ... + s_{H-1}) over its KV-head entries, summed in head order
+// in binary32, with w = query heads per KV-head entry (1 for MHA, the group size
+// for GQA, h_q for MQA and MLA), so that blocks of different architectures are
+// compared per query head.  A block is a candidate only if all its heads are
+// RESIDENT.  The k_blocks candidates first in the order (aggregate, partition,
+// layer, block) are chosen; the output lists all their entries, ascending.
+// n_out receives the number of entries written.
+int32_t okv_select_victim_blocks(void* h, uint64_t k_blocks, uint32_t* out_victims, uint64_t* n_out) {
+  Pool* p = static_cast<Pool*>(h);
+  struct Blk { float agg; int q; int64_t first; };  // first = id of head 0
+  std::vector<Blk> blks;
+  for (int q = 0; q < p->n_parts; ++q) {
+    const Part& pt = p->part[q];
+    int64_t hq = pt.d.model.n_q_heads > 0 ? pt.d.model.n_q_heads : pt.H;
+    float w = (float)(hq / pt.H > 0 ? hq / pt.H : 1);
+    for (int64_t lb = 0; lb < pt.L * pt.NB; ++lb) {
+      int64_t first = pt.base + lb * pt.H;
+      bool all = true;
+      float sum = 0.0f;
+      for (int64_t hd = 0; hd < pt.H; ++hd) {
+        if (p->state[first + hd] != ST_RESIDENT) { all = false; break; }
+        sum = sum + p->score[first + hd];
+      }
+      if (all) blks.push_back(Blk{w * sum, q, first});
+    }
+  }
+  if (k_blocks > blks.size()) return ERR_K_TOO_LARGE;
+  // blks is in (partition, layer, block) order; a stable sort keeps it among equal aggregates
+  std::stable_sort(blks.begin(), blks.end(), [](const Blk& a, const Blk& b) { return a.agg < b.agg; });
+  std::vector<uint32_t> v;
+  for (uint64_t j = 0; j < k_blocks; ++j)
+    for (int64_t hd = 0; hd < p->part[blks[j].q].H; ++hd) v.push_back((uint32_t)(blks[j].first + hd));
+  std::sort(v.begin(), v.end());
+  if (!v.empty() && !out_victims) return ERR_INVALID_ARG;
+  for (size_t j = 0; j < v.size(); ++j) out_victims[j] = v[j];
+  if (n_out) *n_out = v.size();
+  return OK;
+}
+
 // Demotion of a victim list (ascending ids) into the per-partition host rings.
 // The j-th victim of a partition goes to ring slot (cursor + j) mod R; a live
 // slot that is overwritten is dropped (there is no tier below the host here).

@@ -78,6 +78,8 @@ def lib():
         L.okv_epoch_score.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64]
         L.okv_select_victims.restype = C.c_int32
         L.okv_select_victims.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        L.okv_select_victim_blocks.restype = C.c_int32
+        L.okv_select_victim_blocks.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.POINTER(C.c_uint64)]
         L.okv_demote.restype = C.c_int32
         L.okv_demote.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         L.okv_promote.restype = C.c_int32
@@ -226,6 +228,12 @@ class OraclePool:
         out = np.zeros(int(k), dtype=np.uint32)
         rc = lib().okv_select_victims(self._h, int(k), _ptr(out))
         return rc, out
+
+    def select_victim_blocks(self, k_blocks):
+        out = np.zeros(int(self.N), dtype=np.uint32)
+        n = C.c_uint64(0)
+        rc = lib().okv_select_victim_blocks(self._h, int(k_blocks), _ptr(out), C.byref(n))
+        return rc, out[: n.value].copy()
 
     def demote(self, victims):
         victims = np.ascontiguousarray(victims, dtype=np.uint32)

@@ -98,3 +98,48 @@ def test_blend_reacts_to_a_shift_faster_than_the_posterior():
         p.epoch_score(e, np.zeros(10, np.uint32), np.zeros(10, np.uint8))
     assert p.P[3] > 0.85 and p.estimate[3] < 0.3
     assert np.array_equal(p.score[:8], (p.estimate[p.pair[:8]] * p.ema[:8]).astype(np.float32))
+
+
+def test_block_level_selection_equals_brute_force_with_architecture_weights():
+    # three partitions: MHA (w = 1, 3 heads), GQA (w = 4, 2 heads), MLA (w = 16, 1 entry per block)
+    parts = [dict(model=O.model(variant=O.MHA, n_layers=2, n_q_heads=3, n_kv_heads=3, head_dim=8),
+                  block_tokens=4, blocks_per_layer=7, ring_slots=64),
+             dict(model=O.model(variant=O.GQA, n_layers=1, n_q_heads=8, n_kv_heads=2, head_dim=8),
+                  block_tokens=4, blocks_per_layer=9, ring_slots=64),
+             dict(model=O.model(n_layers=2, n_q_heads=16, n_kv_heads=16, head_dim=8, d_latent=12, d_rope=4),
+                  block_tokens=4, blocks_per_layer=5, ring_slots=64)]
+    p = O.OraclePool(parts, n_tags=4096, payload=False)
+    r = np.random.default_rng(4)
+    p.admit(0, 0.5, r.integers(0, 16, p.N, dtype=np.uint8), None)
+    for epoch in range(1, 4):
+        ev = r.integers(0, p.N, 60).astype(np.uint32)
+        p.epoch_score(epoch, ev, np.ones(60, np.uint8))
+    assert p.demote(np.array([4, 44], np.uint32)) == O.OK      # two blocks lose a head: no longer candidates
+    p.epoch_score(4, [], [])
+    H = [3, 2, 1]
+    w = [np.float32(1), np.float32(4), np.float32(16)]
+    blocks = []
+    for q in range(3):
+        inf = p.info(q)
+        for lb in range(inf["n"] // H[q]):
+            first = inf["base"] + lb * H[q]
+            if not all(p.state[first + h] == O.RESIDENT for h in range(H[q])):
+                continue
+            s = np.float32(0)
+            for h in range(H[q]):
+                s = np.float32(s + p.score[first + h])
+            blocks.append((float(np.float32(w[q] * s)), first, H[q]))
+    order = sorted(range(len(blocks)), key=lambda j: (blocks[j][0], blocks[j][1]))
+    for k in (0, 1, 5, len(blocks) // 2, len(blocks)):
+        rc, v = p.select_victim_blocks(k)
+        expect = sorted(i for j in order[:k] for i in range(blocks[j][1], blocks[j][1] + blocks[j][2]))
+        assert rc == O.OK and v.tolist() == expect, k
+    rc, _ = p.select_victim_blocks(len(blocks) + 1)
+    assert rc == O.ERR_K_TOO_LARGE
+    assert len(blocks) == 2 * 7 + 9 + 2 * 5 - 2
+    # all-zero scores: aggregates tie, lowest (partition, layer, block) first, whole blocks come out
+    q = O.OraclePool(parts, n_tags=4096, payload=False)
+    q.admit(0, 0.5, np.zeros(q.N, np.uint8), None)
+    q.epoch_score(1, [], [])
+    rc, v = q.select_victim_blocks(3)
+    assert rc == O.OK and v.tolist() == list(range(9))
