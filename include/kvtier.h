@@ -263,6 +263,25 @@ int32_t kv_demote(kv_pool* pool, const uint32_t* d_victims, uint64_t m, uint64_t
 int32_t kv_promote(kv_pool* pool, int32_t partition, const uint64_t* h_host_slots, uint64_t m,
                    uint64_t batch_bytes, kv_stream_t compute, kv_stream_t copy);
 
+/* Block-granular selection (head-granular eviction section: eviction takes the
+ * block with the lowest weighted aggregate importance across heads, with head
+ * weights uniform for MHA and proportional to the group size for GQA).  The
+ * aggregate of a paged block (layer, block) is w * (s_0 + ... + s_{H-1}) over the
+ * scores of its H KV-head entries, added in head order in binary32, with w = query
+ * heads per KV-head entry (1 for MHA, h_q/h_kv for GQA, h_q for MQA and MLA), so
+ * that blocks of different architectures in one pool compare per query head.
+ * Only blocks whose heads are all RESIDENT are candidates.  The k_blocks
+ * candidates first in the order (aggregate, partition, layer, block) are chosen
+ * and ALL their entries are written to d_victims (device, u32, room for
+ * k_blocks x the largest head count), in ascending id order, ready for kv_demote.
+ * *h_n_victims (host) receives the number of entries: known without waiting for
+ * a single-partition pool; a pool with several partitions waits on the host for a
+ * 32-byte readback (everything enqueued on `stream` before it finishes first).
+ * If k_blocks exceeds the number of candidate blocks (not known to the host) the
+ * device status word gets KV_DEV_SELECT_MISMATCH. */
+int32_t kv_select_victim_blocks(kv_pool* pool, uint64_t k_blocks, uint32_t* d_victims,
+                                uint64_t* h_n_victims, kv_stream_t stream);
+
 /* Selection for callers that cannot allocate (the paper has no counterpart; it
  * is a packaging of kv_select_victims, not another method).  A serving engine
  * that has given all device memory to its own pools, or code that runs where

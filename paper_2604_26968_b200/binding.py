@@ -78,7 +78,7 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
            "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_events", "kv_epoch_counts",
-           "kv_epoch_update", "kv_set_policy", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_select_victims", "kv_select_victims_static", "kv_demote",
+           "kv_epoch_update", "kv_set_policy", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
            "kv_set_move_variant", "kv_set_select_variant", "kv_last_cuda_error", "kv_status_string",
@@ -125,6 +125,8 @@ def load():
     L.kv_reuse_estimate.argtypes = [vp]
     L.kv_select_victims.restype = i32
     L.kv_select_victims.argtypes = [vp, u64, vp, vp]
+    L.kv_select_victim_blocks.restype = i32
+    L.kv_select_victim_blocks.argtypes = [vp, u64, vp, C.POINTER(u64), vp]
     L.kv_select_victims_static.restype = i32
     L.kv_select_victims_static.argtypes = [vp, vp, u64, u64, vp, vp, vp]
     L.kv_demote.restype = i32
@@ -335,6 +337,13 @@ class Pool:
     def kv_select_victims(self, k, d_victims):
         return self.lib.kv_select_victims(self._h, int(k), d_victims.data_ptr() if k else None,
                                           _stream_ptr(self.compute))
+
+    def kv_select_victim_blocks(self, k_blocks, d_victims):
+        """Returns (status, number of entries written)."""
+        n = C.c_uint64(0)
+        rc = self.lib.kv_select_victim_blocks(self._h, int(k_blocks), d_victims.data_ptr() if k_blocks else None,
+                                              C.byref(n), _stream_ptr(self.compute))
+        return rc, n.value
 
     def kv_demote(self, d_victims, m, batch_bytes):
         return self.lib.kv_demote(self._h, d_victims.data_ptr() if m else None, int(m), int(batch_bytes),

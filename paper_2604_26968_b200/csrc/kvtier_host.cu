@@ -100,6 +100,7 @@ struct kv_pool {
   int demote_turn = 0, promote_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
   ScoreOptions score_opt;   // eviction policy and confidence blend
+  BlockGeom bgeom;          // paged blocks of all partitions in one index space
   // optional per-launch timing of the pack / unpack kernels
   struct Timed { cudaEvent_t a, b; int kind; uint64_t bytes; bool pending; };
   bool timing = false;
@@ -111,7 +112,7 @@ struct kv_pool {
 namespace {
 
 struct Layout {
-  uint64_t delta, hist, sel, status, blend, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
+  uint64_t delta, hist, sel, status, blend, block_score, block_state, block_victims, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
   uint64_t ring[4][5];
   uint64_t dev_total;
   uint64_t h_list[2], h_counts, h_status, host_total;
@@ -124,6 +125,7 @@ struct Derived {
   uint64_t heads[4], n[4], entry_bytes[4], chunk_bytes[4], n_chunks[4];
   uint64_t bases[5];
   uint64_t N;
+  uint64_t blocks[4], n_blocks;   // paged blocks (layer x block) per partition and in total
 };
 
 int32_t derive(const kv_pool_desc* d, Derived* out) {
@@ -147,10 +149,13 @@ int32_t derive(const kv_pool_desc* d, Derived* out) {
     out->n[q] = (uint64_t)p.model.n_layers * (uint64_t)p.blocks_per_layer * out->heads[q];
     out->bases[q] = base;
     base += out->n[q];
+    out->blocks[q] = (uint64_t)p.model.n_layers * (uint64_t)p.blocks_per_layer;
   }
   for (int q = d->n_partitions; q <= 4; ++q) out->bases[q] = base;
   if (base == 0 || base >= 0x80000000ull) return KV_ERR_INVALID_ARG;  // ids must fit 31 bits
   out->N = base;
+  out->n_blocks = 0;
+  for (int q = 0; q < d->n_partitions; ++q) out->n_blocks += out->blocks[q];
   return KV_OK;
 }
 
@@ -163,6 +168,9 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
   L->sel = take(sizeof(SelectScalars));
   L->status = take(4);
   L->blend = take(sizeof(BlendState));
+  L->block_score = take(g.n_blocks * 4);
+  L->block_state = take(g.n_blocks);
+  L->block_victims = take(g.n_blocks * 4);
   L->part_counts = take(4 * 8);
   L->tile_counts = take((uint64_t)L->n_tiles * 8);
   L->tile_offsets = take((uint64_t)L->n_tiles * 8);
@@ -323,6 +331,9 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
   p->ws.sel = reinterpret_cast<SelectScalars*>(w + L.sel);
   p->ws.status = reinterpret_cast<uint32_t*>(w + L.status);
   p->ws.blend = reinterpret_cast<BlendState*>(w + L.blend);
+  p->ws.block_score = reinterpret_cast<float*>(w + L.block_score);
+  p->ws.block_state = w + L.block_state;
+  p->ws.block_victims = reinterpret_cast<uint32_t*>(w + L.block_victims);
   p->ws.part_counts = reinterpret_cast<unsigned long long*>(w + L.part_counts);
   p->ws.tile_counts = reinterpret_cast<uint2*>(w + L.tile_counts);
   p->ws.tile_offsets = reinterpret_cast<uint2*>(w + L.tile_offsets);
@@ -361,6 +372,27 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
   }
   for (int b = 0; b < 4; ++b) p->staging[b] = static_cast<uint8_t*>(desc->d_staging[b]);
   p->staging_bytes = desc->staging_bytes;
+  p->bgeom.n_parts = g.n_parts;
+  {
+    uint64_t bb = 0;
+    for (int q = 0; q < 4; ++q) {
+      p->bgeom.block_base[q] = bb;
+      if (q < g.n_parts) {
+        bb += g.blocks[q];
+        p->bgeom.entry_base[q] = g.bases[q];
+        p->bgeom.heads[q] = (uint32_t)g.heads[q];
+        const int64_t hq = desc->part[q].model.n_q_heads > 0 ? desc->part[q].model.n_q_heads : (int64_t)g.heads[q];
+        const int64_t wq = hq / (int64_t)g.heads[q];
+        p->bgeom.weight[q] = (float)(wq > 0 ? wq : 1);
+      } else {
+        p->bgeom.entry_base[q] = g.N;
+        p->bgeom.heads[q] = 1;
+        p->bgeom.weight[q] = 1.0f;
+      }
+    }
+    p->bgeom.block_base[4] = bb;
+    for (int q = g.n_parts; q < 4; ++q) p->bgeom.block_base[q] = bb;
+  }
   p->max_promote = desc->max_promote;
   p->stats.n_entries = g.N;
   p->stats.n_free = g.N;
@@ -446,6 +478,29 @@ int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream
   if (k == 0) return KV_OK;
   if (!d_victims || !aligned16(d_victims)) return KV_ERR_INVALID_ARG;
   KV_CUDA(p, launch_select(p->st, k, d_victims, p->ws, S(stream)));
+  return KV_OK;
+}
+
+int32_t kv_select_victim_blocks(kv_pool* p, uint64_t k_blocks, uint32_t* d_victims, uint64_t* h_n_victims,
+                                kv_stream_t stream) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  if (h_n_victims) *h_n_victims = 0;
+  if (k_blocks > p->bgeom.block_base[p->n_parts]) return KV_ERR_K_TOO_LARGE;
+  if (k_blocks == 0) return KV_OK;
+  if (!d_victims || !aligned16(d_victims)) return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_select_blocks(p->st, p->bgeom, k_blocks, d_victims, p->ws, S(stream)));
+  uint64_t m = 0;
+  if (p->n_parts == 1) {
+    m = k_blocks * p->bgeom.heads[0];
+  } else {
+    // which partitions the chosen blocks fall in is only known on the device
+    KV_CUDA(p, cudaMemcpyAsync(p->h_counts, p->ws.part_counts, 4 * sizeof(uint64_t), cudaMemcpyDeviceToHost,
+                               S(stream)));
+    KV_CUDA(p, cudaEventRecord(p->ev_counts, S(stream)));
+    KV_CUDA(p, cudaEventSynchronize(p->ev_counts));
+    for (int q = 0; q < p->n_parts; ++q) m += p->h_counts[q] * p->bgeom.heads[q];
+  }
+  if (h_n_victims) *h_n_victims = m;
   return KV_OK;
 }
 

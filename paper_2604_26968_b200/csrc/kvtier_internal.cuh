@@ -81,8 +81,21 @@ struct ScoreOptions {
   uint32_t window = 0;  // epochs in the sliding window; 0 = no blending
 };
 
+// Paged blocks (layer, block) of all partitions in one index space, for
+// block-granular selection.
+struct BlockGeom {
+  uint64_t block_base[5];   // first global block index of each partition; [n_parts] = total
+  uint64_t entry_base[4];   // first global entry id of each partition
+  uint32_t heads[4];        // KV-head entries per block
+  float weight[4];          // query heads per KV-head entry
+  int n_parts;
+};
+
 struct Workspace {
   BlendState* blend;
+  float* block_score;       // [blocks] aggregate score per paged block
+  uint8_t* block_state;     // [blocks] RESIDENT iff every head of the block is
+  uint32_t* block_victims;  // [blocks] selected global block indices
   unsigned long long* delta;   // [32] per-epoch (pair, hit) counts: index pair*2+hit
   uint32_t* hist;              // [3][kHistBins]
   SelectScalars* sel;
@@ -114,6 +127,10 @@ extern int g_select_variant;  // which selection launch_select uses (see kv_sele
 // whether it was launched (false: the device cannot co-schedule it, nothing was enqueued)
 cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
                                      const Workspace& ws, cudaStream_t s, bool* used);
+// kv_blocks.cu: k_blocks lowest blocks by weighted aggregate score; writes all their entries
+// (ascending) to d_victims and the per-partition block counts to ws.part_counts
+cudaError_t launch_select_blocks(const EntryState& st, const BlockGeom& bg, uint64_t k_blocks,
+                                 uint32_t* d_victims, const Workspace& ws, cudaStream_t s);
 // ascending ids of FREE entries in [lo, hi), at most `limit` of them, into ws.free_list
 cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uint64_t limit,
                              const Workspace& ws, cudaStream_t s);

@@ -122,7 +122,8 @@ class Lockstep:
                 assert np.array_equal(a[:, c][mask], b[:, c][mask]), (where, q, c)
 
     # ---- one epoch -----------------------------------------------------------
-    def epoch(self, e, k=None, check_payload=None):
+    def epoch(self, e, k=None, check_payload=None, k_blocks=None):
+        """One epoch on both sides.  k_blocks selects whole paged blocks instead of k entries."""
         w, g, o = self.w, self.gpu, self.ora
         k = w.k if k is None else k
         ev_entry, ev_hit = w.events(e, o.pair, self.fresh)
@@ -130,9 +131,16 @@ class Lockstep:
         assert o.epoch_score(e, ev_entry, ev_hit) == O.OK
         g.check(g.pool.kv_epoch_score(e, d_e, d_h, n), "kv_epoch_score")
         self.compare_state("epoch %d score" % e)
-        rc, v = o.select_victims(k)
-        assert rc == O.OK
-        g.check(g.pool.kv_select_victims(k, g.victims), "kv_select_victims")
+        if k_blocks is None:
+            rc, v = o.select_victims(k)
+            assert rc == O.OK
+            g.check(g.pool.kv_select_victims(k, g.victims), "kv_select_victims")
+        else:
+            rc, v = o.select_victim_blocks(k_blocks)
+            assert rc == O.OK
+            rc, k = g.pool.kv_select_victim_blocks(k_blocks, g.victims)
+            g.check(rc, "kv_select_victim_blocks")
+            assert k == len(v), (k, len(v))
         g.pool.sync()
         got = g.victims[:k].cpu().numpy().view(np.uint32)
         assert np.array_equal(got, v), "epoch %d victims" % e
