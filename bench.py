@@ -56,6 +56,8 @@ def parse():
     ap.add_argument("--no-hostlink", action="store_true", help="skip the 1 GiB host-link probe")
     ap.add_argument("--move-variant", type=int, default=1, choices=[0, 1],
                     help="pack/unpack kernels: 1 = bulk-copy engine, 0 = register path")
+    ap.add_argument("--sharded", action="store_true",
+                    help="use the sharded epoch path (kv_epoch_events + all-reduce + kv_epoch_update) even on one rank")
     ap.add_argument("--tiny-entries", action="store_true",
                     help="32-64 byte blocks (same entry count and traces): for profiling scoring/selection")
     ap.add_argument("--select-variant", type=int, default=1, choices=[0, 1],
@@ -257,7 +259,8 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
+    dist_on = world > 1 or args.sharded    # --sharded: take the multi-GPU code path even on one rank
+    if dist_on:
         dist.init_process_group("nccl", device_id=dev)
 
     w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries)
@@ -272,7 +275,7 @@ def main():
     B.kv_set_select_variant(args.select_variant)
     N, k = w.N, w.k
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    counts = pool.kv_epoch_counts() if world > 1 else None
+    counts = pool.kv_epoch_counts() if dist_on else None
 
     def gen_events(e):
         return runner.next_events(e)
@@ -283,7 +286,7 @@ def main():
         overlap the demotion's D2H copies."""
         with torch.cuda.stream(pool.compute):
             ev[0].record(pool.compute)
-        if world > 1:
+        if dist_on:
             runner.check(pool.kv_epoch_events(d_e, d_h, n), "kv_epoch_events")
             with torch.cuda.stream(pool.compute):
                 dist.all_reduce(counts)          # 32 int64 counters shared by all pools
@@ -323,7 +326,7 @@ def main():
     for it in range(args.warmup + args.steps):
         timed = it >= args.warmup
         if it == args.warmup:
-            if world > 1:
+            if dist_on:
                 dist.barrier()
             torch.cuda.synchronize(dev)
             pool.kv_timing_read()                 # discard warm-up launches
@@ -349,14 +352,14 @@ def main():
         between_steps(epoch)
         epoch += 1
     torch.cuda.synchronize(dev)
-    if world > 1:
+    if dist_on:
         dist.barrier()
     clocks = sampler.stop()
     timing = pool.kv_timing_read()
     status = pool.kv_device_status()
     K = args.steps
     t = torch.tensor([tot["ss"], tot["dem"], tot["pro"], tot["all"]], dtype=torch.float64, device=dev)
-    if world > 1:
+    if dist_on:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ss_ms, dem_ms, pro_ms, all_ms = [float(x) / K for x in t.tolist()]
 
@@ -377,7 +380,7 @@ def main():
             d_h = torch.empty_like(h_h, device=dev)
             flush_l2(epoch)
             torch.cuda.synchronize(dev)
-            if world > 1:
+            if dist_on:
                 dist.barrier()
             t0 = time.perf_counter()
             with torch.cuda.stream(pool.compute):
@@ -394,14 +397,14 @@ def main():
             between_steps(epoch)
             epoch += 1
         tw = torch.tensor([wall], dtype=torch.float64, device=dev)
-        if world > 1:
+        if dist_on:
             dist.all_reduce(tw, op=dist.ReduceOp.MAX)
         e2e = {"value": N * world * e2e_steps / float(tw.item()), "unit": "head-blocks/s (whole epoch, host in/out)",
                "h2d_bytes_per_step": h2d_b // e2e_steps, "d2h_bytes_per_step": d2h_b // e2e_steps,
                "steps": e2e_steps, "ms_per_step": 1e3 * float(tw.item()) / e2e_steps}
 
     if rank != 0:
-        if world > 1:
+        if dist_on:
             dist.destroy_process_group()
         return
 
@@ -424,7 +427,7 @@ def main():
                    "events_per_step": tot["events"] // K, "pool_bytes": sum(p.slab_bytes for p in w.parts),
                    "entry_bytes": [p.entry_bytes for p in w.parts], "batch_bytes": runner.batch_bytes,
                    "ring_slots": [p.ring_slots for p in w.parts], "scale": args.scale,
-                   "parallelism": "1 pool per GPU" + (", 256-byte all-reduce of pair counters" if world > 1 else ""),
+                   "parallelism": "1 pool per GPU" + (", 256-byte all-reduce of pair counters" if dist_on else ""),
                    "l2": "flushed before every step: 8 x 256 MiB written on the step's stream (and >1 GB of "
                          "fresh blocks admitted between steps)"},
         "phases": {
@@ -460,7 +463,7 @@ def main():
             "ms_per_epoch_score_select": 1e3 * t_ss / done}
     print(json.dumps(line))
     runner.close()
-    if world > 1:
+    if dist_on:
         dist.destroy_process_group()
 
 
