@@ -56,6 +56,8 @@ def parse():
     ap.add_argument("--no-hostlink", action="store_true", help="skip the 1 GiB host-link probe")
     ap.add_argument("--move-variant", type=int, default=1, choices=[0, 1],
                     help="pack/unpack kernels: 1 = bulk-copy engine, 0 = register path")
+    ap.add_argument("--no-deferred-packing", action="store_true",
+                    help="enqueue the whole demotion before the promotion instead of interleaving their chunks")
     ap.add_argument("--sharded", action="store_true",
                     help="use the sharded epoch path (kv_epoch_events + all-reduce + kv_epoch_update) even on one rank")
     ap.add_argument("--tiny-entries", action="store_true",
@@ -273,6 +275,7 @@ def main():
     from paper_2604_26968_b200 import binding as B
     B.kv_set_move_variant(args.move_variant)
     B.kv_set_select_variant(args.select_variant)
+    pool.kv_set_deferred_packing(not args.no_deferred_packing)
     N, k = w.N, w.k
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     counts = pool.kv_epoch_counts() if dist_on else None
@@ -296,11 +299,12 @@ def main():
         runner.check(pool.kv_select_victims(k, runner.victims), "kv_select_victims")
         ev[1].record(pool.compute)
         runner.check(pool.kv_demote(runner.victims, k, runner.batch_bytes), "kv_demote")
-        ev[2].record(pool.copy)
         lists = runner.promote_lists(e)
         ev[4].record(pool.copy_h2d)
         for q, lst in enumerate(lists):
             runner.check(pool.kv_promote(q, lst, runner.batch_bytes), "kv_promote")
+        runner.check(pool.kv_flush(), "kv_flush")     # the rest of a deferred demotion belongs to the step
+        ev[2].record(pool.copy)
         ev[5].record(pool.copy_h2d)
         ev[3].record(pool.compute)
         return sum(len(x) for x in lists), lists
@@ -426,6 +430,7 @@ def main():
         "config": {"workload": w.name, "pool": args.config, "n_entries": N, "k": k,
                    "events_per_step": tot["events"] // K, "pool_bytes": sum(p.slab_bytes for p in w.parts),
                    "entry_bytes": [p.entry_bytes for p in w.parts], "batch_bytes": runner.batch_bytes,
+                   "deferred_packing": not args.no_deferred_packing,
                    "ring_slots": [p.ring_slots for p in w.parts], "scale": args.scale,
                    "parallelism": "1 pool per GPU" + (", 256-byte all-reduce of pair counters" if dist_on else ""),
                    "l2": "flushed before every step: 8 x 256 MiB written on the step's stream (and >1 GB of "

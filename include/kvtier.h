@@ -308,6 +308,26 @@ int32_t kv_select_victims_static(const float* d_score, const uint8_t* d_state, u
                                  uint64_t k, uint32_t* d_victims, uint32_t* d_status,
                                  kv_stream_t stream);
 
+/* Deferred packing (off by default).  A demotion larger than two staging buffers
+ * keeps the compute stream waiting for its own D2H copies, and a promotion
+ * enqueued after it would only start unpacking when the demotion is nearly over.
+ * With deferred packing on, kv_demote moves the metadata of ALL victims at once
+ * (their slots become FREE immediately) and enqueues only the first two payload
+ * chunks; the remaining chunks are enqueued by the NEXT call on the pool:
+ * kv_promote interleaves them with its own chunks (a promoted entry only ever
+ * lands in a freed slot whose payload has already been packed, because victims
+ * and free slots are both taken in ascending id order), any other call enqueues
+ * all that is left first.  Results are the same as without it.  The price is a
+ * contract: d_victims must stay valid, and the caller's own kernels must not
+ * write into the freed slots, until a later call on the pool has returned and its
+ * work on `compute` has run.  Needs the bulk-copy pack kernels (move variant 1). */
+int32_t kv_set_deferred_packing(kv_pool* pool, int32_t on);
+
+/* Enqueues (on the streams the demotion was given) whatever deferred packing still
+ * holds back.  After it returns, synchronising those streams completes the
+ * demotion, and d_victims may be reused once they have run.  A no-op otherwise. */
+int32_t kv_flush(kv_pool* pool);
+
 /* Largest batch_bytes the staging buffers allow for a partition. */
 uint64_t kv_max_batch_bytes(const kv_pool* pool, int32_t partition);
 

@@ -79,7 +79,7 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
            "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_events", "kv_epoch_counts",
            "kv_epoch_update", "kv_set_policy", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
-           "kv_promote", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
+           "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
            "kv_set_move_variant", "kv_set_select_variant", "kv_last_cuda_error", "kv_status_string",
            "kv_version")
@@ -133,6 +133,10 @@ def load():
     L.kv_demote.argtypes = [vp, vp, u64, u64, vp, vp]
     L.kv_promote.restype = i32
     L.kv_promote.argtypes = [vp, i32, vp, u64, u64, vp, vp]
+    L.kv_set_deferred_packing.restype = i32
+    L.kv_set_deferred_packing.argtypes = [vp, i32]
+    L.kv_flush.restype = i32
+    L.kv_flush.argtypes = [vp]
     L.kv_max_batch_bytes.restype = u64
     L.kv_max_batch_bytes.argtypes = [vp, i32]
     L.kv_admit.restype = i32
@@ -360,6 +364,12 @@ class Pool:
         rc = self.lib.kv_admit(self._h, epoch, decay, d_new_pairs.data_ptr(), d_new_pairs.numel(),
                                1 if fill_pattern else 0, C.byref(n), _stream_ptr(self.compute))
         return rc, n.value
+
+    def kv_set_deferred_packing(self, on=True):
+        return self.lib.kv_set_deferred_packing(self._h, 1 if on else 0)
+
+    def kv_flush(self):
+        return self.lib.kv_flush(self._h)
 
     def kv_max_batch_bytes(self, partition=0):
         return int(self.lib.kv_max_batch_bytes(self._h, partition))

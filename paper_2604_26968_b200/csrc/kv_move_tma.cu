@@ -88,6 +88,11 @@ __device__ __forceinline__ uint64_t slab_chunk_offset(const PartGeom& g, uint64_
   return ((lb * g.n_chunks + c) * g.heads + head) * (uint64_t)g.chunk_bytes;
 }
 
+// A demotion can run its metadata for all victims first and move the payload
+// chunk by chunk later (so that a promotion can already take the freed slots
+// that have been packed).
+constexpr uint32_t kMoveAll = 0, kMoveMetaOnly = 1, kMoveCopyOnly = 2;
+
 struct MoveArgs {
   PartGeom g;
   EntryState st;
@@ -99,6 +104,7 @@ struct MoveArgs {
   uint8_t* staging;
   uint64_t meta_offset;    // pack: where the kv_slot_meta records go (~0 = none)
   uint32_t* status;
+  uint32_t mode;           // pack only: kMoveAll, kMoveMetaOnly or kMoveCopyOnly
 };
 
 // Metadata of one demoted entry (ring slot mirror, block table, slot state).
@@ -179,6 +185,20 @@ move_tma_kernel(const MoveArgs a) {
         continue;
       }
       if (PACK) {
+        if (a.mode == kMoveCopyOnly) {
+          // the entry's metadata moved earlier: the record for the host mirror comes from the ring mirror
+          if (a.meta_offset != ~0ull) {
+            const uint32_t slot = (uint32_t)((a.ring_start + j) % g.ring_slots);
+            uint32_t* rec = reinterpret_cast<uint32_t*>(a.staging + a.meta_offset + j * kMetaBytes);
+            rec[0] = g.r_tag[slot];
+            rec[1] = g.r_last_epoch[slot];
+            rec[2] = __float_as_uint(g.r_ema[slot]);
+            rec[3] = __float_as_uint(g.r_decay[slot]);
+            rec[4] = g.r_pair[slot];
+            rec[5] = 0;
+          }
+          continue;
+        }
         demote_meta(a, j, id);
       } else {
         const uint32_t slot = a.slots[j];
@@ -193,6 +213,7 @@ move_tma_kernel(const MoveArgs a) {
   }
 
   // ---- copy warp: lane 0 drives the bulk copies, all lanes fetch entry ids ----
+  if (PACK && a.mode == kMoveMetaOnly) return;
   if (lane == 0) {
     for (uint32_t s = 0; s < kStages; ++s) mbar_init(&bars[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -290,9 +311,9 @@ static cudaError_t launch_move(const MoveArgs& a, cudaStream_t s) {
 
 cudaError_t launch_pack_tma(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* victims,
                             uint64_t count, uint64_t ring_start, uint8_t* staging, uint64_t meta_offset,
-                            const Workspace& ws, cudaStream_t s) {
+                            const Workspace& ws, cudaStream_t s, uint32_t mode) {
   if (count == 0) return cudaSuccess;
-  MoveArgs a{g, st, loc, victims, nullptr, count, ring_start, staging, meta_offset, ws.status};
+  MoveArgs a{g, st, loc, victims, nullptr, count, ring_start, staging, meta_offset, ws.status, mode};
   return launch_move<true>(a, s);
 }
 
@@ -300,7 +321,7 @@ cudaError_t launch_unpack_tma(const PartGeom& g, const EntryState& st, uint32_t*
                               const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
                               const Workspace& ws, cudaStream_t s) {
   if (count == 0) return cudaSuccess;
-  MoveArgs a{g, st, loc, free_ids, slots, count, 0, const_cast<uint8_t*>(staging), ~0ull, ws.status};
+  MoveArgs a{g, st, loc, free_ids, slots, count, 0, const_cast<uint8_t*>(staging), ~0ull, ws.status, kMoveAll};
   return launch_move<false>(a, s);
 }
 

@@ -100,6 +100,16 @@ struct kv_pool {
   int demote_turn = 0, promote_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
   ScoreOptions score_opt;   // eviction policy and confidence blend
+  // a demotion whose later chunks are not enqueued yet (deferred packing)
+  struct Pending {
+    bool active = false, meta_done = false;
+    const uint32_t* victims = nullptr;
+    uint64_t off[4] = {0, 0, 0, 0}, kq[4] = {0, 0, 0, 0}, per[4] = {0, 0, 0, 0};
+    uint64_t next[4] = {0, 0, 0, 0}, cursor0[4] = {0, 0, 0, 0};
+    cudaStream_t compute = nullptr, copy = nullptr;
+  };
+  Pending pending;
+  bool deferred_packing = false;
   BlockGeom bgeom;          // paged blocks of all partitions in one index space
   // optional per-launch timing of the pack / unpack kernels
   struct Timed { cudaEvent_t a, b; int kind; uint64_t bytes; bool pending; };
@@ -242,6 +252,91 @@ uint64_t entries_per_batch(const kv_pool* p, int q, uint64_t batch_bytes) {
   const uint64_t by_staging = (p->staging_bytes >= 16 ? p->staging_bytes - 16 : 0) / (eb + meta);
   return by_batch < by_staging ? by_batch : by_staging;
 }
+
+}  // namespace
+
+namespace {
+
+// Enqueues one chunk of a demotion: pack victims [c0, c0+cnt) of partition q into
+// a staging buffer on the compute stream, then copy it to the ring on the copy stream.
+int32_t enqueue_pack_chunk(kv_pool* p, int q, uint64_t c0, uint64_t cnt) {
+  kv_pool::Pending& pd = p->pending;
+  const PartGeom& g = p->geom[q];
+  PartHost& h = p->host[q];
+  const uint64_t eb = g.entry_bytes, R = g.ring_slots;
+  cudaStream_t compute = pd.compute, copy = pd.copy;
+  const int b = p->demote_turn;
+  p->demote_turn ^= 1;
+  KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_staging_free[b], 0));
+  const uint64_t meta_off = h.h_meta ? align_up(cnt * eb, 16) : ~0ull;
+  const uint64_t slot0 = (pd.cursor0[q] + c0) % R;
+  const uint32_t* victims = pd.victims + pd.off[q] + c0;
+  {
+    TimedScope ts(p, 0, cnt * eb, compute);
+    if (g_move_variant)
+      KV_CUDA(p, launch_pack_tma(g, p->st, p->desc.d_loc, victims, cnt, slot0, p->staging[b], meta_off, p->ws,
+                                 compute, pd.meta_done ? 2u : 0u));
+    else
+      KV_CUDA(p, launch_pack(g, p->st, p->desc.d_loc, victims, cnt, slot0, p->staging[b], meta_off, p->ws,
+                             compute));
+  }
+  KV_CUDA(p, cudaEventRecord(p->ev_ready[b], compute));
+  KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_ready[b], 0));
+  const uint64_t first = (cnt < R - slot0) ? cnt : R - slot0;
+  KV_CUDA(p, cudaMemcpyAsync(h.h_ring + slot0 * eb, p->staging[b], first * eb, cudaMemcpyDeviceToHost, copy));
+  if (cnt > first)
+    KV_CUDA(p, cudaMemcpyAsync(h.h_ring, p->staging[b] + first * eb, (cnt - first) * eb,
+                               cudaMemcpyDeviceToHost, copy));
+  if (h.h_meta) {
+    const uint64_t mb = sizeof(kv_slot_meta);
+    KV_CUDA(p, cudaMemcpyAsync(h.h_meta + slot0 * mb, p->staging[b] + meta_off, first * mb,
+                               cudaMemcpyDeviceToHost, copy));
+    if (cnt > first)
+      KV_CUDA(p, cudaMemcpyAsync(h.h_meta, p->staging[b] + meta_off + first * mb, (cnt - first) * mb,
+                                 cudaMemcpyDeviceToHost, copy));
+  }
+  KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], copy));
+  return KV_OK;
+}
+
+// Enqueues pending chunks of the last demotion, in order, until partition q_upto
+// has `need` of its victims packed (q_upto < 0: everything), or `max_chunks` were
+// enqueued.
+int32_t drain_pending(kv_pool* p, int q_upto, uint64_t need, uint64_t max_chunks) {
+  kv_pool::Pending& pd = p->pending;
+  if (!pd.active) return KV_OK;
+  uint64_t done = 0;
+  for (int q = 0; q < p->n_parts; ++q) {
+    while (pd.next[q] < pd.kq[q]) {
+      if (q_upto >= 0 && (q > q_upto || (q == q_upto && pd.next[q] >= need))) return KV_OK;
+      if (done >= max_chunks) return KV_OK;
+      const uint64_t c0 = pd.next[q];
+      const uint64_t cnt = (pd.kq[q] - c0 < pd.per[q]) ? pd.kq[q] - c0 : pd.per[q];
+      const int32_t rc = enqueue_pack_chunk(p, q, c0, cnt);
+      if (rc != KV_OK) return rc;
+      pd.next[q] = c0 + cnt;
+      ++done;
+      if (pd.next[q] == pd.kq[q]) {
+        // all copies of this partition are enqueued: remember the slots they write and when they end
+        kv_pool::D2H older = p->d2h[q][1];
+        p->d2h[q][1] = p->d2h[q][0];
+        p->d2h[q][0] = older;  // reuse the older record's event object
+        p->d2h[q][0].start = pd.cursor0[q];
+        p->d2h[q][0].count = pd.kq[q];
+        p->d2h[q][0].valid = true;
+        KV_CUDA(p, cudaEventRecord(p->d2h[q][0].ev, pd.copy));
+      }
+    }
+  }
+  pd.active = false;
+  return KV_OK;
+}
+
+#define KV_DRAIN_ALL(pool)                                                  \
+  do {                                                                      \
+    const int32_t rc__ = drain_pending(pool, -1, 0, ~0ull);                  \
+    if (rc__ != KV_OK) return rc__;                                         \
+  } while (0)
 
 }  // namespace
 
@@ -428,6 +523,7 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
 
 int32_t kv_pool_destroy(kv_pool* p) {
   if (!p) return KV_ERR_INVALID_ARG;
+  (void)drain_pending(p, -1, 0, ~0ull);
   if (p->events_made) {
     cudaEvent_t evs[] = {p->ev_staging_free[0], p->ev_staging_free[1], p->ev_ready[0], p->ev_ready[1],
                          p->ev_staging_free[2], p->ev_staging_free[3], p->ev_ready[2], p->ev_ready[3],
@@ -446,6 +542,7 @@ int32_t kv_pool_destroy(kv_pool* p) {
 int32_t kv_epoch_events(kv_pool* p, const uint32_t* d_ev_entry, const uint8_t* d_ev_hit,
                         uint64_t n_events, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
   if (n_events > 0 && (!d_ev_entry || !d_ev_hit || !aligned16(d_ev_entry) || !aligned16(d_ev_hit)))
     return KV_ERR_INVALID_ARG;
   KV_CUDA(p, launch_event_reduce(d_ev_entry, d_ev_hit, n_events, p->st, p->ws, S(stream)));
@@ -459,6 +556,7 @@ uint64_t* kv_epoch_counts(kv_pool* p) {
 
 int32_t kv_epoch_update(kv_pool* p, uint32_t epoch, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
   KV_CUDA(p, launch_entry_update(p->st, p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
                                  p->desc.beta0, p->ws, epoch, p->score_opt, S(stream)));
   p->stats.epochs += 1;
@@ -474,6 +572,7 @@ int32_t kv_epoch_score(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_entry, c
 
 int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
   if (k > p->stats.n_entries - p->stats.n_free) return KV_ERR_K_TOO_LARGE;
   if (k == 0) return KV_OK;
   if (!d_victims || !aligned16(d_victims)) return KV_ERR_INVALID_ARG;
@@ -484,6 +583,7 @@ int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream
 int32_t kv_select_victim_blocks(kv_pool* p, uint64_t k_blocks, uint32_t* d_victims, uint64_t* h_n_victims,
                                 kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
   if (h_n_victims) *h_n_victims = 0;
   if (k_blocks > p->bgeom.block_base[p->n_parts]) return KV_ERR_K_TOO_LARGE;
   if (k_blocks == 0) return KV_OK;
@@ -513,6 +613,7 @@ uint64_t kv_max_batch_bytes(const kv_pool* p, int32_t q) {
 int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t batch_bytes,
                   kv_stream_t compute_, kv_stream_t copy_) {
   if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
   if (m == 0) {
     for (int q = 0; q < 4; ++q) p->last_counts[q] = 0;
     return KV_OK;
@@ -544,52 +645,32 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
   }
   // ring slots written below may have been read by the last promotion's H2D copies
   if (p->h2d_valid) KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_h2d_done, 0));
+  kv_pool::Pending& pd = p->pending;
+  pd.victims = d_victims;
+  pd.compute = compute;
+  pd.copy = copy;
+  pd.meta_done = p->deferred_packing && g_move_variant == 1;
   uint64_t off = 0;
+  for (int q = 0; q < 4; ++q) {
+    pd.off[q] = off;
+    pd.kq[q] = kq[q];
+    pd.per[q] = per[q];
+    pd.next[q] = 0;
+    pd.cursor0[q] = q < p->n_parts ? p->host[q].cursor : 0;
+    off += kq[q];
+  }
+  if (pd.meta_done) {
+    // metadata of every victim now (slots become FREE, block table and ring mirror are updated);
+    // the payload follows chunk by chunk
+    for (int q = 0; q < p->n_parts; ++q)
+      KV_CUDA(p, launch_pack_tma(p->geom[q], p->st, p->desc.d_loc, d_victims + pd.off[q], kq[q],
+                                 pd.cursor0[q], p->staging[0], ~0ull, p->ws, compute, 1u));
+  }
+  pd.active = true;
+  // host mirror of the rings: slot assignment is fixed here; overwritten live slots are dropped
   for (int q = 0; q < p->n_parts; ++q) {
-    const PartGeom& g = p->geom[q];
     PartHost& h = p->host[q];
-    const uint64_t eb = g.entry_bytes, R = g.ring_slots;
-    for (uint64_t c0 = 0; c0 < kq[q]; c0 += per[q]) {
-      const uint64_t cnt = (kq[q] - c0 < per[q]) ? kq[q] - c0 : per[q];
-      const int b = p->demote_turn;
-      p->demote_turn ^= 1;
-      KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_staging_free[b], 0));
-      const uint64_t meta_off = h.h_meta ? align_up(cnt * eb, 16) : ~0ull;
-      const uint64_t slot0 = (h.cursor + c0) % R;
-      {
-        TimedScope ts(p, 0, cnt * eb, compute);
-        KV_CUDA(p, (g_move_variant ? launch_pack_tma : launch_pack)(
-                       g, p->st, p->desc.d_loc, d_victims + off + c0, cnt, slot0, p->staging[b], meta_off,
-                       p->ws, compute));
-      }
-      KV_CUDA(p, cudaEventRecord(p->ev_ready[b], compute));
-      KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_ready[b], 0));
-      const uint64_t first = (cnt < R - slot0) ? cnt : R - slot0;
-      KV_CUDA(p, cudaMemcpyAsync(h.h_ring + slot0 * eb, p->staging[b], first * eb,
-                                 cudaMemcpyDeviceToHost, copy));
-      if (cnt > first)
-        KV_CUDA(p, cudaMemcpyAsync(h.h_ring, p->staging[b] + first * eb, (cnt - first) * eb,
-                                   cudaMemcpyDeviceToHost, copy));
-      if (h.h_meta) {
-        const uint64_t mb = sizeof(kv_slot_meta);
-        KV_CUDA(p, cudaMemcpyAsync(h.h_meta + slot0 * mb, p->staging[b] + meta_off, first * mb,
-                                   cudaMemcpyDeviceToHost, copy));
-        if (cnt > first)
-          KV_CUDA(p, cudaMemcpyAsync(h.h_meta, p->staging[b] + meta_off + first * mb,
-                                     (cnt - first) * mb, cudaMemcpyDeviceToHost, copy));
-      }
-      KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], copy));
-    }
-    if (kq[q] > 0) {  // remember which slots this demotion's copies are writing, and when they are done
-      kv_pool::D2H older = p->d2h[q][1];
-      p->d2h[q][1] = p->d2h[q][0];
-      p->d2h[q][0] = older;  // reuse the older record's event object
-      p->d2h[q][0].start = h.cursor;
-      p->d2h[q][0].count = kq[q];
-      p->d2h[q][0].valid = true;
-      KV_CUDA(p, cudaEventRecord(p->d2h[q][0].ev, copy));
-    }
-    // host mirror of the ring: overwritten live slots are dropped
+    const uint64_t eb = p->geom[q].entry_bytes, R = p->geom[q].ring_slots;
     for (uint64_t j = 0; j < kq[q]; ++j) {
       const uint64_t slot = (h.cursor + j) % R;
       if (h.live[slot]) {
@@ -602,12 +683,12 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
     if (R) h.cursor = (h.cursor + kq[q]) % R;
     h.n_free += kq[q];
     p->stats.bytes_demoted += kq[q] * eb;
-    off += kq[q];
   }
   for (int q = 0; q < 4; ++q) p->last_counts[q] = kq[q];
   p->stats.victims += m;
   p->stats.n_free += m;
-  return KV_OK;
+  // without deferral everything is enqueued now; with it, the two chunks that need no wait
+  return drain_pending(p, -1, 0, pd.meta_done ? 2 : ~0ull);
 }
 
 int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, uint64_t batch_bytes,
@@ -638,15 +719,30 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
   auto restore = [&]() { for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 1; };
   cudaError_t e = cudaEventSynchronize(p->ev_list_copied[li]);  // the pinned list buffer is ours again
   if (e != cudaSuccess) { restore(); return cuda_fail(p, e); }
-  bool newest = false;  // does the list name a slot that the newest demotion's copies are still writing?
-  const kv_pool::D2H& d0 = p->d2h[q][0];
+  // The H2D copies below may run on another stream than the D2H copies that filled the slots, so the
+  // copy stream has to wait for the demotion(s) whose slot ranges the list touches.  d2h[q][0] is the
+  // newest demotion whose copies are all enqueued; a pending (deferred) demotion is newer still and
+  // has no completion event yet.
+  const kv_pool::Pending& pd = p->pending;
+  const bool q_pending = pd.active && pd.next[q] < pd.kq[q];
+  bool hits_pending = false, hits_newest = false;
   for (uint64_t j = 0; j < m; ++j) {
-    p->h_list[li][j] = (uint32_t)h_slots[j];
-    if (d0.valid && (h_slots[j] + R - d0.start) % R < d0.count) newest = true;
+    const uint64_t s = h_slots[j];
+    p->h_list[li][j] = (uint32_t)s;
+    if (q_pending && (s + R - pd.cursor0[q]) % R < pd.kq[q]) hits_pending = true;
+    if (p->d2h[q][0].valid && (s + R - p->d2h[q][0].start) % R < p->d2h[q][0].count) hits_newest = true;
   }
-  // the H2D copies below may run on another stream than the D2H copies that filled the slots
-  if (e == cudaSuccess && newest) e = cudaStreamWaitEvent(copy, d0.ev, 0);
-  if (e == cudaSuccess && !newest && p->d2h[q][1].valid) e = cudaStreamWaitEvent(copy, p->d2h[q][1].ev, 0);
+  if (hits_pending) {
+    // enqueue all of that demotion's copies for this partition; its record then becomes d2h[q][0]
+    const int32_t rc = drain_pending(p, q, pd.kq[q], ~0ull);
+    if (rc != KV_OK) { restore(); return rc; }
+    hits_newest = true;
+  } else if (q_pending) {
+    hits_newest = p->d2h[q][0].valid;  // everything older than the pending demotion: wait for the newest recorded
+  }
+  if (e == cudaSuccess && hits_newest) e = cudaStreamWaitEvent(copy, p->d2h[q][0].ev, 0);
+  if (e == cudaSuccess && !hits_newest && p->d2h[q][1].valid)
+    e = cudaStreamWaitEvent(copy, p->d2h[q][1].ev, 0);
   if (e == cudaSuccess)
     e = cudaStreamWaitEvent(copy, p->ev_list_free[li], 0);  // older kernels are done reading the device list
   if (e == cudaSuccess)
@@ -670,6 +766,14 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
       j += len;
     }
     KV_CUDA(p, cudaEventRecord(p->ev_ready[b], copy));
+    // The entries of this chunk go to the (c0+cnt) lowest FREE slots of the partition.  Any of those
+    // that the pending demotion freed is among its first (c0+cnt) victims of the partition (victims and
+    // free slots are both in ascending id order), so their payload must have been packed: enqueue
+    // that much of the demotion first.
+    if (p->pending.active) {
+      const int32_t rc = drain_pending(p, q, c0 + cnt, ~0ull);
+      if (rc != KV_OK) return rc;
+    }
     KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_ready[b], 0));
     {
       TimedScope ts(p, 1, cnt * eb, compute);
@@ -694,6 +798,7 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
 int32_t kv_admit(kv_pool* p, uint32_t epoch, float decay, const uint8_t* d_new_pairs, uint64_t n_new_pairs,
                  int32_t fill_pattern, uint64_t* n_admitted, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
   const uint64_t n_free = p->stats.n_free;
   if (n_admitted) *n_admitted = 0;
   if (n_free == 0) return KV_OK;
@@ -739,6 +844,7 @@ int32_t kv_last_demote_counts(const kv_pool* p, uint64_t* counts4) {
 
 int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) {
   if (!p || !status_bits) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
   KV_CUDA(p, cudaMemcpyAsync(p->h_status, p->ws.status, 4, cudaMemcpyDeviceToHost, S(stream)));
   KV_CUDA(p, cudaMemsetAsync(p->ws.status, 0, 4, S(stream)));
   KV_CUDA(p, cudaStreamSynchronize(S(stream)));
@@ -762,6 +868,19 @@ int32_t kv_set_confidence_blend(kv_pool* p, float kappa, int32_t window, kv_stre
 }
 
 const float* kv_reuse_estimate(kv_pool* p) { return p ? p->ws.blend->estimate : nullptr; }
+
+int32_t kv_flush(kv_pool* p) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
+  return KV_OK;
+}
+
+int32_t kv_set_deferred_packing(kv_pool* p, int32_t on) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
+  p->deferred_packing = on != 0;
+  return KV_OK;
+}
 
 int32_t kv_set_move_variant(int32_t variant) {
   if (variant != 0 && variant != 1) return KV_ERR_INVALID_ARG;

@@ -151,9 +151,11 @@ cudaError_t launch_unpack(const PartGeom& g, const EntryState& st, uint32_t* loc
                           const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
                           const Workspace& ws, cudaStream_t s);
 // ---- kv_move_tma.cu: the same two operations on the bulk asynchronous copy engine ----
+// mode: 0 = metadata and payload, 1 = metadata only (staging unused), 2 = payload only
+// (the metadata moved earlier; host-mirror records are rebuilt from the ring mirror)
 cudaError_t launch_pack_tma(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* victims,
                             uint64_t count, uint64_t ring_start, uint8_t* staging, uint64_t meta_offset,
-                            const Workspace& ws, cudaStream_t s);
+                            const Workspace& ws, cudaStream_t s, uint32_t mode = 0);
 cudaError_t launch_unpack_tma(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
                               const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
                               const Workspace& ws, cudaStream_t s);

@@ -85,6 +85,7 @@ class EpochRunner:
             promote_lists = self.promote_lists(epoch)
         for q, lst in enumerate(promote_lists):
             self.check(p.kv_promote(q, lst, self.batch_bytes), "kv_promote")
+        self.check(p.kv_flush(), "kv_flush")
         if admit:
             self.check(self.admit(epoch), "kv_admit")
         return promote_lists
