@@ -4,13 +4,13 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 One step = one epoch of the whole hot path on one pool: event reduction + EMA +
-posterior + score (kv_epoch_score), k-lowest selection (kv_select_victims),
+posterior + score and k-lowest selection (kv_epoch_score_select: two launches),
 pack + D2H to the pinned host ring (kv_demote), H2D + unpack of prefetched
 entries (kv_promote).  Admission of fresh blocks, which keeps the pool full, is
 a harness step and runs untimed between steps, as does an L2 flush.
 
 Prints ONE JSON line.  `value` is KV head-blocks scored + selected per second,
-N / t(kv_epoch_score + kv_select_victims), measured inside full steps; the line
+N / t(scoring + selection), measured inside full steps; the line
 also carries the whole-step rate, per-phase bandwidths, the roofline of the
 dominant kernel, the host-link peak measured in the same run, and the CPU
 oracle timed on the host cores.
@@ -60,6 +60,8 @@ def parse():
                     help="enqueue the whole demotion before the promotion instead of interleaving their chunks")
     ap.add_argument("--sharded", action="store_true",
                     help="use the sharded epoch path (kv_epoch_events + all-reduce + kv_epoch_update) even on one rank")
+    ap.add_argument("--no-fused", action="store_true",
+                    help="score and select with two calls (kv_epoch_score, kv_select_victims) instead of the fused one")
     ap.add_argument("--tiny-entries", action="store_true",
                     help="32-64 byte blocks (same entry count and traces): for profiling scoring/selection")
     ap.add_argument("--select-variant", type=int, default=1, choices=[0, 1],
@@ -294,9 +296,12 @@ def main():
             with torch.cuda.stream(pool.compute):
                 dist.all_reduce(counts)          # 32 int64 counters shared by all pools
             runner.check(pool.kv_epoch_update(e), "kv_epoch_update")
-        else:
+            runner.check(pool.kv_select_victims(k, runner.victims), "kv_select_victims")
+        elif args.no_fused:
             runner.check(pool.kv_epoch_score(e, d_e, d_h, n), "kv_epoch_score")
-        runner.check(pool.kv_select_victims(k, runner.victims), "kv_select_victims")
+            runner.check(pool.kv_select_victims(k, runner.victims), "kv_select_victims")
+        else:
+            runner.check(pool.kv_epoch_score_select(e, d_e, d_h, n, k, runner.victims), "kv_epoch_score_select")
         ev[1].record(pool.compute)
         runner.check(pool.kv_demote(runner.victims, k, runner.batch_bytes), "kv_demote")
         lists = runner.promote_lists(e)
@@ -422,7 +427,9 @@ def main():
     tr = NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE[args.move_variant]
     line = {
         "metric": METRIC, "value": N * world / (ss_ms * 1e-3), "unit": UNIT,
-        "value_definition": "N / t(kv_epoch_score + kv_select_victims), timed with CUDA events inside full steps",
+        "value_definition": "N / t(scoring + selection), timed with CUDA events inside full steps; "
+                            + ("two calls (kv_epoch_score, kv_select_victims)" if (args.no_fused or dist_on)
+                               else "kv_epoch_score_select (event reduction, then entry pass + selection in one kernel)"),
         "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": all_ms,
         "whole_step_head_blocks_per_s": N * world / (all_ms * 1e-3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
@@ -431,6 +438,7 @@ def main():
                    "events_per_step": tot["events"] // K, "pool_bytes": sum(p.slab_bytes for p in w.parts),
                    "entry_bytes": [p.entry_bytes for p in w.parts], "batch_bytes": runner.batch_bytes,
                    "deferred_packing": not args.no_deferred_packing,
+                   "fused_score_select": not (args.no_fused or dist_on),
                    "ring_slots": [p.ring_slots for p in w.parts], "scale": args.scale,
                    "parallelism": "1 pool per GPU" + (", 256-byte all-reduce of pair counters" if dist_on else ""),
                    "l2": "flushed before every step: 8 x 256 MiB written on the step's stream (and >1 GB of "

@@ -141,7 +141,8 @@ typedef struct {
   float* d_decay;         /* EMA decay per entry */
   uint32_t* d_touch;      /* touches seen in the current epoch */
   uint32_t* d_last_epoch; /* epoch of the last touch */
-  uint8_t* d_pair;        /* 4*block_type + transition_type, 0..15 */
+  uint8_t* d_pair;        /* 4*block_type + transition_type, 0..15; the library sets bit 7
+                             while the entry is FREE (the value is then meaningless) */
   uint8_t* d_state;       /* KV_STATE_* */
   uint32_t* d_tag;        /* logical handle of the block in the slot, KV_NONE if FREE */
   float* d_score;         /* eviction score, +inf for FREE entries */
@@ -239,6 +240,20 @@ const float* kv_reuse_estimate(kv_pool* pool);
  * scores, ties broken by lowest (partition, layer, block, head).
  * KV_ERR_K_TOO_LARGE if k exceeds the resident count (tracked on the host). */
 int32_t kv_select_victims(kv_pool* pool, uint64_t k, uint32_t* d_victims, kv_stream_t stream);
+
+/* kv_epoch_score followed by kv_select_victims with the per-entry pass and the
+ * selection in ONE kernel: steps 2-4 of kv_epoch_score (Bayesian reuse section,
+ * Eq. "reuse") hand every fresh score straight to the k-lowest selection, so the
+ * scores are written once for the caller and never read back, and a launch
+ * boundary disappears (two launches in all: the event reduction, then the rest).
+ * State, d_victims and the device status word end up exactly as after the two
+ * calls.  All arguments are checked before anything is enqueued: on an error
+ * (including KV_ERR_K_TOO_LARGE) the epoch has NOT been scored.  k == 0 scores
+ * only.  Where the device cannot keep the kernel's whole grid resident at once,
+ * the separate kernels run one after the other instead. */
+int32_t kv_epoch_score_select(kv_pool* pool, uint32_t epoch, const uint32_t* d_ev_entry,
+                              const uint8_t* d_ev_hit, uint64_t n_events, uint64_t k,
+                              uint32_t* d_victims, kv_stream_t stream);
 
 /* Demotes the m entries listed in d_victims (device, ascending distinct ids of
  * RESIDENT entries, as kv_select_victims writes them): packs their K/V (or MLA)

@@ -77,7 +77,7 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
                             ("decay", "<f4"), ("pair", "<u4"), ("reserved", "<u4")])
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
-           "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_events", "kv_epoch_counts",
+           "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_score_select", "kv_epoch_events", "kv_epoch_counts",
            "kv_epoch_update", "kv_set_policy", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
@@ -111,6 +111,8 @@ def load():
     L.kv_pool_destroy.argtypes = [vp]
     L.kv_epoch_score.restype = i32
     L.kv_epoch_score.argtypes = [vp, u32, vp, vp, u64, vp]
+    L.kv_epoch_score_select.restype = i32
+    L.kv_epoch_score_select.argtypes = [vp, u32, vp, vp, u64, u64, vp, vp]
     L.kv_epoch_events.restype = i32
     L.kv_epoch_events.argtypes = [vp, vp, vp, u64, vp]
     L.kv_epoch_counts.restype = vp
@@ -312,6 +314,14 @@ class Pool:
         return self.lib.kv_epoch_score(self._h, epoch,
                                        d_ev_entry.data_ptr() if n else None,
                                        d_ev_hit.data_ptr() if n else None, n, _stream_ptr(self.compute))
+
+    def kv_epoch_score_select(self, epoch, d_ev_entry, d_ev_hit, n_events, k, d_victims):
+        n = int(n_events)
+        return self.lib.kv_epoch_score_select(self._h, epoch,
+                                              d_ev_entry.data_ptr() if n else None,
+                                              d_ev_hit.data_ptr() if n else None, n, int(k),
+                                              d_victims.data_ptr() if k else None,
+                                              _stream_ptr(self.compute))
 
     def kv_epoch_events(self, d_ev_entry, d_ev_hit, n_events=None):
         n = int(n_events if n_events is not None else (d_ev_entry.numel() if d_ev_entry is not None else 0))

@@ -83,6 +83,7 @@ pack_kernel(const PartGeom g, const EntryState st, uint32_t* __restrict__ loc,
       g.r_last_epoch[slot] = le;
       loc[t] = KV_LOC_HOST | slot;
       st.state[v] = KV_STATE_FREE;
+      st.pair[v] = (uint8_t)(pr | kPairFree);
       st.tag[v] = KV_NONE;
       st.touch[v] = 0;
       if (meta_offset != ~0ull) {
@@ -262,7 +263,7 @@ init_entries_kernel(const EntryState st, uint32_t* __restrict__ loc, uint64_t n_
     st.decay[i] = 0.0f;
     st.touch[i] = 0;
     st.last_epoch[i] = 0;
-    st.pair[i] = 0;
+    st.pair[i] = (uint8_t)kPairFree;
     st.state[i] = KV_STATE_FREE;
     st.tag[i] = KV_NONE;
     st.score[i] = __int_as_float(0x7F800000);

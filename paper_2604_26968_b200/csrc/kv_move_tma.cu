@@ -128,6 +128,7 @@ __device__ __forceinline__ void demote_meta(const MoveArgs& a, uint64_t j, uint3
   g.r_last_epoch[slot] = le;
   a.loc[t] = KV_LOC_HOST | slot;
   st.state[v] = KV_STATE_FREE;
+  st.pair[v] = (uint8_t)(pr | kPairFree);
   st.tag[v] = KV_NONE;
   st.touch[v] = 0;
   if (a.meta_offset != ~0ull) {

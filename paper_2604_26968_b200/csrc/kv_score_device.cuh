@@ -1,0 +1,247 @@
+// Device-side pieces of the scoring pass, shared by the stand-alone scoring
+// kernels (kv_score.cu) and the fused score + select kernel (kv_select_persist.cu).
+//
+// All binary32 arithmetic uses the explicitly rounded intrinsics (__fmul_rn,
+// __fadd_rn, __fsub_rn, __fdiv_rn), which the compiler never contracts into a
+// fused multiply-add, and denormals are kept (no flush-to-zero), so results
+// are bit-identical to the same operations done one at a time on a CPU.
+#pragma once
+#include "kvtier_internal.cuh"
+
+namespace kvt {
+
+// ---- event reduction ---------------------------------------------------------
+// Each event adds one to the (pair, hit) counter of its entry's pair -- the
+// alpha += 1 / beta += 1 update of the Bayesian reuse section -- and one to the
+// entry's touch count.  Counters are integers, so the order of the atomics does
+// not matter.  Lanes of a warp that hit the same counter are merged first
+// (match.any), then a 32-counter shared-memory table per block, then one 64-bit
+// global atomic per non-zero counter per block.
+__device__ __forceinline__ void count_event(uint32_t key, uint32_t* s_cnt, unsigned lane) {
+  const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
+  if (key < 32 && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_cnt[key], __popc(peers));
+}
+
+// The calling block's share of the events: thread `gtid` of `stride` takes four
+// consecutive events at a time, so that its four scattered gathers are in flight
+// together.  One byte per event is gathered: the entry's pair, whose bit 7 says
+// that the entry is FREE.  Every thread of the block must call it (the votes
+// need all lanes).  s_cnt: 32 zeroed shared-memory counters, index 2*pair + hit;
+// returns the KV_DEV_* bits of refused events.
+__device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ ev_entry,
+                                                  const uint8_t* __restrict__ ev_hit, uint64_t n_events,
+                                                  const uint8_t* __restrict__ pair,
+                                                  uint32_t* __restrict__ touch, uint64_t n, uint64_t gtid,
+                                                  uint64_t stride, uint32_t* s_cnt) {
+  const uint64_t n4 = n_events / 4;
+  const uint64_t iters = (n4 + stride - 1) / stride;  // same for every thread
+  const unsigned lane = threadIdx.x & 31u;
+  uint32_t bad = 0;
+  for (uint64_t it = 0; it < iters; ++it) {
+    const uint64_t v = it * stride + gtid;
+    const bool valid = v < n4;
+    uint4 id4 = make_uint4(0, 0, 0, 0);
+    uchar4 h4 = make_uchar4(0, 0, 0, 0);
+    if (valid) {
+      id4 = reinterpret_cast<const uint4*>(ev_entry)[v];
+      h4 = reinterpret_cast<const uchar4*>(ev_hit)[v];
+    }
+    const uint32_t ids[4] = {id4.x, id4.y, id4.z, id4.w};
+    const uint32_t hit[4] = {h4.x != 0, h4.y != 0, h4.z != 0, h4.w != 0};
+    uint32_t pr[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)  // all gathers issued before any is used
+      pr[j] = (valid && ids[j] < n) ? pair[ids[j]] : kPairFree;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t key = 32;  // 32 = nothing to count
+      if (valid) {
+        if (ids[j] >= n) {
+          bad |= KV_DEV_EVENT_BAD_ID;
+        } else if (pr[j] & kPairFree) {
+          bad |= KV_DEV_EVENT_NOT_RESIDENT;
+        } else {
+          key = (pr[j] & 15u) * 2u + hit[j];
+          atomicAdd(&touch[ids[j]], 1u);
+        }
+      }
+      count_event(key, s_cnt, lane);
+    }
+  }
+  // ragged tail (n_events not a multiple of 4): first warp of the grid
+  if (gtid < 32) {
+    const uint64_t e = n4 * 4 + gtid;
+    uint32_t key = 32;
+    if (e < n_events) {
+      const uint32_t i = ev_entry[e];
+      const uint32_t pr = i < n ? pair[i] : kPairFree;
+      if (i >= n) {
+        bad |= KV_DEV_EVENT_BAD_ID;
+      } else if (pr & kPairFree) {
+        bad |= KV_DEV_EVENT_NOT_RESIDENT;
+      } else {
+        key = (pr & 15u) * 2u + (ev_hit[e] != 0);
+        atomicAdd(&touch[i], 1u);
+      }
+    }
+    count_event(key, s_cnt, lane);
+  }
+  return bad;
+}
+
+// ---- per-entry step -----------------------------------------------------------
+// One step of the per-entry EMA, then the eviction score of the chosen policy:
+// 0 = reuse estimate x EMA importance, 1 = EMA only, 2 = LRU (epoch of the last
+// touch, this epoch's touches included) -- the three policies the paper compares.
+__device__ __forceinline__ void entry_step(float& ema, float decay, uint32_t touch, uint32_t pair,
+                                           uint32_t state, const float* sP, int policy,
+                                           uint32_t last_epoch, uint32_t epoch, float& score) {
+  if (state == KV_STATE_RESIDENT) {
+    const float x = __uint2float_rn(touch);
+    const float t1 = __fmul_rn(decay, ema);
+    const float t2 = __fsub_rn(1.0f, decay);
+    const float t3 = __fmul_rn(t2, x);
+    ema = __fadd_rn(t1, t3);
+    if (policy == 0) score = __fmul_rn(sP[pair & 15u], ema);
+    else if (policy == 1) score = ema;
+    else score = __uint2float_rn(touch ? epoch : last_epoch);
+  } else {
+    score = __int_as_float(0x7F800000);  // +inf: not a candidate
+  }
+}
+
+// ---- the predictor ---------------------------------------------------------------
+struct Predictor {
+  uint64_t* hits;
+  uint64_t* misses;
+  float* P;
+  float alpha0, beta0;
+  unsigned long long* delta;   // [32] this epoch's counts, index 2*pair + hit
+  unsigned int* ticket;        // blocks that have finished (the last one commits)
+  int policy;
+  float kappa;                 // confidence saturation constant of the blend
+  uint32_t window;             // epochs in the sliding window; 0 = no blending
+  BlendState* blend;
+};
+
+// Reuse estimate of pair p: the posterior P, or -- when a window is set -- its
+// confidence-weighted blend with the hit frequency of the last `window` epochs
+// (the current one included).  The paper describes the blend in words (Bayesian
+// reuse section: confidence saturates toward 1 as observations accumulate; young
+// pairs lean on the windowed frequency); the form used is c = n/(n+kappa),
+// estimate = c*P + (1-c)*f, every operation rounded once.  wm/wh receive the
+// window's new sums.
+__device__ __forceinline__ float reuse_estimate(const Predictor& pd, unsigned p, float P,
+                                                unsigned long long h, unsigned long long m,
+                                                unsigned long long& wh, unsigned long long& wm) {
+  wh = wm = 0;
+  if (pd.window == 0) return P;
+  const uint32_t head = pd.blend->head;
+  wm = pd.blend->wsum[2 * p] - pd.blend->win[head * 32 + 2 * p] + __ldcg(&pd.delta[2 * p]);
+  wh = pd.blend->wsum[2 * p + 1] - pd.blend->win[head * 32 + 2 * p + 1] + __ldcg(&pd.delta[2 * p + 1]);
+  const float n = __ull2float_rn(h + m);
+  const float c = __fdiv_rn(n, __fadd_rn(n, pd.kappa));
+  const float fh = __ull2float_rn(wh);
+  const float fn = __ull2float_rn(wh + wm);
+  const float f = fn > 0.0f ? __fdiv_rn(fh, fn) : P;
+  const float t1 = __fmul_rn(c, P);
+  const float t2 = __fsub_rn(1.0f, c);
+  const float t3 = __fmul_rn(t2, f);
+  return __fadd_rn(t1, t3);
+}
+
+// Posterior mean of Eq. "reuse" for pair p from the running totals plus this
+// epoch's counts: P = alpha / (alpha + beta), alpha = alpha0 + hits, beta =
+// beta0 + misses.  The 64-bit counts convert to binary32 with round to nearest
+// even; the division is IEEE.  The epoch's counts are read from L2 (other blocks
+// of the same launch may have produced them).
+__device__ __forceinline__ float posterior(const Predictor& pd, unsigned p, unsigned long long& h,
+                                           unsigned long long& m) {
+  h = pd.hits[p] + __ldcg(&pd.delta[2 * p + 1]);
+  m = pd.misses[p] + __ldcg(&pd.delta[2 * p]);
+  const float a = __fadd_rn(pd.alpha0, __ull2float_rn(h));
+  const float b = __fadd_rn(pd.beta0, __ull2float_rn(m));
+  return __fdiv_rn(a, __fadd_rn(a, b));
+}
+
+// End of an epoch, run by lanes 0..15 of one warp (p = lane) once every block
+// has read the counters: folds the epoch's counts into the totals, publishes P
+// and the estimate, advances the blend's window and clears the counts.
+__device__ __forceinline__ void commit_predictor(const Predictor& pd, unsigned p) {
+  unsigned long long h, m, wh, wm;
+  const float P = posterior(pd, p, h, m);
+  const float est = reuse_estimate(pd, p, P, h, m, wh, wm);
+  pd.hits[p] = h;
+  pd.misses[p] = m;
+  pd.P[p] = P;
+  pd.blend->estimate[p] = est;
+  const uint32_t head = pd.blend->head;
+  __syncwarp(0xFFFFu);  // all 16 lanes have read the head and the expiring window slot
+  if (pd.window > 0) {   // this epoch's counts replace the oldest slot of the window
+    pd.blend->win[head * 32 + 2 * p] = __ldcg(&pd.delta[2 * p]);
+    pd.blend->win[head * 32 + 2 * p + 1] = __ldcg(&pd.delta[2 * p + 1]);
+    pd.blend->wsum[2 * p] = wm;
+    pd.blend->wsum[2 * p + 1] = wh;
+    if (p == 0) pd.blend->head = (head + 1) % pd.window;
+  }
+  pd.delta[2 * p] = 0;
+  pd.delta[2 * p + 1] = 0;
+}
+
+// Four consecutive entries (a 16-byte vector of each array) through entry_step,
+// in two halves so that a caller can have the next vector's loads in flight
+// while it finishes this one.  v indexes vectors.  The touch counts are read from
+// L2: other blocks' atomics made them.
+struct EntryVec {
+  float4 e, d;
+  uint4 t, le;
+  uchar4 pr, st;
+};
+
+__device__ __forceinline__ EntryVec entry_load4(const EntryState& st, uint64_t v, int policy) {
+  EntryVec x;
+  x.e = reinterpret_cast<const float4*>(st.ema)[v];
+  x.d = reinterpret_cast<const float4*>(st.decay)[v];
+  x.t = __ldcg(reinterpret_cast<const uint4*>(st.touch) + v);
+  x.pr = reinterpret_cast<const uchar4*>(st.pair)[v];
+  x.st = reinterpret_cast<const uchar4*>(st.state)[v];
+  x.le = make_uint4(0, 0, 0, 0);
+  if (policy == 2) x.le = reinterpret_cast<const uint4*>(st.last_epoch)[v];  // only LRU reads it
+  return x;
+}
+
+// touch and last_epoch are only written where an entry was touched.
+__device__ __forceinline__ void entry_finish4(const EntryState& st, uint64_t v, EntryVec& x, const float* sP,
+                                              int policy, uint32_t epoch, float4& sc) {
+  entry_step(x.e.x, x.d.x, x.t.x, x.pr.x, x.st.x, sP, policy, x.le.x, epoch, sc.x);
+  entry_step(x.e.y, x.d.y, x.t.y, x.pr.y, x.st.y, sP, policy, x.le.y, epoch, sc.y);
+  entry_step(x.e.z, x.d.z, x.t.z, x.pr.z, x.st.z, sP, policy, x.le.z, epoch, sc.z);
+  entry_step(x.e.w, x.d.w, x.t.w, x.pr.w, x.st.w, sP, policy, x.le.w, epoch, sc.w);
+  reinterpret_cast<float4*>(st.ema)[v] = x.e;
+  reinterpret_cast<float4*>(st.score)[v] = sc;
+  // touch counts of FREE entries are always zero (events on them are refused)
+  if (x.t.x | x.t.y | x.t.z | x.t.w) {
+    reinterpret_cast<uint4*>(st.touch)[v] = make_uint4(0, 0, 0, 0);
+    if (x.t.x) st.last_epoch[4 * v + 0] = epoch;
+    if (x.t.y) st.last_epoch[4 * v + 1] = epoch;
+    if (x.t.z) st.last_epoch[4 * v + 2] = epoch;
+    if (x.t.w) st.last_epoch[4 * v + 3] = epoch;
+  }
+}
+
+// The same for one entry (ragged ends).
+__device__ __forceinline__ void entry_update1(const EntryState& st, uint64_t i, const float* sP, int policy,
+                                              uint32_t epoch, float& sc, uint32_t& state1) {
+  float e = st.ema[i];
+  const uint32_t t = __ldcg(&st.touch[i]);
+  state1 = st.state[i];
+  entry_step(e, st.decay[i], t, st.pair[i], state1, sP, policy, policy == 2 ? st.last_epoch[i] : 0u, epoch, sc);
+  st.ema[i] = e;
+  st.score[i] = sc;
+  if (t) {
+    st.touch[i] = 0;
+    st.last_epoch[i] = epoch;
+  }
+}
+
+}  // namespace kvt

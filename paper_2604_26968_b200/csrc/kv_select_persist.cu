@@ -14,7 +14,15 @@
 // then polls.  A cooperative launch guarantees that all CTAs are resident, so
 // the wait ends; it is nevertheless bounded, and a CTA that gives up sets
 // KV_DEV_WAIT_EXPIRED and leaves (every other CTA then runs into the same limit).
-#include "kvtier_internal.cuh"
+//
+// The same kernel also exists fused with the per-entry scoring pass (FUSED =
+// true): every CTA first updates the entries of its own slice (posterior, EMA,
+// score) and turns the fresh scores straight into keys -- the score array is
+// written for the caller but never read back, and a kernel boundary disappears.
+// The event reduction stays a launch of its own ahead of it: it is bound by the
+// latency of scattered accesses and wants twice the threads per SM that this
+// kernel's shared-memory footprint allows (measured: 2.5x slower inside it).
+#include "kv_score_device.cuh"
 
 namespace kvt {
 
@@ -60,6 +68,10 @@ struct PArgs {
   uint2* cta_counts;      // [gridDim.x]
   uint32_t* status;
   unsigned long long per; // entries per CTA slice (multiple of 4)
+  // the scoring pass of the fused form
+  EntryState st;
+  Predictor pd;
+  uint32_t epoch;
 };
 
 // Bounded grid-wide barrier; false if the wait ran out.
@@ -135,11 +147,13 @@ __device__ __forceinline__ void pick_bin(const uint32_t* __restrict__ hist, uint
   __syncthreads();
 }
 
+template <bool FUSED>
 __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const PArgs a) {
   extern __shared__ __align__(16) uint32_t s_keys[];  // kPKeyCap keys
   __shared__ uint32_t s_hist[kPHistBins];
   __shared__ uint32_t s_warp[32];
   __shared__ uint32_t s_pick[2];
+  __shared__ float sP[16];
   const uint32_t t = threadIdx.x;
   unsigned int* bar = &a.sel->bar_arrive;
   const unsigned int G = gridDim.x;
@@ -207,9 +221,66 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     }
   };
 
+  if constexpr (FUSED) {
+    // reuse estimates from the totals plus this epoch's counts (final: the event
+    // reduction is an earlier launch)
+    if (t < 16) {
+      unsigned long long h, m, wh, wm;
+      const float P = posterior(a.pd, t, h, m);
+      sP[t] = reuse_estimate(a.pd, t, P, h, m, wh, wm);
+    }
+  }
+
   // ---- phase A: keys into shared memory, then the histogram of digit 0 (bits 31..21) ----
   clear_hist();
-  {
+  if constexpr (FUSED) {
+    // the slice's entries go through the EMA and score update on the way; keys of
+    // the far part are histogrammed here too, from registers
+    const int policy = a.pd.policy;
+    const uint32_t jt = 4u * t;
+    EntryVec cur;
+    if (jt + 4 <= len) cur = entry_load4(a.st, (s0 + jt) / 4, policy);
+    for (uint32_t c = 0; c < n_chunks; ++c) {
+      const uint32_t j0 = c * kPChunk + jt;
+      const unsigned long long i0 = s0 + j0;
+      // the next chunk's loads fly while this one is finished
+      EntryVec nxt;
+      if (c + 1 < n_chunks && j0 + kPChunk + 4 <= len) nxt = entry_load4(a.st, (i0 + kPChunk) / 4, policy);
+      uint32_t key[4] = {kExcluded, kExcluded, kExcluded, kExcluded};
+      if (j0 + 4 <= len) {
+        float4 sc;
+        entry_finish4(a.st, i0 / 4, cur, sP, policy, a.epoch, sc);
+        key[0] = cur.st.x == KV_STATE_RESIDENT ? p_score_key(sc.x) : kExcluded;
+        key[1] = cur.st.y == KV_STATE_RESIDENT ? p_score_key(sc.y) : kExcluded;
+        key[2] = cur.st.z == KV_STATE_RESIDENT ? p_score_key(sc.z) : kExcluded;
+        key[3] = cur.st.w == KV_STATE_RESIDENT ? p_score_key(sc.w) : kExcluded;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (j0 + j < len) {
+            float sc;
+            uint32_t s1;
+            entry_update1(a.st, i0 + j, sP, policy, a.epoch, sc, s1);
+            if (s1 == KV_STATE_RESIDENT) key[j] = p_score_key(sc);
+          }
+        }
+      }
+      cur = nxt;
+      if (c < first_far) {
+        reinterpret_cast<uint4*>(s_keys)[c * kPThreads + t] = make_uint4(key[0], key[1], key[2], key[3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) p_warp_hist_add(s_hist, key[j] != kExcluded, key[j] >> 21);
+      }
+    }
+    __syncthreads();
+    const uint32_t iters = (cached + kPThreads - 1) / kPThreads;
+    for (uint32_t i = 0; i < iters; ++i) {
+      const uint32_t j = i * kPThreads + t;
+      const uint32_t key = j < cached ? s_keys[j] : kExcluded;
+      p_warp_hist_add(s_hist, key != kExcluded, key >> 21);
+    }
+  } else {
     const uint32_t cached_chunks = (cached + kPChunk - 1) / kPChunk;
 #pragma unroll 4
     for (uint32_t c = 0; c < cached_chunks; ++c) {
@@ -218,13 +289,17 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       reinterpret_cast<uint4*>(s_keys)[c * kPThreads + t] = make_uint4(key[0], key[1], key[2], key[3]);
     }
     __syncthreads();
+    for_each_key([&](uint32_t key) { p_warp_hist_add(s_hist, key != kExcluded, key >> 21); });
   }
-  for_each_key([&](uint32_t key) { p_warp_hist_add(s_hist, key != kExcluded, key >> 21); });
   flush_hist(a.hist, 2048);
   stamp(1);
   ok = grid_barrier(bar, G);
   stamp(2);
   if (!ok) goto fail;
+  if constexpr (FUSED) {
+    // every CTA has formed its estimates: the epoch's counts can be folded in
+    if (blockIdx.x == 0 && t < 16) commit_predictor(a.pd, t);
+  }
 
   {
     // ---- phase B: fix digit 0, histogram of digit 1 (bits 20..10) ----
@@ -378,24 +453,32 @@ done:
   }
 }
 
-// Launches the persistent selection if the device can hold one CTA per SM of it
-// co-resident; *used = false (and nothing launched) otherwise.
+// Launches the persistent selection (fused with the entry pass when fs is given)
+// if the device can hold one CTA per SM of it co-resident; *used = false (and
+// nothing launched) otherwise.
 cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
-                                     const Workspace& ws, cudaStream_t s, bool* used) {
+                                     const Workspace& ws, cudaStream_t s, bool* used, const FusedScore* fs) {
   *used = false;
   static int state = 0;  // 0 = not probed, 1 = usable, -1 = not usable
   static int n_sm = 0;
   const size_t smem = (size_t)kPKeyCap * 4;
   if (state == 0) {
-    int dev = 0, coop = 0, blocks = 0;
+    int dev = 0, coop = 0, blocks = 0, blocks_f = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(select_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(select_persistent_kernel<false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess)
-      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, select_persistent_kernel, (int)kPThreads, smem);
-    state = (e == cudaSuccess && coop && blocks >= 1 && n_sm > 0) ? 1 : -1;
+      e = cudaFuncSetAttribute(select_persistent_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)smem);
+    if (e == cudaSuccess)
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, select_persistent_kernel<false>,
+                                                        (int)kPThreads, smem);
+    if (e == cudaSuccess)
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_f, select_persistent_kernel<true>,
+                                                        (int)kPThreads, smem);
+    state = (e == cudaSuccess && coop && blocks >= 1 && blocks_f >= 1 && n_sm > 0) ? 1 : -1;
     (void)cudaGetLastError();
   }
   if (state != 1) return cudaSuccess;
@@ -415,9 +498,17 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   a.cta_counts = ws.tile_counts;
   a.status = ws.status;
   a.per = ((st.n + G - 1) / G + 3) / 4 * 4;
+  a.st = st;
+  a.pd = Predictor{};
+  a.epoch = 0;
+  if (fs) {
+    a.pd = Predictor{fs->hits,       fs->misses,    fs->P,          fs->alpha0, fs->beta0, ws.delta, nullptr,
+                     fs->opt.policy, fs->opt.kappa, fs->opt.window, ws.blend};
+    a.epoch = fs->epoch;
+  }
   void* args[] = {&a};
-  cudaError_t e = cudaLaunchCooperativeKernel((void*)select_persistent_kernel, dim3(G), dim3(kPThreads), args,
-                                              smem, s);
+  void* fn = fs ? (void*)select_persistent_kernel<true> : (void*)select_persistent_kernel<false>;
+  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(G), dim3(kPThreads), args, smem, s);
   if (e != cudaSuccess) return e;
   count_launches(1);
   *used = true;

@@ -580,6 +580,32 @@ int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream
   return KV_OK;
 }
 
+int32_t kv_epoch_score_select(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_entry,
+                              const uint8_t* d_ev_hit, uint64_t n_events, uint64_t k, uint32_t* d_victims,
+                              kv_stream_t stream) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
+  if (n_events > 0 && (!d_ev_entry || !d_ev_hit || !aligned16(d_ev_entry) || !aligned16(d_ev_hit)))
+    return KV_ERR_INVALID_ARG;
+  if (k > p->stats.n_entries - p->stats.n_free) return KV_ERR_K_TOO_LARGE;
+  if (k > 0 && (!d_victims || !aligned16(d_victims))) return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_event_reduce(d_ev_entry, d_ev_hit, n_events, p->st, p->ws, S(stream)));
+  p->stats.events += n_events;
+  bool used = false;
+  if (k > 0 && g_select_variant != 0) {
+    const FusedScore fs{p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
+                        p->desc.beta0,  epoch,            p->score_opt};
+    KV_CUDA(p, launch_select_persistent(p->st, k, d_victims, p->ws, S(stream), &used, &fs));
+  }
+  if (used) {
+    p->stats.epochs += 1;
+    return KV_OK;
+  }
+  const int32_t rc = kv_epoch_update(p, epoch, stream);
+  if (rc != KV_OK || k == 0) return rc;
+  return kv_select_victims(p, k, d_victims, stream);
+}
+
 int32_t kv_select_victim_blocks(kv_pool* p, uint64_t k_blocks, uint32_t* d_victims, uint64_t* h_n_victims,
                                 kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;

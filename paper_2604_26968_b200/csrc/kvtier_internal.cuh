@@ -14,6 +14,9 @@ constexpr int kThreads = 256;
 constexpr uint32_t kRadixBits1 = 11, kRadixBits2 = 11, kRadixBits3 = 10;
 constexpr uint32_t kHistBins = 2048;  // bins of the widest digit
 constexpr uint32_t kTileEntries = 2048;  // entries per compaction tile (256 threads x 8)
+// Bit 7 of an entry's pair byte is set while the entry is FREE, so that the event
+// reduction learns both the pair and the state from one gathered byte.
+constexpr uint32_t kPairFree = 0x80u;
 
 // Kernels launched by this library in this process (all pools).
 extern std::atomic<uint64_t> g_kernel_launches;
@@ -125,8 +128,19 @@ cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims,
 extern int g_select_variant;  // which selection launch_select uses (see kv_select.cu)
 // kv_select_persist.cu: the same selection as one cooperative launch; *used tells
 // whether it was launched (false: the device cannot co-schedule it, nothing was enqueued)
+// With fs the launch also does the entry pass first (posterior, EMA, score; the
+// epoch's events have been reduced by an earlier launch).
+struct FusedScore {
+  uint64_t* hits;
+  uint64_t* misses;
+  float* P;
+  float alpha0, beta0;
+  uint32_t epoch;
+  ScoreOptions opt;
+};
 cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
-                                     const Workspace& ws, cudaStream_t s, bool* used);
+                                     const Workspace& ws, cudaStream_t s, bool* used,
+                                     const FusedScore* fs = nullptr);
 // kv_blocks.cu: k_blocks lowest blocks by weighted aggregate score; writes all their entries
 // (ascending) to d_victims and the per-partition block counts to ws.part_counts
 cudaError_t launch_select_blocks(const EntryState& st, const BlockGeom& bg, uint64_t k_blocks,

@@ -75,11 +75,15 @@ class EpochRunner:
             out.append(self.w.promote_list(epoch, q, m_q, cur, live, just_written=counts[q]))
         return out
 
-    def step(self, epoch, d_ev_entry, d_ev_hit, n_events, promote_lists=None, admit=True):
+    def step(self, epoch, d_ev_entry, d_ev_hit, n_events, promote_lists=None, admit=True, fused=True):
         """One full epoch.  Returns the promote lists used."""
         p = self.pool
-        self.check(p.kv_epoch_score(epoch, d_ev_entry, d_ev_hit, n_events), "kv_epoch_score")
-        self.check(p.kv_select_victims(self.k, self.victims), "kv_select_victims")
+        if fused:
+            self.check(p.kv_epoch_score_select(epoch, d_ev_entry, d_ev_hit, n_events, self.k, self.victims),
+                       "kv_epoch_score_select")
+        else:
+            self.check(p.kv_epoch_score(epoch, d_ev_entry, d_ev_hit, n_events), "kv_epoch_score")
+            self.check(p.kv_select_victims(self.k, self.victims), "kv_select_victims")
         self.check(p.kv_demote(self.victims, self.k, self.batch_bytes), "kv_demote")
         if promote_lists is None:
             promote_lists = self.promote_lists(epoch)

@@ -36,13 +36,14 @@ def oracle_admit(w, pool, epoch, key=None):
 
 class Lockstep:
     def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True,
-                 policy=0, blend=None, deferred=False):
+                 policy=0, blend=None, deferred=False, fused=False):
         self.w = w
         self.payload = payload
         self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
                                fill_pattern=True, host_meta=host_meta)
         self.options = (policy, blend)
         self.deferred = deferred
+        self.fused = fused   # score and select through the single fused call
         if deferred:
             assert self.gpu.pool.kv_set_deferred_packing(True) == 0
         # room for any k a test may ask for
@@ -132,12 +133,17 @@ class Lockstep:
         ev_entry, ev_hit = w.events(e, o.pair, self.fresh)
         d_e, d_h, n = g.stage_events(ev_entry, ev_hit)
         assert o.epoch_score(e, ev_entry, ev_hit) == O.OK
-        g.check(g.pool.kv_epoch_score(e, d_e, d_h, n), "kv_epoch_score")
+        fused = self.fused and k_blocks is None
+        if fused:
+            g.check(g.pool.kv_epoch_score_select(e, d_e, d_h, n, k, g.victims), "kv_epoch_score_select")
+        else:
+            g.check(g.pool.kv_epoch_score(e, d_e, d_h, n), "kv_epoch_score")
         self.compare_state("epoch %d score" % e)
         if k_blocks is None:
             rc, v = o.select_victims(k)
             assert rc == O.OK
-            g.check(g.pool.kv_select_victims(k, g.victims), "kv_select_victims")
+            if not fused:
+                g.check(g.pool.kv_select_victims(k, g.victims), "kv_select_victims")
         else:
             rc, v = o.select_victim_blocks(k_blocks)
             assert rc == O.OK
