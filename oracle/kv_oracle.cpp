@@ -13,7 +13,9 @@
 //     section exactly (Eq. "unified", Eq. "total" and the batch formula).
 //   * the posterior mean alpha/(alpha+beta) with +1 updates follows the
 //     Bayesian-reuse section exactly (Eq. "reuse").
-//   * the EMA recurrence, the product score, the ring organisation of the host
+//   * the EMA recurrence, the product score, the per-(layer, head) importance
+//     weighting (recurrence, group maximum, multipliers: okv_head_importance_update),
+//     the ring organisation of the host
 //     tier and the free-slot rule of promotion are NOT printed in the paper
 //     (it withholds them): they are this build's readings, so their agreement
 //     with the paper is "parity unpinned"; their internal consistency (closed
@@ -147,6 +149,12 @@ struct Part {
   std::vector<uint32_t> r_tag, r_last_epoch;
   std::vector<float> r_ema, r_decay;
   std::vector<uint8_t> r_pair, r_live;
+  // head-granular importance (see okv_head_importance_update)
+  int64_t QH;                   // query heads tracked per layer (1 for MLA)
+  bool head_weights;            // scores of this partition are weighted per (layer, KV head)
+  std::vector<float> h_imp;     // [L][QH] importance matrix
+  std::vector<float> h_mult;    // [L][H] task-transition multipliers
+  std::vector<float> h_w;       // [L][H] weight of a KV head: group maximum x multiplier
 };
 
 struct Stats {
@@ -204,6 +212,24 @@ void copy_image_to_entry(Part& pt, int64_t local, const uint8_t* image) {
   for (int c = 0; c < pt.n_chunks; ++c)
     std::memcpy(pt.slab.data() + chunk_offset(pt, local, c), image + c * pt.chunk_bytes,
                 (size_t)pt.chunk_bytes);
+}
+
+// Weight of KV head (l, h): the maximum importance over the query heads that
+// share it (the group of h is query heads h*G .. h*G+G-1, G = QH/H; one head for
+// MHA, all of them for MQA, the single column for MLA), times the head's
+// task-transition multiplier (head-granular eviction section).
+void recompute_head_weights(Part& pt) {
+  const int64_t G = pt.QH / pt.H;
+  for (int64_t l = 0; l < pt.L; ++l) {
+    for (int64_t hh = 0; hh < pt.H; ++hh) {
+      float m = pt.h_imp[(size_t)(l * pt.QH + hh * G)];
+      for (int64_t g = 1; g < G; ++g) {
+        float v = pt.h_imp[(size_t)(l * pt.QH + hh * G + g)];
+        if (v > m) m = v;
+      }
+      pt.h_w[(size_t)(l * pt.H + hh)] = m * pt.h_mult[(size_t)(l * pt.H + hh)];
+    }
+  }
 }
 
 }  // namespace
@@ -277,6 +303,15 @@ void* okv_create(int32_t n_parts, const PartDesc* parts, float alpha0, float bet
     pt.r_decay.assign((size_t)pt.R, 0.0f);
     pt.r_pair.assign((size_t)pt.R, 0);
     pt.r_live.assign((size_t)pt.R, 0);
+    pt.QH = (pt.variant == VAR_MLA) ? 1 : pt.d.model.n_q_heads;
+    if (pt.QH < pt.H || pt.QH % pt.H != 0) {  // every KV head serves a whole group of query heads
+      delete p;
+      return nullptr;
+    }
+    pt.head_weights = false;
+    pt.h_imp.assign((size_t)(pt.L * pt.QH), 1.0f);
+    pt.h_mult.assign((size_t)(pt.L * pt.H), 1.0f);
+    pt.h_w.assign((size_t)(pt.L * pt.H), 1.0f);
     base += pt.n;
   }
   if (base >= (int64_t)HOST_BIT) {  // ids and slots must fit 31 bits
@@ -402,6 +437,61 @@ int32_t okv_set_confidence_blend(void* h, float kappa, int32_t window) {
 // The 16 reuse estimates used by the Bayesian score (the posterior, or its blend).
 float* okv_estimate(void* h) { return static_cast<Pool*>(h)->estimate; }
 
+// Head-granular importance (head-granular eviction section).  The paper keeps a
+// [layer][head] importance matrix per model, an EMA updated on every attention
+// step; for GQA the query heads that share a KV head are grouped and the group's
+// maximum is the KV head's score; for MLA the matrix is [layer][1]; and at task
+// transitions per-head multipliers bias eviction.  Recurrence and the way the
+// matrix enters the eviction score are not printed [reading]:
+//   M[l][j] <- d*M[l][j] + (1-d)*x[l][j]      for every query head j (binary32,
+//                                              each operation rounded once);
+//   W[l][h] = max_{j in group(h)} M[l][j] * mult[l][h];
+//   score of entry (l, block, h) = (policy score) * W[l][h]   (Bayesian, EMA only).
+// M starts at 1 and multipliers at 1, and a partition's scores are weighted only
+// after the first call for it, so a pool that never calls this is unchanged.
+// x: QH*L observations (>= 0, finite), row-major [layer][query head].
+int32_t okv_head_importance_update(void* h, int32_t q, const float* x, float d) {
+  Pool* p = static_cast<Pool*>(h);
+  if (q < 0 || q >= p->n_parts || !x || !(d >= 0.0f) || !(d <= 1.0f)) return ERR_INVALID_ARG;
+  Part& pt = p->part[q];
+  const int64_t n = pt.L * pt.QH;
+  for (int64_t i = 0; i < n; ++i)
+    if (!(x[i] >= 0.0f) || !(x[i] <= std::numeric_limits<float>::max())) return ERR_INVALID_ARG;
+  for (int64_t i = 0; i < n; ++i) {
+    float t1 = d * pt.h_imp[(size_t)i];
+    float t2 = 1.0f - d;
+    float t3 = t2 * x[i];
+    pt.h_imp[(size_t)i] = t1 + t3;
+  }
+  pt.head_weights = true;
+  recompute_head_weights(pt);
+  return OK;
+}
+
+// Task-transition multipliers of partition q: L*H values (>= 0, finite), row-major
+// [layer][KV head]; NULL resets them to 1.
+int32_t okv_set_head_multipliers(void* h, int32_t q, const float* mult) {
+  Pool* p = static_cast<Pool*>(h);
+  if (q < 0 || q >= p->n_parts) return ERR_INVALID_ARG;
+  Part& pt = p->part[q];
+  const int64_t n = pt.L * pt.H;
+  if (mult)
+    for (int64_t i = 0; i < n; ++i)
+      if (!(mult[i] >= 0.0f) || !(mult[i] <= std::numeric_limits<float>::max())) return ERR_INVALID_ARG;
+  for (int64_t i = 0; i < n; ++i) pt.h_mult[(size_t)i] = mult ? mult[i] : 1.0f;
+  pt.head_weights = true;
+  recompute_head_weights(pt);
+  return OK;
+}
+
+// which: 0 importance matrix [L][QH], 1 multipliers [L][H], 2 weights [L][H]
+float* okv_head_array(void* h, int32_t q, int32_t which) {
+  Pool* p = static_cast<Pool*>(h);
+  if (q < 0 || q >= p->n_parts) return nullptr;
+  Part& pt = p->part[q];
+  return which == 0 ? pt.h_imp.data() : which == 1 ? pt.h_mult.data() : which == 2 ? pt.h_w.data() : nullptr;
+}
+
 // One epoch of scoring, in the order update-then-decide:
 //   1. every observed event adds one to alpha (reuse) or beta (miss) of the
 //      entry's (block-type, transition-type) pair, and counts a touch;
@@ -480,12 +570,19 @@ int32_t okv_epoch_score(void* h, uint32_t epoch, const uint32_t* ev_entry, const
   for (int64_t i = 0; i < p->N; ++i) {
     if (p->state[i] != ST_RESIDENT) {
       p->score[i] = std::numeric_limits<float>::infinity();
-    } else if (p->policy == 1) {
-      p->score[i] = p->ema[i];
     } else if (p->policy == 2) {
       p->score[i] = (float)p->last_epoch[i];
     } else {
-      p->score[i] = p->estimate[p->pair[i]] * p->ema[i];
+      float sc = (p->policy == 1) ? p->ema[i] : p->estimate[p->pair[i]] * p->ema[i];
+      // step 4b (optional): the importance of the entry's (layer, KV head), see
+      // okv_head_importance_update; recency-only LRU ignores it
+      const Part& pt = p->part[part_of(*p, i)];
+      if (pt.head_weights) {
+        int64_t local = i - pt.base;
+        int64_t layer = local / (pt.NB * pt.H), head = local % pt.H;
+        sc = sc * pt.h_w[(size_t)(layer * pt.H + head)];
+      }
+      p->score[i] = sc;
     }
   }
   p->st.epochs += 1;

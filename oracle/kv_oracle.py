@@ -74,6 +74,12 @@ def lib():
         L.okv_set_confidence_blend.argtypes = [C.c_void_p, C.c_float, C.c_int32]
         L.okv_estimate.restype = C.c_void_p
         L.okv_estimate.argtypes = [C.c_void_p]
+        L.okv_head_importance_update.restype = C.c_int32
+        L.okv_head_importance_update.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_float]
+        L.okv_set_head_multipliers.restype = C.c_int32
+        L.okv_set_head_multipliers.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+        L.okv_head_array.restype = C.c_void_p
+        L.okv_head_array.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
         L.okv_epoch_score.restype = C.c_int32
         L.okv_epoch_score.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64]
         L.okv_select_victims.restype = C.c_int32
@@ -143,6 +149,7 @@ class OraclePool:
             arr[q] = PartDesc(p["model"], p["block_tokens"], 0, p["blocks_per_layer"],
                               p["ring_slots"])
         self.n_parts = len(parts)
+        self._parts = list(parts)
         self._n_tags = int(n_tags) if n_tags is not None else 0
         self._h = L.okv_create(len(parts), arr, alpha0, beta0, self._n_tags, 1 if payload else 0)
         if not self._h:
@@ -194,6 +201,33 @@ class OraclePool:
 
     def set_confidence_blend(self, kappa, window):
         return lib().okv_set_confidence_blend(self._h, kappa, window)
+
+    def head_importance_update(self, q, x, decay):
+        """EMA step of partition q's [layer][query head] importance matrix with observations x."""
+        x = np.ascontiguousarray(x, dtype=np.float32)
+        if not 0 <= q < self.n_parts:
+            return ERR_INVALID_ARG
+        assert x.size == self._head_shape(q, 0)
+        return lib().okv_head_importance_update(self._h, q, _ptr(x), float(decay))
+
+    def set_head_multipliers(self, q, mult):
+        if not 0 <= q < self.n_parts:
+            return ERR_INVALID_ARG
+        if mult is not None:
+            mult = np.ascontiguousarray(mult, dtype=np.float32)
+            assert mult.size == self._head_shape(q, 1)
+        return lib().okv_set_head_multipliers(self._h, q, _ptr(mult) if mult is not None else None)
+
+    def _head_shape(self, q, which):
+        m = self._parts[q]["model"]
+        mla = lib().okv_infer_variant(C.byref(m)) == 3
+        qh = 1 if mla else m.n_q_heads
+        return m.n_layers * (qh if which == 0 else self.info(q)["H"])
+
+    def head_array(self, q, name):
+        """'importance' [L*QH], 'multipliers' [L*H] or 'weights' [L*H] of partition q."""
+        which = {"importance": 0, "multipliers": 1, "weights": 2}[name]
+        return _view(lib().okv_head_array(self._h, q, which), np.float32, self._head_shape(q, min(which, 1)))
 
     def info(self, q):
         L = lib()
