@@ -62,6 +62,8 @@ def parse():
                     help="use the sharded epoch path (kv_epoch_events + all-reduce + kv_epoch_update) even on one rank")
     ap.add_argument("--no-fused", action="store_true",
                     help="score and select with two calls (kv_epoch_score, kv_select_victims) instead of the fused one")
+    ap.add_argument("--head-weights", action="store_true",
+                    help="update every partition's head-importance matrix each step and weight the scores with it")
     ap.add_argument("--tiny-entries", action="store_true",
                     help="32-64 byte blocks (same entry count and traces): for profiling scoring/selection")
     ap.add_argument("--select-variant", type=int, default=1, choices=[0, 1],
@@ -285,12 +287,18 @@ def main():
     def gen_events(e):
         return runner.next_events(e)
 
+    head_obs = [runner.to_device(w.head_observations(0, q).reshape(-1), None) for q in range(len(w.parts))] \
+        if args.head_weights else None
+
     def one_step(e, d_e, d_h, n, ev):
         """Enqueues one full step; ev = (start, selected, D2H done, unpack done, H2D start,
         H2D done) CUDA events.  The promotion's H2D copies run on their own stream and
         overlap the demotion's D2H copies."""
         with torch.cuda.stream(pool.compute):
             ev[0].record(pool.compute)
+        if args.head_weights:
+            for q in range(len(w.parts)):
+                runner.check(pool.kv_head_importance_update(q, head_obs[q], 0.9), "kv_head_importance_update")
         if dist_on:
             runner.check(pool.kv_epoch_events(d_e, d_h, n), "kv_epoch_events")
             with torch.cuda.stream(pool.compute):
@@ -439,6 +447,7 @@ def main():
                    "entry_bytes": [p.entry_bytes for p in w.parts], "batch_bytes": runner.batch_bytes,
                    "deferred_packing": not args.no_deferred_packing,
                    "fused_score_select": not (args.no_fused or dist_on),
+                   "head_weights": bool(args.head_weights),
                    "ring_slots": [p.ring_slots for p in w.parts], "scale": args.scale,
                    "parallelism": "1 pool per GPU" + (", 256-byte all-reduce of pair counters" if dist_on else ""),
                    "l2": "flushed before every step: 8 x 256 MiB written on the step's stream (and >1 GB of "

@@ -76,6 +76,7 @@ typedef enum { KV_AUTO = -1, KV_MHA = 0, KV_GQA = 1, KV_MQA = 2, KV_MLA = 3 } kv
 #define KV_DEV_VICTIM_NOT_RESIDENT 8u
 #define KV_DEV_BAD_INDEX 16u         /* an index was out of range and the access was skipped */
 #define KV_DEV_WAIT_EXPIRED 32u      /* a bounded wait inside a kernel gave up */
+#define KV_DEV_BAD_HEAD_VALUE 64u    /* a head observation or multiplier was negative or not finite */
 
 typedef struct {
   int32_t variant;    /* kv_variant_t; KV_AUTO infers it from the fields below */
@@ -234,6 +235,36 @@ int32_t kv_set_confidence_blend(kv_pool* pool, float kappa, int32_t window, kv_s
 
 /* Device address of the 16 reuse estimates (f32) the Bayesian score used last. */
 const float* kv_reuse_estimate(kv_pool* pool);
+
+/* Head-granular importance (head-granular eviction section).  The paper keeps,
+ * per model, a [layer][head] importance matrix as an exponential moving average
+ * updated on every attention step; for GQA the query heads that share a KV head
+ * form a group whose maximum is the KV head's score; for MLA the matrix is
+ * [layer][1]; at task transitions per-head multipliers bias eviction.  It prints
+ * no formula; the form used here, per partition q (one model):
+ *   M[l][j] <- decay*M[l][j] + (1-decay)*x[l][j]     every query head j
+ *                                 (binary32, each operation rounded once; M starts at 1)
+ *   W[l][h] = max{ M[l][j] : j in group(h) } * mult[l][h]
+ *             group(h) = query heads h*G .. h*G+G-1, G = n_q_heads / KV heads
+ *             (G = 1 for MHA; MLA tracks one column per layer)
+ *   score of entry (l, block, h) = policy score * W[l][h]   for KV_POLICY_BAYESIAN
+ *             and KV_POLICY_EMA; KV_POLICY_LRU, pure recency, ignores the matrix.
+ * A partition's scores are weighted from its first call of either function on;
+ * a pool that never calls them computes exactly what it did before.
+ *   kv_head_importance_update  d_x: device f32 [n_layers][n_q_heads] ([n_layers][1]
+ *                              for MLA), observations >= 0; 0 <= decay <= 1.
+ *   kv_set_head_multipliers    d_mult: device f32 [n_layers][KV heads], >= 0; NULL
+ *                              resets all multipliers of the partition to 1.
+ * Both are enqueued on `stream` and take effect for kernels enqueued after them
+ * (use the stream of kv_epoch_score).  A value that is negative, NaN or infinite
+ * is skipped (the element keeps its old value) and sets KV_DEV_BAD_HEAD_VALUE.
+ * kv_head_importance / kv_head_weights: device addresses of M ([L][query heads])
+ * and W ([L][KV heads]) of partition q. */
+int32_t kv_head_importance_update(kv_pool* pool, int32_t q, const float* d_x, float decay,
+                                  kv_stream_t stream);
+int32_t kv_set_head_multipliers(kv_pool* pool, int32_t q, const float* d_mult, kv_stream_t stream);
+const float* kv_head_importance(kv_pool* pool, int32_t q);
+const float* kv_head_weights(kv_pool* pool, int32_t q);
 
 /* Writes to d_victims (device, u32[k]) the k RESIDENT entries that come first in
  * the total order (score, global id), in ascending id order: the k lowest

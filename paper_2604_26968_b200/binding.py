@@ -26,6 +26,7 @@ KV_AUTO, KV_MHA, KV_GQA, KV_MQA, KV_MLA = -1, 0, 1, 2, 3
 KV_STATE_FREE, KV_STATE_RESIDENT = 0, 1
 KV_POLICY_BAYESIAN, KV_POLICY_EMA, KV_POLICY_LRU = 0, 1, 2
 KV_NONE = 0xFFFFFFFF
+KV_DEV_BAD_HEAD_VALUE = 64
 KV_LOC_HOST = 0x80000000
 
 
@@ -78,7 +79,7 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
            "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_score_select", "kv_epoch_events", "kv_epoch_counts",
-           "kv_epoch_update", "kv_set_policy", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
+           "kv_epoch_update", "kv_set_policy", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
            "kv_set_move_variant", "kv_set_select_variant", "kv_last_cuda_error", "kv_status_string",
@@ -125,6 +126,14 @@ def load():
     L.kv_set_confidence_blend.argtypes = [vp, C.c_float, i32, vp]
     L.kv_reuse_estimate.restype = vp
     L.kv_reuse_estimate.argtypes = [vp]
+    L.kv_head_importance_update.restype = i32
+    L.kv_head_importance_update.argtypes = [vp, i32, vp, C.c_float, vp]
+    L.kv_set_head_multipliers.restype = i32
+    L.kv_set_head_multipliers.argtypes = [vp, i32, vp, vp]
+    L.kv_head_importance.restype = vp
+    L.kv_head_importance.argtypes = [vp, i32]
+    L.kv_head_weights.restype = vp
+    L.kv_head_weights.argtypes = [vp, i32]
     L.kv_select_victims.restype = i32
     L.kv_select_victims.argtypes = [vp, u64, vp, vp]
     L.kv_select_victim_blocks.restype = i32
@@ -347,6 +356,29 @@ class Pool:
         """The 16 reuse estimates as a float32 tensor aliasing the library's device memory."""
         off = self.lib.kv_reuse_estimate(self._h) - self.workspace.data_ptr()
         return self.workspace[off:off + 64].view(self.torch.float32)
+
+    def kv_head_importance_update(self, q, d_x, decay):
+        return self.lib.kv_head_importance_update(self._h, int(q), d_x.data_ptr(), float(decay),
+                                                  _stream_ptr(self.compute))
+
+    def kv_set_head_multipliers(self, q, d_mult):
+        return self.lib.kv_set_head_multipliers(self._h, int(q), d_mult.data_ptr() if d_mult is not None else None,
+                                                _stream_ptr(self.compute))
+
+    def _head_view(self, ptr, n):
+        off = ptr - self.workspace.data_ptr()
+        return self.workspace[off:off + 4 * n].view(self.torch.float32)
+
+    def kv_head_importance(self, q):
+        """Partition q's [layers][query heads] importance matrix (float32 tensor aliasing device memory)."""
+        p = self.parts[q]
+        qh = 1 if p.variant == KV_MLA else p.n_q_heads
+        return self._head_view(self.lib.kv_head_importance(self._h, int(q)), p.n_layers * qh)
+
+    def kv_head_weights(self, q):
+        """Partition q's [layers][KV heads] score weights."""
+        p = self.parts[q]
+        return self._head_view(self.lib.kv_head_weights(self._h, int(q)), p.n_layers * p.heads)
 
     def kv_select_victims(self, k, d_victims):
         return self.lib.kv_select_victims(self._h, int(k), d_victims.data_ptr() if k else None,

@@ -43,7 +43,7 @@ cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit,
 // block to finish folds the epoch's counts into the totals, clears them and
 // publishes P; by then every block has read them.
 __global__ void __launch_bounds__(kThreads, 4)
-entry_update_kernel(const EntryState st, const Predictor pd, uint32_t epoch) {
+entry_update_kernel(const EntryState st, const Predictor pd, const HeadWeights hw, uint32_t epoch) {
   __shared__ float sP[16];
   __shared__ bool s_last;
   const int policy = pd.policy;
@@ -62,7 +62,7 @@ entry_update_kernel(const EntryState st, const Predictor pd, uint32_t epoch) {
     EntryVec nxt;
     if (v + stride < n4) nxt = entry_load4(st, v + stride, policy);
     float4 sc;
-    entry_finish4(st, v, cur, sP, policy, epoch, sc);
+    entry_finish4(st, v, cur, sP, policy, epoch, hw, sc);
     cur = nxt;
   }
   // ragged tail (n not a multiple of 4)
@@ -70,7 +70,7 @@ entry_update_kernel(const EntryState st, const Predictor pd, uint32_t epoch) {
   if (i < st.n) {
     float sc;
     uint32_t s1;
-    entry_update1(st, i, sP, policy, epoch, sc, s1);
+    entry_update1(st, i, sP, policy, epoch, hw, sc, s1);
   }
   // commit by the last block to finish
   __syncthreads();
@@ -99,14 +99,14 @@ cudaError_t launch_blend_reset(const Workspace& ws, cudaStream_t s) {
 
 cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P,
                                 float alpha0, float beta0, const Workspace& ws, uint32_t epoch,
-                                const ScoreOptions& opt, cudaStream_t s) {
+                                const ScoreOptions& opt, const HeadWeights& hw, cudaStream_t s) {
   uint64_t blocks = (st.n / 4 + kThreads - 1) / kThreads;
   if (blocks == 0) blocks = 1;
   const uint64_t cap = (uint64_t)kSMs * 8;
   if (blocks > cap) blocks = cap;
   const Predictor pd{hits,       misses,    P,          alpha0, beta0, ws.delta, &ws.sel->update_ticket,
                      opt.policy, opt.kappa, opt.window, ws.blend};
-  entry_update_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(st, pd, epoch);
+  entry_update_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(st, pd, hw, epoch);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -89,21 +89,36 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
   return bad;
 }
 
+// ---- head-granular weight -------------------------------------------------------
+// Weight of entry i's (layer, KV head) from the partition's [layer][KV head]
+// table (head-granular eviction section); 1 for partitions that are not weighted.
+// id = base + (layer * blocks_per_layer + block) * heads + head.
+__device__ __forceinline__ float head_weight(const HeadWeights& hw, uint64_t i) {
+  int q = 0;
+  while (q + 1 < hw.n_parts && i >= hw.base[q + 1]) ++q;
+  if (!((hw.on >> q) & 1u)) return 1.0f;
+  const uint32_t local = (uint32_t)(i - hw.base[q]);
+  const uint32_t layer = local / hw.per_layer[q], head = local % hw.heads[q];
+  return __ldg(&hw.w[hw.w_off[q] + layer * hw.heads[q] + head]);
+}
+
 // ---- per-entry step -----------------------------------------------------------
 // One step of the per-entry EMA, then the eviction score of the chosen policy:
 // 0 = reuse estimate x EMA importance, 1 = EMA only, 2 = LRU (epoch of the last
 // touch, this epoch's touches included) -- the three policies the paper compares.
+// w: weight of the entry's (layer, head), which the two importance-based policies
+// multiply in (1 = unweighted; x * 1 is exact).
 __device__ __forceinline__ void entry_step(float& ema, float decay, uint32_t touch, uint32_t pair,
                                            uint32_t state, const float* sP, int policy,
-                                           uint32_t last_epoch, uint32_t epoch, float& score) {
+                                           uint32_t last_epoch, uint32_t epoch, float w, float& score) {
   if (state == KV_STATE_RESIDENT) {
     const float x = __uint2float_rn(touch);
     const float t1 = __fmul_rn(decay, ema);
     const float t2 = __fsub_rn(1.0f, decay);
     const float t3 = __fmul_rn(t2, x);
     ema = __fadd_rn(t1, t3);
-    if (policy == 0) score = __fmul_rn(sP[pair & 15u], ema);
-    else if (policy == 1) score = ema;
+    if (policy == 0) score = __fmul_rn(__fmul_rn(sP[pair & 15u], ema), w);
+    else if (policy == 1) score = __fmul_rn(ema, w);
     else score = __uint2float_rn(touch ? epoch : last_epoch);
   } else {
     score = __int_as_float(0x7F800000);  // +inf: not a candidate
@@ -212,11 +227,18 @@ __device__ __forceinline__ EntryVec entry_load4(const EntryState& st, uint64_t v
 
 // touch and last_epoch are only written where an entry was touched.
 __device__ __forceinline__ void entry_finish4(const EntryState& st, uint64_t v, EntryVec& x, const float* sP,
-                                              int policy, uint32_t epoch, float4& sc) {
-  entry_step(x.e.x, x.d.x, x.t.x, x.pr.x, x.st.x, sP, policy, x.le.x, epoch, sc.x);
-  entry_step(x.e.y, x.d.y, x.t.y, x.pr.y, x.st.y, sP, policy, x.le.y, epoch, sc.y);
-  entry_step(x.e.z, x.d.z, x.t.z, x.pr.z, x.st.z, sP, policy, x.le.z, epoch, sc.z);
-  entry_step(x.e.w, x.d.w, x.t.w, x.pr.w, x.st.w, sP, policy, x.le.w, epoch, sc.w);
+                                              int policy, uint32_t epoch, const HeadWeights& hw, float4& sc) {
+  float4 w = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
+  if (hw.on) {
+    w.x = head_weight(hw, 4 * v + 0);
+    w.y = head_weight(hw, 4 * v + 1);
+    w.z = head_weight(hw, 4 * v + 2);
+    w.w = head_weight(hw, 4 * v + 3);
+  }
+  entry_step(x.e.x, x.d.x, x.t.x, x.pr.x, x.st.x, sP, policy, x.le.x, epoch, w.x, sc.x);
+  entry_step(x.e.y, x.d.y, x.t.y, x.pr.y, x.st.y, sP, policy, x.le.y, epoch, w.y, sc.y);
+  entry_step(x.e.z, x.d.z, x.t.z, x.pr.z, x.st.z, sP, policy, x.le.z, epoch, w.z, sc.z);
+  entry_step(x.e.w, x.d.w, x.t.w, x.pr.w, x.st.w, sP, policy, x.le.w, epoch, w.w, sc.w);
   reinterpret_cast<float4*>(st.ema)[v] = x.e;
   reinterpret_cast<float4*>(st.score)[v] = sc;
   // touch counts of FREE entries are always zero (events on them are refused)
@@ -231,11 +253,14 @@ __device__ __forceinline__ void entry_finish4(const EntryState& st, uint64_t v, 
 
 // The same for one entry (ragged ends).
 __device__ __forceinline__ void entry_update1(const EntryState& st, uint64_t i, const float* sP, int policy,
-                                              uint32_t epoch, float& sc, uint32_t& state1) {
+                                              uint32_t epoch, const HeadWeights& hw, float& sc,
+                                              uint32_t& state1) {
   float e = st.ema[i];
   const uint32_t t = __ldcg(&st.touch[i]);
   state1 = st.state[i];
-  entry_step(e, st.decay[i], t, st.pair[i], state1, sP, policy, policy == 2 ? st.last_epoch[i] : 0u, epoch, sc);
+  const float w = hw.on ? head_weight(hw, i) : 1.0f;
+  entry_step(e, st.decay[i], t, st.pair[i], state1, sP, policy, policy == 2 ? st.last_epoch[i] : 0u, epoch, w,
+             sc);
   st.ema[i] = e;
   st.score[i] = sc;
   if (t) {

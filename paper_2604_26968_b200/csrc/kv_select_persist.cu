@@ -71,6 +71,7 @@ struct PArgs {
   // the scoring pass of the fused form
   EntryState st;
   Predictor pd;
+  HeadWeights hw;
   uint32_t epoch;
 };
 
@@ -249,7 +250,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       uint32_t key[4] = {kExcluded, kExcluded, kExcluded, kExcluded};
       if (j0 + 4 <= len) {
         float4 sc;
-        entry_finish4(a.st, i0 / 4, cur, sP, policy, a.epoch, sc);
+        entry_finish4(a.st, i0 / 4, cur, sP, policy, a.epoch, a.hw, sc);
         key[0] = cur.st.x == KV_STATE_RESIDENT ? p_score_key(sc.x) : kExcluded;
         key[1] = cur.st.y == KV_STATE_RESIDENT ? p_score_key(sc.y) : kExcluded;
         key[2] = cur.st.z == KV_STATE_RESIDENT ? p_score_key(sc.z) : kExcluded;
@@ -260,7 +261,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
           if (j0 + j < len) {
             float sc;
             uint32_t s1;
-            entry_update1(a.st, i0 + j, sP, policy, a.epoch, sc, s1);
+            entry_update1(a.st, i0 + j, sP, policy, a.epoch, a.hw, sc, s1);
             if (s1 == KV_STATE_RESIDENT) key[j] = p_score_key(sc);
           }
         }
@@ -500,10 +501,12 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   a.per = ((st.n + G - 1) / G + 3) / 4 * 4;
   a.st = st;
   a.pd = Predictor{};
+  a.hw = HeadWeights{};
   a.epoch = 0;
   if (fs) {
     a.pd = Predictor{fs->hits,       fs->misses,    fs->P,          fs->alpha0, fs->beta0, ws.delta, nullptr,
                      fs->opt.policy, fs->opt.kappa, fs->opt.window, ws.blend};
+    a.hw = fs->hw;
     a.epoch = fs->epoch;
   }
   void* args[] = {&a};

@@ -100,6 +100,8 @@ struct kv_pool {
   int demote_turn = 0, promote_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
   ScoreOptions score_opt;   // eviction policy and confidence blend
+  HeadWeights head{};       // head-granular importance matrices and weights
+  uint32_t n_head_imp = 0, n_head_w = 0;
   // a demotion whose later chunks are not enqueued yet (deferred packing)
   struct Pending {
     bool active = false, meta_done = false;
@@ -122,6 +124,7 @@ struct kv_pool {
 namespace {
 
 struct Layout {
+  uint64_t head_imp, head_mult, head_w;
   uint64_t delta, hist, sel, status, blend, block_score, block_state, block_victims, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
   uint64_t ring[4][5];
   uint64_t dev_total;
@@ -136,6 +139,8 @@ struct Derived {
   uint64_t bases[5];
   uint64_t N;
   uint64_t blocks[4], n_blocks;   // paged blocks (layer x block) per partition and in total
+  uint64_t layers[4], q_heads[4];  // importance matrix of a partition: [layers][q_heads] (q_heads 1 for MLA)
+  uint64_t n_head_imp, n_head_w;   // matrix elements / (layer, KV head) pairs over all partitions
 };
 
 int32_t derive(const kv_pool_desc* d, Derived* out) {
@@ -160,6 +165,17 @@ int32_t derive(const kv_pool_desc* d, Derived* out) {
     out->bases[q] = base;
     base += out->n[q];
     out->blocks[q] = (uint64_t)p.model.n_layers * (uint64_t)p.blocks_per_layer;
+    out->layers[q] = (uint64_t)p.model.n_layers;
+    out->q_heads[q] = (v == KV_MLA) ? 1 : (uint64_t)p.model.n_q_heads;
+    // every KV head serves a whole group of query heads
+    if (out->q_heads[q] < out->heads[q] || out->q_heads[q] % out->heads[q] != 0) return KV_ERR_INVALID_ARG;
+    if (out->layers[q] * out->q_heads[q] >= (1ull << 24)) return KV_ERR_INVALID_ARG;
+    if ((uint64_t)p.blocks_per_layer * out->heads[q] >= (1ull << 32)) return KV_ERR_INVALID_ARG;
+  }
+  out->n_head_imp = out->n_head_w = 0;
+  for (int q = 0; q < d->n_partitions; ++q) {
+    out->n_head_imp += out->layers[q] * out->q_heads[q];
+    out->n_head_w += out->layers[q] * out->heads[q];
   }
   for (int q = d->n_partitions; q <= 4; ++q) out->bases[q] = base;
   if (base == 0 || base >= 0x80000000ull) return KV_ERR_INVALID_ARG;  // ids must fit 31 bits
@@ -178,6 +194,9 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
   L->sel = take(sizeof(SelectScalars));
   L->status = take(4);
   L->blend = take(sizeof(BlendState));
+  L->head_imp = take(g.n_head_imp * 4);
+  L->head_mult = take(g.n_head_w * 4);
+  L->head_w = take(g.n_head_w * 4);
   L->block_score = take(g.n_blocks * 4);
   L->block_state = take(g.n_blocks);
   L->block_victims = take(g.n_blocks * 4);
@@ -465,6 +484,29 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
     ph.h_ring = static_cast<uint8_t*>(desc->part[q].h_ring);
     ph.h_meta = static_cast<uint8_t*>(desc->part[q].h_meta);
   }
+  {
+    HeadWeights& hd = p->head;
+    hd.imp = reinterpret_cast<float*>(w + L.head_imp);
+    hd.mult = reinterpret_cast<float*>(w + L.head_mult);
+    hd.w = reinterpret_cast<float*>(w + L.head_w);
+    hd.on = 0;
+    hd.n_parts = g.n_parts;
+    uint32_t io = 0, wo = 0;
+    for (int q = 0; q < 4; ++q) {
+      const bool in = q < g.n_parts;
+      hd.base[q] = g.bases[q];
+      hd.heads[q] = in ? (uint32_t)g.heads[q] : 1u;
+      hd.q_heads[q] = in ? (uint32_t)g.q_heads[q] : 1u;
+      hd.layers[q] = in ? (uint32_t)g.layers[q] : 0u;
+      hd.per_layer[q] = in ? (uint32_t)(g.n[q] / g.layers[q]) : 1u;
+      hd.imp_off[q] = io;
+      hd.w_off[q] = wo;
+      if (in) { io += hd.layers[q] * hd.q_heads[q]; wo += hd.layers[q] * hd.heads[q]; }
+    }
+    hd.base[4] = g.bases[4];
+    p->n_head_imp = (uint32_t)g.n_head_imp;
+    p->n_head_w = (uint32_t)g.n_head_w;
+  }
   for (int b = 0; b < 4; ++b) p->staging[b] = static_cast<uint8_t*>(desc->d_staging[b]);
   p->staging_bytes = desc->staging_bytes;
   p->bgeom.n_parts = g.n_parts;
@@ -511,6 +553,7 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
     const float p0 = desc->alpha0 / (desc->alpha0 + desc->beta0);
     e = launch_init(p->st, desc->d_hits, desc->d_misses, desc->d_P, p0, desc->d_loc, desc->n_tags,
                     p->geom, p->n_parts, p->ws, S(stream));
+    if (e == cudaSuccess) e = launch_head_init(p->head, p->n_head_imp, p->n_head_w, S(stream));
   }
   if (e != cudaSuccess) {
     for (int i = 0; i < made; ++i) cudaEventDestroy(*evs[i]);
@@ -558,7 +601,7 @@ int32_t kv_epoch_update(kv_pool* p, uint32_t epoch, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
   KV_DRAIN_ALL(p);
   KV_CUDA(p, launch_entry_update(p->st, p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
-                                 p->desc.beta0, p->ws, epoch, p->score_opt, S(stream)));
+                                 p->desc.beta0, p->ws, epoch, p->score_opt, p->head, S(stream)));
   p->stats.epochs += 1;
   return KV_OK;
 }
@@ -568,6 +611,31 @@ int32_t kv_epoch_score(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_entry, c
   const int32_t rc = kv_epoch_events(p, d_ev_entry, d_ev_hit, n_events, stream);
   if (rc != KV_OK) return rc;
   return kv_epoch_update(p, epoch, stream);
+}
+
+int32_t kv_head_importance_update(kv_pool* p, int32_t q, const float* d_x, float decay, kv_stream_t stream) {
+  if (!p || q < 0 || q >= p->n_parts || !d_x || !aligned16(d_x)) return KV_ERR_INVALID_ARG;
+  if (!(decay >= 0.0f) || !(decay <= 1.0f)) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
+  KV_CUDA(p, launch_head_update(p->head, q, 0, d_x, decay, p->ws, S(stream)));
+  p->head.on |= 1u << q;
+  return KV_OK;
+}
+
+int32_t kv_set_head_multipliers(kv_pool* p, int32_t q, const float* d_mult, kv_stream_t stream) {
+  if (!p || q < 0 || q >= p->n_parts || (d_mult && !aligned16(d_mult))) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
+  KV_CUDA(p, launch_head_update(p->head, q, 1, d_mult, 0.0f, p->ws, S(stream)));
+  p->head.on |= 1u << q;
+  return KV_OK;
+}
+
+const float* kv_head_importance(kv_pool* p, int32_t q) {
+  return (p && q >= 0 && q < p->n_parts) ? p->head.imp + p->head.imp_off[q] : nullptr;
+}
+
+const float* kv_head_weights(kv_pool* p, int32_t q) {
+  return (p && q >= 0 && q < p->n_parts) ? p->head.w + p->head.w_off[q] : nullptr;
 }
 
 int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream_t stream) {
@@ -594,7 +662,7 @@ int32_t kv_epoch_score_select(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_e
   bool used = false;
   if (k > 0 && g_select_variant != 0) {
     const FusedScore fs{p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
-                        p->desc.beta0,  epoch,            p->score_opt};
+                        p->desc.beta0,  epoch,            p->score_opt,  p->head};
     KV_CUDA(p, launch_select_persistent(p->st, k, d_victims, p->ws, S(stream), &used, &fs));
   }
   if (used) {

@@ -94,6 +94,23 @@ struct BlockGeom {
   int n_parts;
 };
 
+// Head-granular importance (head-granular eviction section): per partition a
+// [layer][query head] importance matrix, [layer][KV head] multipliers and the
+// resulting [layer][KV head] score weights, each partition's block at its offset.
+struct HeadWeights {
+  float* imp;              // importance matrices, partition q at imp_off[q]
+  float* mult;             // multipliers, partition q at w_off[q]
+  float* w;                // weights, partition q at w_off[q]
+  uint64_t base[5];        // first global entry id of each partition; [n_parts] = N
+  uint32_t per_layer[4];   // entries per layer: blocks per layer x KV heads
+  uint32_t heads[4];       // KV heads (1 for MLA)
+  uint32_t q_heads[4];     // tracked query heads per layer (1 for MLA)
+  uint32_t layers[4];
+  uint32_t imp_off[4], w_off[4];
+  uint32_t on;             // bit q: scores of partition q are weighted
+  int n_parts;
+};
+
 struct Workspace {
   BlendState* blend;
   float* block_score;       // [blocks] aggregate score per paged block
@@ -118,7 +135,13 @@ cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit,
 // folds ws.delta into hits/misses, clears it and writes P
 cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P,
                                 float alpha0, float beta0, const Workspace& ws, uint32_t epoch,
-                                const ScoreOptions& opt, cudaStream_t s);
+                                const ScoreOptions& opt, const HeadWeights& hw, cudaStream_t s);
+// kv_heads.cu: mode 0 = EMA step of partition q's importance matrix with observations
+// src [L][QH]; mode 1 = multipliers of q from src [L][H] (nullptr: all 1).  Both then
+// recompute q's weights.  Values that are negative or not finite are skipped and flagged.
+cudaError_t launch_head_update(const HeadWeights& hw, int q, int mode, const float* src, float decay,
+                               const Workspace& ws, cudaStream_t s);
+cudaError_t launch_head_init(const HeadWeights& hw, uint32_t n_imp, uint32_t n_w, cudaStream_t s);
 // empties the sliding window of the blend (the estimates stay as they are)
 cudaError_t launch_blend_reset(const Workspace& ws, cudaStream_t s);
 
@@ -137,6 +160,7 @@ struct FusedScore {
   float alpha0, beta0;
   uint32_t epoch;
   ScoreOptions opt;
+  HeadWeights hw;
 };
 cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
                                      const Workspace& ws, cudaStream_t s, bool* used,

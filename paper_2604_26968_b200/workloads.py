@@ -133,6 +133,25 @@ class Workload:
             return r.integers(0, 16, size=n, dtype=np.uint8)
         return r.choice(16, size=n, p=self.pair_weights).astype(np.uint8)
 
+    def head_observations(self, epoch: int, q: int) -> np.ndarray:
+        """Per-(layer, query head) observations of one epoch for partition q, float32
+        [layers][query heads] ([layers][1] for MLA): a fixed per-head profile (a few
+        heads matter much more than the rest, later layers more than early ones)
+        times log-normal noise."""
+        p = self.parts[q]
+        qh = 1 if p.variant == MLA else p.n_q_heads
+        prof = np.random.default_rng([self.seed, 77, q]).lognormal(0.0, 1.0, size=(p.n_layers, qh))
+        prof *= np.linspace(0.5, 1.5, p.n_layers)[:, None]
+        noise = self.rng(epoch, 7 + 16 * q).lognormal(0.0, 0.25, size=(p.n_layers, qh))
+        return (prof * noise).astype(np.float32)
+
+    def head_multipliers(self, epoch: int, q: int) -> np.ndarray:
+        """Task-transition multipliers for partition q, float32 [layers][KV heads] in
+        {0.5, 1, 2}."""
+        p = self.parts[q]
+        r = self.rng(epoch, 8 + 16 * q)
+        return r.choice(np.array([0.5, 1.0, 2.0], np.float32), size=(p.n_layers, p.heads)).astype(np.float32)
+
     def events(self, epoch: int, pair: np.ndarray, fresh: Optional[np.ndarray] = None):
         """(ev_entry u32[E], ev_hit u8[E]) of one epoch.
 

@@ -36,7 +36,7 @@ def oracle_admit(w, pool, epoch, key=None):
 
 class Lockstep:
     def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True,
-                 policy=0, blend=None, deferred=False, fused=False):
+                 policy=0, blend=None, deferred=False, fused=False, heads=None):
         self.w = w
         self.payload = payload
         self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
@@ -44,6 +44,9 @@ class Lockstep:
         self.options = (policy, blend)
         self.deferred = deferred
         self.fused = fused   # score and select through the single fused call
+        # heads = (decay, every): importance matrices of all partitions updated before every
+        # epoch's scoring, multipliers set on epochs divisible by `every` and reset on the next
+        self.heads = heads
         if deferred:
             assert self.gpu.pool.kv_set_deferred_packing(True) == 0
         # room for any k a test may ask for
@@ -125,6 +128,32 @@ class Lockstep:
             for c in range(nc):
                 assert np.array_equal(a[:, c][mask], b[:, c][mask]), (where, q, c)
 
+    def head_step(self, e):
+        w, g, o = self.w, self.gpu, self.ora
+        decay, every = self.heads
+        keep = []
+        for q in range(len(w.parts)):
+            x = w.head_observations(e, q)
+            assert o.head_importance_update(q, x, decay) == O.OK
+            d_x = g.to_device(x.reshape(-1), None)
+            keep.append(d_x)
+            g.check(g.pool.kv_head_importance_update(q, d_x, decay), "kv_head_importance_update")
+            if e % every == 0:
+                m = w.head_multipliers(e, q)
+                assert o.set_head_multipliers(q, m) == O.OK
+                d_m = g.to_device(m.reshape(-1), None)
+                keep.append(d_m)
+                g.check(g.pool.kv_set_head_multipliers(q, d_m), "kv_set_head_multipliers")
+            elif e % every == 1:
+                assert o.set_head_multipliers(q, None) == O.OK
+                g.check(g.pool.kv_set_head_multipliers(q, None), "kv_set_head_multipliers")
+        g.pool.sync()
+        for q in range(len(w.parts)):
+            assert np.array_equal(g.pool.kv_head_importance(q).cpu().numpy().view(np.uint32),
+                                  o.head_array(q, "importance").view(np.uint32)), ("importance", e, q)
+            assert np.array_equal(g.pool.kv_head_weights(q).cpu().numpy().view(np.uint32),
+                                  o.head_array(q, "weights").view(np.uint32)), ("weights", e, q)
+
     # ---- one epoch -----------------------------------------------------------
     def epoch(self, e, k=None, check_payload=None, k_blocks=None):
         """One epoch on both sides.  k_blocks selects whole paged blocks instead of k entries."""
@@ -132,6 +161,8 @@ class Lockstep:
         k = w.k if k is None else k
         ev_entry, ev_hit = w.events(e, o.pair, self.fresh)
         d_e, d_h, n = g.stage_events(ev_entry, ev_hit)
+        if self.heads is not None:
+            self.head_step(e)
         assert o.epoch_score(e, ev_entry, ev_hit) == O.OK
         fused = self.fused and k_blocks is None
         if fused:
