@@ -14,20 +14,41 @@ namespace kvt {
 // Each event adds one to the (pair, hit) counter of its entry's pair -- the
 // alpha += 1 / beta += 1 update of the Bayesian reuse section -- and one to the
 // entry's touch count.  Counters are integers, so the order of the atomics does
-// not matter.  Lanes of a warp that hit the same counter are merged first
-// (match.any), then a 32-counter shared-memory table per block, then one 64-bit
-// global atomic per non-zero counter per block.
-__device__ __forceinline__ void count_event(uint32_t key, uint32_t* s_cnt, unsigned lane) {
-  const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
-  if (key < 32 && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&s_cnt[key], __popc(peers));
-}
+// not matter.
+//
+// The 32 (pair, hit) counters are kept one per lane: for every event slot the
+// warp takes six votes (valid, and the five bits of key = 2*pair + hit); lane L
+// combines them into the mask of lanes whose key is L and adds its population
+// count to a register.  No shared-memory atomics and no match instruction in the
+// loop; a warp's 32 registers go to 32 shared counters once, at the end, and a
+// block issues one 64-bit global atomic per non-zero counter.
+struct EventCounter {
+  uint32_t flip[5];  // bit b of the lane id clear -> all ones (selects lanes whose key bit b is clear)
+  uint32_t cnt;      // events seen with key == lane id
+  __device__ __forceinline__ void init(unsigned lane) {
+#pragma unroll
+    for (int b = 0; b < 5; ++b) flip[b] = ((lane >> b) & 1u) ? 0u : 0xFFFFFFFFu;
+    cnt = 0;
+  }
+  // every lane of the warp must call it
+  __device__ __forceinline__ void add(bool counted, uint32_t key) {
+    uint32_t m = __ballot_sync(0xFFFFFFFFu, counted);
+#pragma unroll
+    for (int b = 0; b < 5; ++b) m &= __ballot_sync(0xFFFFFFFFu, (key >> b) & 1u) ^ flip[b];
+    cnt += __popc(m);
+  }
+};
 
 // The calling block's share of the events: thread `gtid` of `stride` takes four
 // consecutive events at a time, so that its four scattered gathers are in flight
 // together.  One byte per event is gathered: the entry's pair, whose bit 7 says
-// that the entry is FREE.  Every thread of the block must call it (the votes
-// need all lanes).  s_cnt: 32 zeroed shared-memory counters, index 2*pair + hit;
-// returns the KV_DEV_* bits of refused events.
+// that the entry is FREE.  Two consecutive events on the two entries of an
+// aligned pair (2i, 2i+1) -- the normal case when a touched block reports all its
+// heads -- share one 64-bit atomic on the two 32-bit touch counts (a carry out of
+// the low count would need 2^32 touches, where the count wraps anyway).  Every
+// thread of the block must call it (the votes need all lanes).  s_cnt: 32 zeroed
+// shared-memory counters, index 2*pair + hit; returns the KV_DEV_* bits of
+// refused events.
 __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ ev_entry,
                                                   const uint8_t* __restrict__ ev_hit, uint64_t n_events,
                                                   const uint8_t* __restrict__ pair,
@@ -36,6 +57,8 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
   const uint64_t n4 = n_events / 4;
   const uint64_t iters = (n4 + stride - 1) / stride;  // same for every thread
   const unsigned lane = threadIdx.x & 31u;
+  EventCounter ec;
+  ec.init(lane);
   uint32_t bad = 0;
   for (uint64_t it = 0; it < iters; ++it) {
     const uint64_t v = it * stride + gtid;
@@ -52,26 +75,29 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
 #pragma unroll
     for (int j = 0; j < 4; ++j)  // all gathers issued before any is used
       pr[j] = (valid && ids[j] < n) ? pair[ids[j]] : kPairFree;
+    bool ok[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      uint32_t key = 32;  // 32 = nothing to count
-      if (valid) {
-        if (ids[j] >= n) {
-          bad |= KV_DEV_EVENT_BAD_ID;
-        } else if (pr[j] & kPairFree) {
-          bad |= KV_DEV_EVENT_NOT_RESIDENT;
-        } else {
-          key = (pr[j] & 15u) * 2u + hit[j];
-          atomicAdd(&touch[ids[j]], 1u);
-        }
-      }
-      count_event(key, s_cnt, lane);
+      ok[j] = valid && ids[j] < n && !(pr[j] & kPairFree);
+      if (valid && !ok[j]) bad |= ids[j] >= n ? KV_DEV_EVENT_BAD_ID : KV_DEV_EVENT_NOT_RESIDENT;
     }
+#pragma unroll
+    for (int j = 0; j < 4; j += 2) {
+      if (ok[j] && ok[j + 1] && ids[j + 1] == ids[j] + 1u && !(ids[j] & 1u)) {
+        atomicAdd(reinterpret_cast<unsigned long long*>(touch + ids[j]), 0x100000001ull);
+      } else {
+        if (ok[j]) atomicAdd(&touch[ids[j]], 1u);
+        if (ok[j + 1]) atomicAdd(&touch[ids[j + 1]], 1u);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) ec.add(ok[j], (pr[j] & 15u) * 2u + hit[j]);
   }
   // ragged tail (n_events not a multiple of 4): first warp of the grid
   if (gtid < 32) {
     const uint64_t e = n4 * 4 + gtid;
-    uint32_t key = 32;
+    bool ok = false;
+    uint32_t key = 0;
     if (e < n_events) {
       const uint32_t i = ev_entry[e];
       const uint32_t pr = i < n ? pair[i] : kPairFree;
@@ -80,12 +106,14 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
       } else if (pr & kPairFree) {
         bad |= KV_DEV_EVENT_NOT_RESIDENT;
       } else {
+        ok = true;
         key = (pr & 15u) * 2u + (ev_hit[e] != 0);
         atomicAdd(&touch[i], 1u);
       }
     }
-    count_event(key, s_cnt, lane);
+    ec.add(ok, key);
   }
+  if (ec.cnt) atomicAdd(&s_cnt[lane], ec.cnt);
   return bad;
 }
 
