@@ -22,6 +22,8 @@ namespace kvt {
 // count to a register.  No shared-memory atomics and no match instruction in the
 // loop; a warp's 32 registers go to 32 shared counters once, at the end, and a
 // block issues one 64-bit global atomic per non-zero counter.
+constexpr uint32_t kEventVecs = 2;  // 4-event vectors a thread has in flight per iteration
+
 struct EventCounter {
   uint32_t flip[5];  // bit b of the lane id clear -> all ones (selects lanes whose key bit b is clear)
   uint32_t cnt;      // events seen with key == lane id
@@ -39,9 +41,9 @@ struct EventCounter {
   }
 };
 
-// The calling block's share of the events: thread `gtid` of `stride` takes four
-// consecutive events at a time, so that its four scattered gathers are in flight
-// together.  One byte per event is gathered: the entry's pair, whose bit 7 says
+// The calling block's share of the events: thread `gtid` of `stride` takes
+// kEventVecs vectors of four consecutive events at a time, so that all their
+// scattered gathers are in flight together.  One byte per event is gathered: the entry's pair, whose bit 7 says
 // that the entry is FREE.  Two consecutive events on the two entries of an
 // aligned pair (2i, 2i+1) -- the normal case when a touched block reports all its
 // heads -- share one 64-bit atomic on the two 32-bit touch counts (a carry out of
@@ -55,43 +57,52 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
                                                   uint32_t* __restrict__ touch, uint64_t n, uint64_t gtid,
                                                   uint64_t stride, uint32_t* s_cnt) {
   const uint64_t n4 = n_events / 4;
-  const uint64_t iters = (n4 + stride - 1) / stride;  // same for every thread
+  const uint64_t iters = (n4 + stride * kEventVecs - 1) / (stride * kEventVecs);  // same for every thread
   const unsigned lane = threadIdx.x & 31u;
   EventCounter ec;
   ec.init(lane);
   uint32_t bad = 0;
   for (uint64_t it = 0; it < iters; ++it) {
-    const uint64_t v = it * stride + gtid;
-    const bool valid = v < n4;
-    uint4 id4 = make_uint4(0, 0, 0, 0);
-    uchar4 h4 = make_uchar4(0, 0, 0, 0);
-    if (valid) {
-      id4 = reinterpret_cast<const uint4*>(ev_entry)[v];
-      h4 = reinterpret_cast<const uchar4*>(ev_hit)[v];
-    }
-    const uint32_t ids[4] = {id4.x, id4.y, id4.z, id4.w};
-    const uint32_t hit[4] = {h4.x != 0, h4.y != 0, h4.z != 0, h4.w != 0};
-    uint32_t pr[4];
+    uint32_t ids[kEventVecs][4], hit[kEventVecs][4], pr[kEventVecs][4];
+    bool valid[kEventVecs];
 #pragma unroll
-    for (int j = 0; j < 4; ++j)  // all gathers issued before any is used
-      pr[j] = (valid && ids[j] < n) ? pair[ids[j]] : kPairFree;
-    bool ok[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      ok[j] = valid && ids[j] < n && !(pr[j] & kPairFree);
-      if (valid && !ok[j]) bad |= ids[j] >= n ? KV_DEV_EVENT_BAD_ID : KV_DEV_EVENT_NOT_RESIDENT;
-    }
-#pragma unroll
-    for (int j = 0; j < 4; j += 2) {
-      if (ok[j] && ok[j + 1] && ids[j + 1] == ids[j] + 1u && !(ids[j] & 1u)) {
-        atomicAdd(reinterpret_cast<unsigned long long*>(touch + ids[j]), 0x100000001ull);
-      } else {
-        if (ok[j]) atomicAdd(&touch[ids[j]], 1u);
-        if (ok[j + 1]) atomicAdd(&touch[ids[j + 1]], 1u);
+    for (uint32_t u = 0; u < kEventVecs; ++u) {  // all event loads first
+      const uint64_t v = (it * kEventVecs + u) * stride + gtid;
+      valid[u] = v < n4;
+      uint4 id4 = make_uint4(0, 0, 0, 0);
+      uchar4 h4 = make_uchar4(0, 0, 0, 0);
+      if (valid[u]) {
+        id4 = reinterpret_cast<const uint4*>(ev_entry)[v];
+        h4 = reinterpret_cast<const uchar4*>(ev_hit)[v];
       }
+      ids[u][0] = id4.x; ids[u][1] = id4.y; ids[u][2] = id4.z; ids[u][3] = id4.w;
+      hit[u][0] = h4.x != 0; hit[u][1] = h4.y != 0; hit[u][2] = h4.z != 0; hit[u][3] = h4.w != 0;
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) ec.add(ok[j], (pr[j] & 15u) * 2u + hit[j]);
+    for (uint32_t u = 0; u < kEventVecs; ++u)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)  // then all gathers, before any is used
+        pr[u][j] = (valid[u] && ids[u][j] < n) ? pair[ids[u][j]] : kPairFree;
+#pragma unroll
+    for (uint32_t u = 0; u < kEventVecs; ++u) {
+      bool ok[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        ok[j] = valid[u] && ids[u][j] < n && !(pr[u][j] & kPairFree);
+        if (valid[u] && !ok[j]) bad |= ids[u][j] >= n ? KV_DEV_EVENT_BAD_ID : KV_DEV_EVENT_NOT_RESIDENT;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; j += 2) {
+        if (ok[j] && ok[j + 1] && ids[u][j + 1] == ids[u][j] + 1u && !(ids[u][j] & 1u)) {
+          atomicAdd(reinterpret_cast<unsigned long long*>(touch + ids[u][j]), 0x100000001ull);
+        } else {
+          if (ok[j]) atomicAdd(&touch[ids[u][j]], 1u);
+          if (ok[j + 1]) atomicAdd(&touch[ids[u][j + 1]], 1u);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) ec.add(ok[j], (pr[u][j] & 15u) * 2u + hit[u][j]);
+    }
   }
   // ragged tail (n_events not a multiple of 4): first warp of the grid
   if (gtid < 32) {
