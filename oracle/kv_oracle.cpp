@@ -147,6 +147,7 @@ struct Part {
   std::vector<uint8_t> slab;  // paged HBM image (payload mode only)
   std::vector<uint8_t> ring;  // host ring image (payload mode only)
   std::vector<uint32_t> r_tag, r_last_epoch;
+  std::vector<uint32_t> r_depoch;  // epoch in which the slot's block was demoted
   std::vector<float> r_ema, r_decay;
   std::vector<uint8_t> r_pair, r_live;
   // head-granular importance (see okv_head_importance_update)
@@ -175,6 +176,8 @@ struct Pool {
   std::vector<uint64_t> win;      // [window][32] per-epoch counts, index 2*pair + hit
   uint64_t wsum[32] = {0};        // sums over the window
   float estimate[16] = {0};       // reuse estimate used for scoring
+  int lazy_decay = 0;             // promotion applies the EMA steps missed on the host
+  uint32_t cur_epoch = 0;         // epoch of the last scoring pass
   std::vector<float> ema, decay, score;
   std::vector<uint32_t> touch, last_epoch, tag;
   std::vector<uint8_t> pair, state;
@@ -299,6 +302,7 @@ void* okv_create(int32_t n_parts, const PartDesc* parts, float alpha0, float bet
     }
     pt.r_tag.assign((size_t)pt.R, NONE);
     pt.r_last_epoch.assign((size_t)pt.R, 0);
+    pt.r_depoch.assign((size_t)pt.R, 0);
     pt.r_ema.assign((size_t)pt.R, 0.0f);
     pt.r_decay.assign((size_t)pt.R, 0.0f);
     pt.r_pair.assign((size_t)pt.R, 0);
@@ -365,7 +369,7 @@ void* okv_array(void* h, int32_t which) {
 }
 
 // Per-partition views. which: 0 slab u8, 1 ring u8, 2 r_tag u32, 3 r_pair u8,
-// 4 r_ema f32, 5 r_decay f32, 6 r_last_epoch u32, 7 r_live u8
+// 4 r_ema f32, 5 r_decay f32, 6 r_last_epoch u32, 7 r_live u8, 8 r_depoch u32
 void* okv_part_array(void* h, int32_t q, int32_t which) {
   Pool* p = static_cast<Pool*>(h);
   if (q < 0 || q >= p->n_parts) return nullptr;
@@ -379,6 +383,7 @@ void* okv_part_array(void* h, int32_t q, int32_t which) {
     case 5: return pt.r_decay.data();
     case 6: return pt.r_last_epoch.data();
     case 7: return pt.r_live.data();
+    case 8: return pt.r_depoch.data();
     default: return nullptr;
   }
 }
@@ -414,6 +419,12 @@ void okv_get_stats(void* h, uint64_t* out8) {
 }
 
 uint64_t okv_next_tag(void* h) { return static_cast<Pool*>(h)->next_tag; }
+
+// Lazy decay of promoted entries: off (default) restores the EMA verbatim.
+int32_t okv_set_lazy_decay(void* h, int32_t on) {
+  static_cast<Pool*>(h)->lazy_decay = on ? 1 : 0;
+  return OK;
+}
 
 // Eviction policy: 0 Bayesian (default), 1 EMA only, 2 LRU.
 int32_t okv_set_policy(void* h, int32_t policy) {
@@ -509,6 +520,7 @@ int32_t okv_epoch_score(void* h, uint32_t epoch, const uint32_t* ev_entry, const
     if ((int64_t)ev_entry[e] >= p->N || p->state[ev_entry[e]] != ST_RESIDENT)
       return ERR_INVALID_ARG;
   }
+  p->cur_epoch = epoch;
   // step 1
   uint64_t epoch_hits[16] = {0}, epoch_misses[16] = {0};
   for (uint64_t e = 0; e < n_events; ++e) {
@@ -685,6 +697,7 @@ int32_t okv_demote(void* h, const uint32_t* victims, uint64_t m) {
     pt.r_ema[slot] = p->ema[v];
     pt.r_decay[slot] = p->decay[v];
     pt.r_last_epoch[slot] = p->last_epoch[v];
+    pt.r_depoch[slot] = p->cur_epoch;
     pt.r_live[slot] = 1;
     p->loc[p->tag[v]] = HOST_BIT | (uint32_t)slot;
     p->state[v] = ST_FREE;
@@ -698,7 +711,13 @@ int32_t okv_demote(void* h, const uint32_t* victims, uint64_t m) {
 }
 
 // Promotion: the j-th listed host slot goes to the j-th lowest FREE entry of
-// the partition; its metadata is restored as it was when demoted.
+// the partition; its metadata is restored as it was when demoted.  With lazy
+// decay on (okv_set_lazy_decay) the EMA first catches up on the scoring passes
+// it missed: a resident entry that nobody touches goes ema <- decay*ema + (1 -
+// decay)*0 = decay*ema per pass, so a block demoted in epoch e_d and promoted
+// after the pass of epoch e_p takes e_p - e_d such steps, one rounded multiply
+// each [reading: the paper does not say what happens to importance while a block
+// is in a lower tier].
 int32_t okv_promote(void* h, int32_t q, const uint64_t* slots, uint64_t m) {
   Pool* p = static_cast<Pool*>(h);
   if (q < 0 || q >= p->n_parts) return ERR_INVALID_ARG;
@@ -720,6 +739,11 @@ int32_t okv_promote(void* h, int32_t q, const uint64_t* slots, uint64_t m) {
       copy_image_to_entry(pt, f - pt.base, pt.ring.data() + slot * (uint64_t)pt.entry_bytes);
     p->pair[f] = pt.r_pair[slot];
     p->ema[f] = pt.r_ema[slot];
+    if (p->lazy_decay && p->cur_epoch > pt.r_depoch[slot]) {
+      // one untouched EMA step per scoring pass the block sat out on the host
+      const uint32_t missed = p->cur_epoch - pt.r_depoch[slot];
+      for (uint32_t s = 0; s < missed; ++s) p->ema[f] = pt.r_decay[slot] * p->ema[f];
+    }
     p->decay[f] = pt.r_decay[slot];
     p->last_epoch[f] = pt.r_last_epoch[slot];
     p->tag[f] = pt.r_tag[slot];

@@ -70,6 +70,8 @@ def lib():
         L.okv_next_tag.argtypes = [C.c_void_p]
         L.okv_set_policy.restype = C.c_int32
         L.okv_set_policy.argtypes = [C.c_void_p, C.c_int32]
+        L.okv_set_lazy_decay.restype = C.c_int32
+        L.okv_set_lazy_decay.argtypes = [C.c_void_p, C.c_int32]
         L.okv_set_confidence_blend.restype = C.c_int32
         L.okv_set_confidence_blend.argtypes = [C.c_void_p, C.c_float, C.c_int32]
         L.okv_estimate.restype = C.c_void_p
@@ -140,7 +142,7 @@ class OraclePool:
             "tag": (6, np.uint32), "score": (7, np.float32)}
     _PARR = {"slab": (0, np.uint8), "ring": (1, np.uint8), "r_tag": (2, np.uint32),
              "r_pair": (3, np.uint8), "r_ema": (4, np.float32), "r_decay": (5, np.float32),
-             "r_last_epoch": (6, np.uint32), "r_live": (7, np.uint8)}
+             "r_last_epoch": (6, np.uint32), "r_live": (7, np.uint8), "r_depoch": (8, np.uint32)}
 
     def __init__(self, parts, alpha0=1.0, beta0=1.0, n_tags=None, payload=True):
         L = lib()
@@ -198,6 +200,10 @@ class OraclePool:
 
     def set_policy(self, policy):
         return lib().okv_set_policy(self._h, policy)
+
+    def set_lazy_decay(self, on=True):
+        """Promoted entries catch up on the EMA steps they missed while on the host."""
+        return lib().okv_set_lazy_decay(self._h, int(bool(on)))
 
     def set_confidence_blend(self, kappa, window):
         return lib().okv_set_confidence_blend(self._h, kappa, window)
