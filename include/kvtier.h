@@ -130,7 +130,7 @@ typedef struct {
   float ema;
   float decay;
   uint32_t pair;
-  uint32_t reserved;
+  uint32_t demote_epoch; /* epoch of the pool's last scoring pass when the block was demoted */
 } kv_slot_meta; /* 24 bytes */
 
 typedef struct {
@@ -305,9 +305,24 @@ int32_t kv_demote(kv_pool* pool, const uint32_t* d_victims, uint64_t m, uint64_t
  * call; all live and distinct) into partition `partition`: runs of consecutive
  * slots are copied to staging on `copy`, and the j-th listed entry is scattered
  * into the j-th lowest FREE slot of the partition on `compute`, with the pair,
- * EMA, decay, last epoch and tag it had when demoted; the host slot dies. */
+ * EMA, decay, last epoch and tag it had when demoted (the EMA decayed for the
+ * passes it missed if kv_set_lazy_decay is on); the host slot dies. */
 int32_t kv_promote(kv_pool* pool, int32_t partition, const uint64_t* h_host_slots, uint64_t m,
                    uint64_t batch_bytes, kv_stream_t compute, kv_stream_t copy);
+
+/* Lazy decay of promoted entries (off by default).  The head-granular eviction
+ * section updates importance on every step for blocks in HBM; the paper does not
+ * say what a block's importance is when it returns from a lower tier.  Off, the
+ * EMA comes back exactly as it left.  On, kv_promote first applies the EMA steps
+ * the block missed: a resident entry that nobody touches goes
+ *   ema <- decay*ema + (1-decay)*0 = decay*ema
+ * per scoring pass, so a block demoted after the pass of epoch e_d and promoted
+ * after the pass of epoch e_p takes e_p - e_d such steps (binary32, one rounded
+ * multiply each) and ends with exactly the EMA of an entry that stayed resident
+ * and untouched.  "Epoch" is the one given to the pool's last kv_epoch_score /
+ * kv_epoch_update / kv_epoch_score_select; each ring slot remembers it
+ * (kv_slot_meta.demote_epoch).  Takes effect for promotions enqueued after the call. */
+int32_t kv_set_lazy_decay(kv_pool* pool, int32_t on);
 
 /* Block-granular selection (head-granular eviction section: eviction takes the
  * block with the lowest weighted aggregate importance across heads, with head

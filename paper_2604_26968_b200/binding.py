@@ -71,15 +71,15 @@ class kv_timing(C.Structure):
 
 class kv_slot_meta(C.Structure):
     _fields_ = [("tag", C.c_uint32), ("last_epoch", C.c_uint32), ("ema", C.c_float),
-                ("decay", C.c_float), ("pair", C.c_uint32), ("reserved", C.c_uint32)]
+                ("decay", C.c_float), ("pair", C.c_uint32), ("demote_epoch", C.c_uint32)]
 
 
 SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"),
-                            ("decay", "<f4"), ("pair", "<u4"), ("reserved", "<u4")])
+                            ("decay", "<f4"), ("pair", "<u4"), ("demote_epoch", "<u4")])
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
            "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_score_select", "kv_epoch_events", "kv_epoch_counts",
-           "kv_epoch_update", "kv_set_policy", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
+           "kv_epoch_update", "kv_set_policy", "kv_set_lazy_decay", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
            "kv_set_move_variant", "kv_set_select_variant", "kv_last_cuda_error", "kv_status_string",
@@ -122,6 +122,8 @@ def load():
     L.kv_epoch_update.argtypes = [vp, u32, vp]
     L.kv_set_policy.restype = i32
     L.kv_set_policy.argtypes = [vp, i32]
+    L.kv_set_lazy_decay.restype = i32
+    L.kv_set_lazy_decay.argtypes = [vp, i32]
     L.kv_set_confidence_blend.restype = i32
     L.kv_set_confidence_blend.argtypes = [vp, C.c_float, i32, vp]
     L.kv_reuse_estimate.restype = vp
@@ -348,6 +350,9 @@ class Pool:
 
     def kv_set_policy(self, policy):
         return self.lib.kv_set_policy(self._h, int(policy))
+
+    def kv_set_lazy_decay(self, on=True):
+        return self.lib.kv_set_lazy_decay(self._h, int(bool(on)))
 
     def kv_set_confidence_blend(self, kappa, window):
         return self.lib.kv_set_confidence_blend(self._h, float(kappa), int(window), _stream_ptr(self.compute))

@@ -81,6 +81,7 @@ pack_kernel(const PartGeom g, const EntryState st, uint32_t* __restrict__ loc,
       g.r_ema[slot] = em;
       g.r_decay[slot] = de;
       g.r_last_epoch[slot] = le;
+      g.r_depoch[slot] = g.epoch_now;
       loc[t] = KV_LOC_HOST | slot;
       st.state[v] = KV_STATE_FREE;
       st.pair[v] = (uint8_t)(pr | kPairFree);
@@ -93,7 +94,7 @@ pack_kernel(const PartGeom g, const EntryState st, uint32_t* __restrict__ loc,
         rec[2] = __float_as_uint(em);
         rec[3] = __float_as_uint(de);
         rec[4] = pr;
-        rec[5] = 0;
+        rec[5] = g.epoch_now;
       }
     }
   }
@@ -153,8 +154,11 @@ unpack_kernel(const PartGeom g, const EntryState st, uint32_t* __restrict__ loc,
         continue;
       }
       st.pair[f] = g.r_pair[slot];
-      st.ema[f] = g.r_ema[slot];
-      st.decay[f] = g.r_decay[slot];
+      const float de = g.r_decay[slot];
+      float em = g.r_ema[slot];
+      if (g.lazy_decay && g.epoch_now > g.r_depoch[slot]) em = ema_catch_up(em, de, g.epoch_now - g.r_depoch[slot]);
+      st.ema[f] = em;
+      st.decay[f] = de;
       st.last_epoch[f] = g.r_last_epoch[slot];
       st.tag[f] = t;
       st.touch[f] = 0;
@@ -276,6 +280,7 @@ __global__ void __launch_bounds__(kThreads) init_ring_kernel(const PartGeom g) {
   for (uint64_t s = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; s < g.ring_slots; s += stride) {
     g.r_tag[s] = KV_NONE;
     g.r_last_epoch[s] = 0;
+    g.r_depoch[s] = 0;
     g.r_ema[s] = 0.0f;
     g.r_decay[s] = 0.0f;
     g.r_pair[s] = 0;

@@ -126,6 +126,7 @@ __device__ __forceinline__ void demote_meta(const MoveArgs& a, uint64_t j, uint3
   g.r_ema[slot] = em;
   g.r_decay[slot] = de;
   g.r_last_epoch[slot] = le;
+  g.r_depoch[slot] = g.epoch_now;
   a.loc[t] = KV_LOC_HOST | slot;
   st.state[v] = KV_STATE_FREE;
   st.pair[v] = (uint8_t)(pr | kPairFree);
@@ -138,11 +139,12 @@ __device__ __forceinline__ void demote_meta(const MoveArgs& a, uint64_t j, uint3
     rec[2] = __float_as_uint(em);
     rec[3] = __float_as_uint(de);
     rec[4] = pr;
-    rec[5] = 0;
+    rec[5] = g.epoch_now;
   }
 }
 
-// Metadata of one promoted entry: restored as it was when demoted.
+// Metadata of one promoted entry: restored as it was when demoted (with lazy decay on,
+// the EMA first takes the steps it missed).
 __device__ __forceinline__ void promote_meta(const MoveArgs& a, uint32_t f, uint32_t slot) {
   const PartGeom& g = a.g;
   const EntryState& st = a.st;
@@ -152,8 +154,11 @@ __device__ __forceinline__ void promote_meta(const MoveArgs& a, uint32_t f, uint
     return;
   }
   st.pair[f] = g.r_pair[slot];
-  st.ema[f] = g.r_ema[slot];
-  st.decay[f] = g.r_decay[slot];
+  const float de = g.r_decay[slot];
+  float em = g.r_ema[slot];
+  if (g.lazy_decay && g.epoch_now > g.r_depoch[slot]) em = ema_catch_up(em, de, g.epoch_now - g.r_depoch[slot]);
+  st.ema[f] = em;
+  st.decay[f] = de;
   st.last_epoch[f] = g.r_last_epoch[slot];
   st.tag[f] = t;
   st.touch[f] = 0;
@@ -196,7 +201,7 @@ move_tma_kernel(const MoveArgs a) {
             rec[2] = __float_as_uint(g.r_ema[slot]);
             rec[3] = __float_as_uint(g.r_decay[slot]);
             rec[4] = g.r_pair[slot];
-            rec[5] = 0;
+            rec[5] = g.r_depoch[slot];
           }
           continue;
         }

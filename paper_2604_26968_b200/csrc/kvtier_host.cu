@@ -126,7 +126,7 @@ namespace {
 struct Layout {
   uint64_t head_imp, head_mult, head_w;
   uint64_t delta, hist, sel, status, blend, block_score, block_state, block_victims, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
-  uint64_t ring[4][5];
+  uint64_t ring[4][6];
   uint64_t dev_total;
   uint64_t h_list[2], h_counts, h_status, host_total;
   uint32_t n_tiles;
@@ -210,6 +210,7 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
     const uint64_t R = d->part[q].ring_slots;
     for (int a = 0; a < 4; ++a) L->ring[q][a] = take(R * 4);
     L->ring[q][4] = take(R);
+    L->ring[q][5] = take(R * 4);
   }
   L->dev_total = o;
   uint64_t h = 0;
@@ -477,6 +478,9 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
     pg.r_ema = reinterpret_cast<float*>(w + L.ring[q][2]);
     pg.r_decay = reinterpret_cast<float*>(w + L.ring[q][3]);
     pg.r_pair = w + L.ring[q][4];
+    pg.r_depoch = reinterpret_cast<uint32_t*>(w + L.ring[q][5]);
+    pg.epoch_now = 0;
+    pg.lazy_decay = 0;
     PartHost& ph = p->host[q];
     ph.variant = g.variant[q];
     ph.n_free = g.n[q];
@@ -603,6 +607,7 @@ int32_t kv_epoch_update(kv_pool* p, uint32_t epoch, kv_stream_t stream) {
   KV_CUDA(p, launch_entry_update(p->st, p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
                                  p->desc.beta0, p->ws, epoch, p->score_opt, p->head, S(stream)));
   p->stats.epochs += 1;
+  for (int q = 0; q < p->n_parts; ++q) p->geom[q].epoch_now = epoch;
   return KV_OK;
 }
 
@@ -667,6 +672,7 @@ int32_t kv_epoch_score_select(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_e
   }
   if (used) {
     p->stats.epochs += 1;
+    for (int q = 0; q < p->n_parts; ++q) p->geom[q].epoch_now = epoch;
     return KV_OK;
   }
   const int32_t rc = kv_epoch_update(p, epoch, stream);
@@ -943,6 +949,12 @@ int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) 
   KV_CUDA(p, cudaMemsetAsync(p->ws.status, 0, 4, S(stream)));
   KV_CUDA(p, cudaStreamSynchronize(S(stream)));
   *status_bits = *p->h_status;
+  return KV_OK;
+}
+
+int32_t kv_set_lazy_decay(kv_pool* p, int32_t on) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  for (int q = 0; q < p->n_parts; ++q) p->geom[q].lazy_decay = on ? 1u : 0u;
   return KV_OK;
 }
 

@@ -38,7 +38,23 @@ struct PartGeom {
   float* r_ema;
   float* r_decay;
   uint8_t* r_pair;
+  uint32_t* r_depoch;    // epoch in which the slot's block was demoted
+  uint32_t epoch_now;    // epoch of the pool's last scoring pass (set by the host before a launch)
+  uint32_t lazy_decay;   // promotion applies the EMA steps missed on the host
 };
+
+// EMA of a block that sat out `missed` scoring passes untouched: every pass is
+// ema <- decay*ema + (1 - decay)*0 = decay*ema, one rounded multiply.  Stops early
+// at a fixed point (0, decay 1, or a denormal that no longer shrinks), where
+// further steps change nothing.
+__device__ __forceinline__ float ema_catch_up(float ema, float decay, uint32_t missed) {
+  for (uint32_t s = 0; s < missed; ++s) {
+    const float nx = __fmul_rn(decay, ema);
+    if (nx == ema) break;
+    ema = nx;
+  }
+  return ema;
+}
 
 // Per-entry state arrays.
 struct EntryState {

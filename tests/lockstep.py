@@ -36,7 +36,7 @@ def oracle_admit(w, pool, epoch, key=None):
 
 class Lockstep:
     def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True,
-                 policy=0, blend=None, deferred=False, fused=False, heads=None):
+                 policy=0, blend=None, deferred=False, fused=False, heads=None, lazy=False):
         self.w = w
         self.payload = payload
         self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
@@ -59,6 +59,8 @@ class Lockstep:
         if blend is not None:
             assert self.ora.set_confidence_blend(*blend) == O.OK
             assert self.gpu.pool.kv_set_confidence_blend(*blend) == 0
+        if lazy:   # promoted entries catch up on the EMA steps they missed on the host
+            assert self.ora.set_lazy_decay(True) == O.OK and self.gpu.pool.kv_set_lazy_decay(True) == 0
         self.compare_state("initial fill")
         if payload:
             self.compare_payload("initial fill")
@@ -103,6 +105,7 @@ class Lockstep:
             for name in ("tag", "pair", "last_epoch"):
                 assert np.array_equal(meta[name.replace("r_", "")][lv].astype(np.uint32),
                                       o.part_array(q, "r_" + name)[lv].astype(np.uint32)), (where, name)
+            assert np.array_equal(meta["demote_epoch"][lv], o.part_array(q, "r_depoch")[lv]), (where, "demote_epoch")
             for name in ("ema", "decay"):
                 assert np.array_equal(meta[name][lv].view(np.uint32),
                                       o.part_array(q, "r_" + name)[lv].view(np.uint32)), (where, name)
