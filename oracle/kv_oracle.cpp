@@ -420,6 +420,17 @@ void okv_get_stats(void* h, uint64_t* out8) {
 
 uint64_t okv_next_tag(void* h) { return static_cast<Pool*>(h)->next_tag; }
 
+// The image of entry `id` as the host tier and the content hash see it: K chunk
+// then V chunk (or the single MLA chunk).  out holds entry_bytes; returns that
+// size, or a negative status (payload mode only).
+int64_t okv_entry_image(void* h, uint32_t id, uint8_t* out) {
+  Pool* p = static_cast<Pool*>(h);
+  if (!p->payload || (int64_t)id >= p->N || !out) return ERR_INVALID_ARG;
+  const Part& pt = p->part[part_of(*p, id)];
+  copy_entry_to_image(pt, (int64_t)id - pt.base, out);
+  return pt.entry_bytes;
+}
+
 // Lazy decay of promoted entries: off (default) restores the EMA verbatim.
 int32_t okv_set_lazy_decay(void* h, int32_t on) {
   static_cast<Pool*>(h)->lazy_decay = on ? 1 : 0;

@@ -70,6 +70,8 @@ def lib():
         L.okv_next_tag.argtypes = [C.c_void_p]
         L.okv_set_policy.restype = C.c_int32
         L.okv_set_policy.argtypes = [C.c_void_p, C.c_int32]
+        L.okv_entry_image.restype = C.c_int64
+        L.okv_entry_image.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         L.okv_set_lazy_decay.restype = C.c_int32
         L.okv_set_lazy_decay.argtypes = [C.c_void_p, C.c_int32]
         L.okv_set_confidence_blend.restype = C.c_int32
@@ -258,6 +260,19 @@ class OraclePool:
                  "bytes_promoted", "bytes_dropped")
         return {n: int(v) for n, v in zip(names, out)}
 
+    def entry_image(self, i):
+        """Bytes of entry i as one image: K chunk then V chunk (or the MLA chunk)."""
+        q = max(q for q in range(self.n_parts) if self.info(q)["base"] <= i)
+        out = np.zeros(self.info(q)["entry_bytes"], dtype=np.uint8)
+        assert lib().okv_entry_image(self._h, int(i), _ptr(out)) == out.size
+        return out
+
+    def entry_digests(self, ids):
+        """SHA-256 of each listed entry's image (content-addressable deduplication
+        section: blocks are indexed by the SHA-256 hash of their content); uint8 [m, 32]."""
+        return np.stack([sha256_bytes(self.entry_image(i)) for i in ids]) if len(ids) else \
+            np.zeros((0, 32), np.uint8)
+
     def epoch_score(self, epoch, ev_entry, ev_hit):
         ev_entry = np.ascontiguousarray(ev_entry, dtype=np.uint32)
         ev_hit = np.ascontiguousarray(ev_hit, dtype=np.uint8)
@@ -289,3 +304,29 @@ class OraclePool:
             new_payload = np.ascontiguousarray(new_payload, dtype=np.uint8)
         return int(lib().okv_admit(self._h, epoch, decay, _ptr(new_pairs), new_pairs.size,
                                    _ptr(new_payload) if new_payload is not None else None))
+
+
+# ---- content-addressable deduplication -----------------------------------------
+def sha256_bytes(data):
+    """SHA-256 (FIPS 180-4) of a byte string, as 32 uint8; the library routine is the step."""
+    import hashlib
+    return np.frombuffer(hashlib.sha256(bytes(memoryview(np.ascontiguousarray(data)))).digest(), dtype=np.uint8)
+
+
+def dedup(digests):
+    """Deduplication of a list of blocks by content hash (content-addressable
+    deduplication section: a new block's hash is checked against the store; on a
+    match a reference count is incremented instead of duplicating the block).
+    Blocks are taken in list order, so the first block with a digest is the stored
+    copy.  Returns (canon, refcount, n_unique): canon[j] = position of the stored
+    copy block j refers to (j itself if it is the copy), refcount[i] = references
+    to stored copy i, itself included (0 for blocks that are not stored)."""
+    digests = np.asarray(digests, dtype=np.uint8).reshape(-1, 32)
+    store = {}
+    canon = np.zeros(len(digests), np.uint32)
+    refcount = np.zeros(len(digests), np.uint32)
+    for j, d in enumerate(digests):
+        i = store.setdefault(d.tobytes(), j)
+        canon[j] = i
+        refcount[i] += 1
+    return canon, refcount, len(store)
