@@ -324,6 +324,39 @@ int32_t kv_promote(kv_pool* pool, int32_t partition, const uint64_t* h_host_slot
  * (kv_slot_meta.demote_epoch).  Takes effect for promotions enqueued after the call. */
 int32_t kv_set_lazy_decay(kv_pool* pool, int32_t on);
 
+/* Content hashing (content-addressable deduplication section: blocks are indexed
+ * by the SHA-256 hash of their content).  Writes to d_digests (device, 32 bytes
+ * per entry, in the byte order the standard prints) the SHA-256 digest (FIPS
+ * 180-4) of the image of each of the m entries listed in d_ids (device, u32 global
+ * ids; NULL = entries 0..m-1): the entry's K chunk followed by its V chunk, or its
+ * single MLA chunk, exactly the bytes kv_demote would send to the host ring.  The
+ * entries need not be RESIDENT (a FREE slot's bytes are whatever was left there).
+ * An id >= N sets KV_DEV_BAD_INDEX and leaves its digest unwritten. */
+int32_t kv_hash_entries(kv_pool* pool, const uint32_t* d_ids, uint64_t m, uint8_t* d_digests,
+                        kv_stream_t stream);
+
+/* Deduplication by content hash (same section: when a new block's hash is already
+ * in the store, a reference count is incremented instead of duplicating the block;
+ * the paper keeps the store in a radix tree on the CPU, here it is an
+ * open-addressing table on the GPU).  The m digests are taken as a list of blocks
+ * entering the store in list order, so the first block with a given digest is the
+ * stored copy:
+ *   d_canon[j]    (device, u32[m]) position of the stored copy that block j refers
+ *                 to; j itself if block j is the stored copy
+ *   d_refcount[i] (device, u32[m]) references to stored copy i, itself included; 0
+ *                 for blocks that are not stored
+ *   d_n_unique    (device, optional) one u32: number of stored copies; the bytes
+ *                 saved are (m - n_unique) * entry_bytes
+ * The result does not depend on thread scheduling (the smallest position wins).
+ * d_table (device) is scratch of table_slots u32, table_slots a power of two >=
+ * kv_dedup_table_slots(m) = 2*m rounded up; d_status (device, one u32 the caller
+ * zeroes) receives KV_DEV_* bits if the table was found inconsistent.  m < 2^32-1.
+ * Pointers 16-byte aligned.  Needs no pool. */
+uint64_t kv_dedup_table_slots(uint64_t m);
+int32_t kv_dedup_digests(const uint8_t* d_digests, uint64_t m, uint32_t* d_canon, uint32_t* d_refcount,
+                         uint32_t* d_table, uint64_t table_slots, uint32_t* d_n_unique,
+                         uint32_t* d_status, kv_stream_t stream);
+
 /* Block-granular selection (head-granular eviction section: eviction takes the
  * block with the lowest weighted aggregate importance across heads, with head
  * weights uniform for MHA and proportional to the group size for GQA).  The

@@ -26,6 +26,7 @@ KV_AUTO, KV_MHA, KV_GQA, KV_MQA, KV_MLA = -1, 0, 1, 2, 3
 KV_STATE_FREE, KV_STATE_RESIDENT = 0, 1
 KV_POLICY_BAYESIAN, KV_POLICY_EMA, KV_POLICY_LRU = 0, 1, 2
 KV_NONE = 0xFFFFFFFF
+KV_DEV_BAD_INDEX = 16
 KV_DEV_BAD_HEAD_VALUE = 64
 KV_LOC_HOST = 0x80000000
 
@@ -79,7 +80,7 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
            "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_score_select", "kv_epoch_events", "kv_epoch_counts",
-           "kv_epoch_update", "kv_set_policy", "kv_set_lazy_decay", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
+           "kv_epoch_update", "kv_set_policy", "kv_set_lazy_decay", "kv_hash_entries", "kv_dedup_table_slots", "kv_dedup_digests", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
            "kv_set_move_variant", "kv_set_select_variant", "kv_last_cuda_error", "kv_status_string",
@@ -124,6 +125,12 @@ def load():
     L.kv_set_policy.argtypes = [vp, i32]
     L.kv_set_lazy_decay.restype = i32
     L.kv_set_lazy_decay.argtypes = [vp, i32]
+    L.kv_hash_entries.restype = i32
+    L.kv_hash_entries.argtypes = [vp, vp, u64, vp, vp]
+    L.kv_dedup_table_slots.restype = u64
+    L.kv_dedup_table_slots.argtypes = [u64]
+    L.kv_dedup_digests.restype = i32
+    L.kv_dedup_digests.argtypes = [vp, u64, vp, vp, vp, u64, vp, vp, vp]
     L.kv_set_confidence_blend.restype = i32
     L.kv_set_confidence_blend.argtypes = [vp, C.c_float, i32, vp]
     L.kv_reuse_estimate.restype = vp
@@ -214,6 +221,18 @@ def kv_set_move_variant(variant: int) -> int:
 
 def _stream_ptr(s):
     return C.c_void_p(s.cuda_stream if s is not None else 0)
+
+
+def kv_dedup_table_slots(m: int) -> int:
+    return int(load().kv_dedup_table_slots(int(m)))
+
+
+def kv_dedup_digests(d_digests, m, d_canon, d_refcount, d_table, d_n_unique, d_status, stream=None) -> int:
+    """First position per digest and reference counts; arguments are torch device tensors."""
+    return load().kv_dedup_digests(d_digests.data_ptr(), int(m), d_canon.data_ptr(), d_refcount.data_ptr(),
+                                   d_table.data_ptr(), int(d_table.numel()),
+                                   d_n_unique.data_ptr() if d_n_unique is not None else None,
+                                   d_status.data_ptr(), _stream_ptr(stream) if stream is not None else None)
 
 
 def kv_select_victims_static(d_score, d_state, n, k, d_victims, d_status=None, stream=None) -> int:
@@ -350,6 +369,11 @@ class Pool:
 
     def kv_set_policy(self, policy):
         return self.lib.kv_set_policy(self._h, int(policy))
+
+    def kv_hash_entries(self, d_ids, m, d_digests):
+        """SHA-256 of the images of entries d_ids[:m] (None: entries 0..m-1) into d_digests (uint8 [m, 32])."""
+        return self.lib.kv_hash_entries(self._h, d_ids.data_ptr() if d_ids is not None else None, int(m),
+                                        d_digests.data_ptr(), _stream_ptr(self.compute))
 
     def kv_set_lazy_decay(self, on=True):
         return self.lib.kv_set_lazy_decay(self._h, int(bool(on)))

@@ -952,6 +952,35 @@ int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) 
   return KV_OK;
 }
 
+int32_t kv_hash_entries(kv_pool* p, const uint32_t* d_ids, uint64_t m, uint8_t* d_digests, kv_stream_t stream) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
+  if (m == 0) return KV_OK;
+  if (!d_digests || !aligned16(d_digests) || (d_ids && !aligned16(d_ids))) return KV_ERR_INVALID_ARG;
+  if (!d_ids && m > p->stats.n_entries) return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_hash_entries(p->geom, p->n_parts, d_ids, m, d_digests, p->ws, S(stream)));
+  return KV_OK;
+}
+
+uint64_t kv_dedup_table_slots(uint64_t m) {
+  uint64_t s = 16;
+  while (s < 2 * m) s <<= 1;
+  return s;
+}
+
+int32_t kv_dedup_digests(const uint8_t* d_digests, uint64_t m, uint32_t* d_canon, uint32_t* d_refcount,
+                         uint32_t* d_table, uint64_t table_slots, uint32_t* d_n_unique, uint32_t* d_status,
+                         kv_stream_t stream) {
+  if (m >= 0xFFFFFFFFull) return KV_ERR_INVALID_ARG;
+  if (!d_table || !aligned16(d_table) || table_slots < kv_dedup_table_slots(m) ||
+      (table_slots & (table_slots - 1)) != 0 || !d_status)
+    return KV_ERR_INVALID_ARG;
+  if (m > 0 && (!d_digests || !aligned16(d_digests) || !d_canon || !d_refcount)) return KV_ERR_INVALID_ARG;
+  const cudaError_t e = launch_dedup(d_digests, m, d_canon, d_refcount, d_table, table_slots, d_n_unique,
+                                     d_status, S(stream));
+  return e == cudaSuccess ? KV_OK : KV_ERR_CUDA;
+}
+
 int32_t kv_set_lazy_decay(kv_pool* p, int32_t on) {
   if (!p) return KV_ERR_INVALID_ARG;
   for (int q = 0; q < p->n_parts; ++q) p->geom[q].lazy_decay = on ? 1u : 0u;

@@ -191,6 +191,15 @@ cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uin
 cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const uint64_t* bases5,
                                     int n_parts, const Workspace& ws, cudaStream_t s);
 
+// ---- kv_dedup.cu ----
+// SHA-256 of the images of entries ids[0..m) (ids == nullptr: entries 0..m-1), 32 bytes each
+cudaError_t launch_hash_entries(const PartGeom* parts, int n_parts, const uint32_t* ids, uint64_t m,
+                                uint8_t* digests, const Workspace& ws, cudaStream_t s);
+// first position per digest and reference counts; table_slots is a power of two >= 2*m
+cudaError_t launch_dedup(const uint8_t* digests, uint64_t m, uint32_t* canon, uint32_t* refcount,
+                         uint32_t* table, uint64_t table_slots, uint32_t* n_unique, uint32_t* status,
+                         cudaStream_t s);
+
 // ---- kv_move.cu ----
 cudaError_t launch_init(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P, float p0,
                         uint32_t* loc, uint64_t n_tags, const PartGeom* parts, int n_parts,
