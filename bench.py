@@ -64,6 +64,9 @@ def parse():
                     help="score and select with two calls (kv_epoch_score, kv_select_victims) instead of the fused one")
     ap.add_argument("--head-weights", action="store_true",
                     help="update every partition's head-importance matrix each step and weight the scores with it")
+    ap.add_argument("--dedup", action="store_true",
+                    help="after the timed steps, also time content hashing (SHA-256 of every entry) and "
+                         "deduplication of the digests; reported under phases, not part of a step")
     ap.add_argument("--tiny-entries", action="store_true",
                     help="32-64 byte blocks (same entry count and traces): for profiling scoring/selection")
     ap.add_argument("--select-variant", type=int, default=1, choices=[0, 1],
@@ -177,6 +180,44 @@ def hostlink_probe(torch, dev, nbytes=1 << 30, reps=10):
     out["how"] = "1 GiB pinned<->device copies, best of %d, CUDA events" % reps
     del h, d, h2, d2
     return out
+
+
+# Instruction slots of one SHA-256 compression (64 bytes) as the kernel issues it: 64 rounds of
+# 6 funnel shifts + 4 three-input logic ops + 4 three-input adds, 48 schedule steps of 6 shifts +
+# 2 logic ops + 2 adds, 16 byte swaps; a funnel shift issues at half the rate of the others, so it
+# takes two slots.  An SM issues 128 lanes per clock (4 schedulers x 32).
+SHA_SLOTS_PER_64B = 64 * (2 * 6 + 4 + 4) + 48 * (2 * 6 + 2 + 2) + 16
+
+
+def time_dedup(torch, pool, w, B, reps=3):
+    """Times kv_hash_entries over every entry and kv_dedup_digests over the digests."""
+    N = w.N
+    dev = pool.device
+    d = torch.zeros((N, 32), dtype=torch.uint8, device=dev)
+    table = torch.empty(B.kv_dedup_table_slots(N), dtype=torch.int32, device=dev)
+    canon = torch.empty(N, dtype=torch.int32, device=dev)
+    ref = torch.empty(N, dtype=torch.int32, device=dev)
+    extra = torch.zeros(8, dtype=torch.int32, device=dev)
+    t_hash, t_dedup = [], []
+    for _ in range(reps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record(pool.compute)
+        rc = pool.kv_hash_entries(None, N, d)
+        ev[1].record(pool.compute)
+        rc2 = B.kv_dedup_digests(d, N, canon, ref, table, extra[0:], extra[4:], pool.compute)
+        ev[2].record(pool.compute)
+        torch.cuda.synchronize(dev)
+        if rc != B.KV_OK or rc2 != B.KV_OK:
+            raise B.KVError(rc or rc2, "kv_hash_entries / kv_dedup_digests")
+        t_hash.append(ev[0].elapsed_time(ev[1]))
+        t_dedup.append(ev[1].elapsed_time(ev[2]))
+    nbytes = sum(p.slab_bytes for p in w.parts)
+    gbs = nbytes / min(t_hash) / 1e6
+    sm_clock_ghz = 1.965     # clocks.max.sm; the kernel draws far less than the power cap
+    alu_peak_gbs = 148 * 128 * sm_clock_ghz * 64 / SHA_SLOTS_PER_64B
+    return {"hash_ms": min(t_hash), "hash_gbs": gbs, "hash_alu_peak_gbs": alu_peak_gbs,
+            "hash_frac_of_alu_peak": gbs / alu_peak_gbs, "dedup_ms": min(t_dedup),
+            "dedup_unique": int(extra[0].item()), "dedup_status": int(extra[4].item())}
 
 
 def oracle_pool(w):
@@ -420,6 +461,10 @@ def main():
                "h2d_bytes_per_step": h2d_b // e2e_steps, "d2h_bytes_per_step": d2h_b // e2e_steps,
                "steps": e2e_steps, "ms_per_step": 1e3 * float(tw.item()) / e2e_steps}
 
+    dedup = None
+    if args.dedup and rank == 0:
+        dedup = time_dedup(torch, pool, w, B)
+
     if rank != 0:
         if dist_on:
             dist.destroy_process_group()
@@ -473,6 +518,8 @@ def main():
     if link:
         line["phases"]["demote_frac_of_d2h_link"] = line["phases"]["demote_gbs"] / link["d2h_gbs"]
         line["phases"]["promote_frac_of_h2d_link"] = line["phases"]["promote_gbs"] / link["h2d_gbs"]
+    if dedup:
+        line["phases"].update(dedup)
     if e2e:
         line["e2e"] = e2e
     if not args.no_cpu_baseline:
