@@ -64,6 +64,8 @@ def parse():
                     help="score and select with two calls (kv_epoch_score, kv_select_victims) instead of the fused one")
     ap.add_argument("--head-weights", action="store_true",
                     help="update every partition's head-importance matrix each step and weight the scores with it")
+    ap.add_argument("--no-breakdown", action="store_true",
+                    help="skip the three extra epochs that time event reduction, entry pass and selection one by one")
     ap.add_argument("--dedup", action="store_true",
                     help="after the timed steps, also time content hashing (SHA-256 of every entry) and "
                          "deduplication of the digests; reported under phases, not part of a step")
@@ -461,6 +463,41 @@ def main():
                "h2d_bytes_per_step": h2d_b // e2e_steps, "d2h_bytes_per_step": d2h_b // e2e_steps,
                "steps": e2e_steps, "ms_per_step": 1e3 * float(tw.item()) / e2e_steps}
 
+    # ---- per-call breakdown of scoring + selection (extra epochs after the timed ones) -----
+    breakdown = None
+    if not args.no_breakdown and not dist_on:
+        acc = {"event_reduce": [], "entry_pass": [], "select": []}
+        for it in range(3):
+            ev_entry, ev_hit = gen_events(epoch)
+            d_e, d_h, n = runner.stage_events(ev_entry, ev_hit)
+            torch.cuda.synchronize(dev)
+            evb = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            flush_l2(epoch)
+            evb[0].record(pool.compute)
+            runner.check(pool.kv_epoch_events(d_e, d_h, n), "kv_epoch_events")
+            evb[1].record(pool.compute)
+            runner.check(pool.kv_epoch_update(epoch), "kv_epoch_update")
+            evb[2].record(pool.compute)
+            runner.check(pool.kv_select_victims(k, runner.victims), "kv_select_victims")
+            evb[3].record(pool.compute)
+            runner.check(pool.kv_demote(runner.victims, k, runner.batch_bytes), "kv_demote")
+            for q, lst in enumerate(runner.promote_lists(epoch)):
+                runner.check(pool.kv_promote(q, lst, runner.batch_bytes), "kv_promote")
+            runner.check(pool.kv_flush(), "kv_flush")
+            torch.cuda.synchronize(dev)
+            for name, i in (("event_reduce", 0), ("entry_pass", 1), ("select", 2)):
+                acc[name].append(evb[i].elapsed_time(evb[i + 1]))
+            between_steps(epoch)
+            epoch += 1
+        med = {kk: float(np.median(v)) for kk, v in acc.items()}
+        peak_b, kind_b = measured_peaks()
+        entry_gbs = 30 * N / (med["entry_pass"] * 1e-3) / 1e9
+        breakdown = {"how": "median of 3 extra epochs with the three calls timed one by one (CUDA events, L2 flushed)",
+                     "event_reduce_us": 1e3 * med["event_reduce"], "entry_pass_us": 1e3 * med["entry_pass"],
+                     "select_us": 1e3 * med["select"],
+                     "entry_pass_gbs": entry_gbs, "entry_pass_algorithmic_bytes_per_entry": 30,
+                     "entry_pass_frac_of_%s_hbm" % kind_b: entry_gbs / peak_b}
+
     dedup = None
     if args.dedup and rank == 0:
         dedup = time_dedup(torch, pool, w, B)
@@ -520,6 +557,8 @@ def main():
         line["phases"]["promote_frac_of_h2d_link"] = line["phases"]["promote_gbs"] / link["h2d_gbs"]
     if dedup:
         line["phases"].update(dedup)
+    if breakdown:
+        line["phases"]["score_select_breakdown"] = breakdown
     if e2e:
         line["e2e"] = e2e
     if not args.no_cpu_baseline:
