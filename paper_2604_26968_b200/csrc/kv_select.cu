@@ -434,6 +434,7 @@ constexpr uint64_t kStaticMaxTiles = kStaticMaxEntries / kvt::kTileEntries + 2;
 constexpr uint64_t kOffHist = 0;
 constexpr uint64_t kOffSel = 3 * kvt::kHistBins * 4;
 constexpr uint64_t kOffStatus = kOffSel + 256;
+static_assert(sizeof(kvt::SelectScalars) <= 256, "the scalars have 256 bytes of the built-in scratch");
 constexpr uint64_t kOffTileCounts = kOffStatus + 256;
 constexpr uint64_t kOffTileOffsets = kOffTileCounts + ((kStaticMaxTiles * 8 + 255) / 256) * 256;
 constexpr uint64_t kStaticScratchBytes = kOffTileOffsets + ((kStaticMaxTiles * 8 + 255) / 256) * 256;

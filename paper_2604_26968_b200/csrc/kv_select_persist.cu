@@ -32,6 +32,8 @@ constexpr uint32_t kPKeyCap = 49152;                    // keys kept in shared m
 constexpr uint32_t kPHistBins = 2048;
 constexpr uint32_t kExcluded = 0xFFFFFFFFu;             // key of a non-candidate (FREE) entry
 constexpr uint32_t kBarrierSpins = 1u << 22;
+constexpr uint32_t kBracketShift = 11;                  // a bracket bin is 2^11 keys wide ...
+constexpr uint32_t kBracketHalf = 1u << 21;             // ... and the 2,048 bins reach 2^21 keys to either side of the hint
 
 static_assert(kPKeyCap % kPChunk == 0, "the cached part of a slice is a whole number of chunks");
 static_assert(kPKeyCap < 65536, "per-CTA counts of the cached part are packed in 16 bits");
@@ -232,7 +234,25 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     }
   }
 
-  // ---- phase A: keys into shared memory, then the histogram of digit 0 (bits 31..21) ----
+  // ---- phase A: keys into shared memory, and the first histogram ----
+  // Without a hint the first histogram is digit 0 of a plain radix select (bits
+  // 31..21 of every key).  With a hint -- tau of the previous selection over the
+  // same number of keys -- it covers only the bracket [lo, lo + 2^22) around that
+  // tau in 2,048 bins of 2^11 keys, and keys below lo are merely counted: scores
+  // move little from one epoch to the next, so the k-th key is almost always
+  // inside, few keys need an atomic, and one later pass (2^11 keys wide) finishes
+  // the selection instead of two.  If rank k falls outside the bracket the plain
+  // radix select runs after all, from the cached keys.
+  const bool hint = a.sel->hint_valid != 0 && a.sel->hint_n == a.n;
+  const uint32_t hint_tau = a.sel->hint_tau;
+  const uint32_t base0 = hint ? (hint_tau > kBracketHalf ? hint_tau - kBracketHalf : 0u) : 0u;
+  const uint32_t shift0 = hint ? kBracketShift : 21u;
+  uint32_t n_below0 = 0;  // keys of this thread below the bracket
+  auto first_pass = [&](uint32_t key) {
+    n_below0 += (key < base0);  // (an excluded key is 0xFFFFFFFF: never below)
+    const bool cand = key != kExcluded && key >= base0 && ((key - base0) >> shift0) < kPHistBins;
+    p_warp_hist_add(s_hist, cand, (key - base0) >> shift0);
+  };
   clear_hist();
   if constexpr (FUSED) {
     // the slice's entries go through the EMA and score update on the way; keys of
@@ -271,15 +291,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         reinterpret_cast<uint4*>(s_keys)[c * kPThreads + t] = make_uint4(key[0], key[1], key[2], key[3]);
       } else {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) p_warp_hist_add(s_hist, key[j] != kExcluded, key[j] >> 21);
+        for (int j = 0; j < 4; ++j) first_pass(key[j]);
       }
     }
     __syncthreads();
     const uint32_t iters = (cached + kPThreads - 1) / kPThreads;
     for (uint32_t i = 0; i < iters; ++i) {
       const uint32_t j = i * kPThreads + t;
-      const uint32_t key = j < cached ? s_keys[j] : kExcluded;
-      p_warp_hist_add(s_hist, key != kExcluded, key >> 21);
+      first_pass(j < cached ? s_keys[j] : kExcluded);
     }
   } else {
     const uint32_t cached_chunks = (cached + kPChunk - 1) / kPChunk;
@@ -290,9 +309,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       reinterpret_cast<uint4*>(s_keys)[c * kPThreads + t] = make_uint4(key[0], key[1], key[2], key[3]);
     }
     __syncthreads();
-    for_each_key([&](uint32_t key) { p_warp_hist_add(s_hist, key != kExcluded, key >> 21); });
+    for_each_key(first_pass);
   }
-  flush_hist(a.hist, 2048);
+  flush_hist(a.hist, kPHistBins);
+  if (hint) {
+    uint32_t tot;
+    (void)block_scan_excl(n_below0, s_warp, tot);
+    if (t == 0 && tot) atomicAdd(&a.sel->below, (unsigned long long)tot);
+  }
   stamp(1);
   ok = grid_barrier(bar, G);
   stamp(2);
@@ -303,45 +327,71 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   }
 
   {
-    // ---- phase B: fix digit 0, histogram of digit 1 (bits 20..10) ----
-    uint32_t bin, before;
+    // ---- phases B, C: narrow [base, base + 2^shift) around rank k, one histogram per step ----
+    // The current histogram is a.hist[h]; it was built over [base, base + 2048 << shift).
+    // Every CTA reads the same global data, so all of them take the same path.
+    uint32_t h = 0, nbar = 1, base = base0, shift = shift0;
     unsigned long long k_rem = a.k;
-    pick_bin(a.hist, 2048, k_rem, s_warp, s_pick, bin, before);
-    const bool found0 = bin != 0xFFFFFFFFu;
-    uint32_t prefix = bin << 21;
-    k_rem -= before;
-    clear_hist();
-    for_each_key([&](uint32_t key) {
-      p_warp_hist_add(s_hist, key != kExcluded && (key & 0xFFE00000u) == prefix, (key >> 10) & 2047u);
-    });
-    flush_hist(a.hist + kPHistBins, 2048);
-    ok = grid_barrier(bar, 2 * G);
-    stamp(3);
-    if (!ok) goto fail;
-    if (blockIdx.x == 0)
-      for (uint32_t b = t; b < 2048; b += kPThreads) a.hist[b] = 0;  // nobody reads digit 0 any more
+    uint32_t bin, before;
+    bool found = true;
+    bool clear_below = hint;
+    auto hist_pass = [&](uint32_t width_log2, uint32_t new_shift, uint32_t h_new) {
+      // histogram of ((key - base) >> new_shift) over the keys in [base, base + 2^width_log2)
+      clear_hist();
+      const uint32_t top = width_log2 - new_shift;  // log2 of the number of bins
+      for_each_key([&](uint32_t key) {
+        const uint32_t d = key - base;
+        p_warp_hist_add(s_hist, key != kExcluded && key >= base && ((d >> new_shift) >> top) == 0u, d >> new_shift);
+      });
+      flush_hist(a.hist + h_new * kPHistBins, 1u << top);
+    };
+    auto retire = [&](uint32_t h_old) {   // after a barrier: nobody reads histogram h_old any more
+      if (blockIdx.x == 0) {
+        for (uint32_t b = t; b < kPHistBins; b += kPThreads) a.hist[h_old * kPHistBins + b] = 0;
+        if (clear_below && t == 0) a.sel->below = 0;
+      }
+      clear_below = false;
+    };
+    if (hint) {
+      const unsigned long long below = __ldcg(&a.sel->below);
+      const bool above = a.k > below;
+      pick_bin(a.hist, kPHistBins, above ? a.k - below : 1ull, s_warp, s_pick, bin, before);
+      if (above && bin != 0xFFFFFFFFu) {
+        k_rem = a.k - below;
+      } else {
+        // rank k is outside the bracket: digit 0 of the plain radix select, from the cached keys
+        base = 0;
+        shift = 21;
+        hist_pass(32, 21, 1);
+        ok = grid_barrier(bar, ++nbar * G);
+        if (!ok) goto fail;
+        retire(0);
+        h = 1;
+        pick_bin(a.hist + kPHistBins, kPHistBins, k_rem, s_warp, s_pick, bin, before);
+      }
+    } else {
+      pick_bin(a.hist, kPHistBins, k_rem, s_warp, s_pick, bin, before);
+    }
+    for (int step = 0;; ++step) {
+      found = found && bin != 0xFFFFFFFFu;
+      k_rem -= before;
+      base += (bin & (kPHistBins - 1u)) << shift;   // rank k lies in [base, base + 2^shift)
+      if (shift == 0) break;
+      const uint32_t new_shift = shift > 11u ? shift - 11u : 0u;
+      const uint32_t h_new = (h + 1u) % 3u;
+      hist_pass(shift, new_shift, h_new);
+      ok = grid_barrier(bar, ++nbar * G);
+      if (step < 2) stamp(3 + step);
+      if (!ok) goto fail;
+      retire(h);
+      pick_bin(a.hist + h_new * kPHistBins, 1u << (shift - new_shift), k_rem, s_warp, s_pick, bin, before);
+      h = h_new;
+      shift = new_shift;
+    }
 
-    // ---- phase C: fix digit 1, histogram of digit 2 (bits 9..0) ----
-    pick_bin(a.hist + kPHistBins, 2048, k_rem, s_warp, s_pick, bin, before);
-    const bool found1 = bin != 0xFFFFFFFFu;
-    prefix |= (bin & 2047u) << 10;
-    k_rem -= before;
-    clear_hist();
-    for_each_key([&](uint32_t key) {
-      p_warp_hist_add(s_hist, key != kExcluded && (key & 0xFFFFFC00u) == prefix, key & 1023u);
-    });
-    flush_hist(a.hist + 2 * kPHistBins, 1024);
-    ok = grid_barrier(bar, 3 * G);
-    stamp(4);
-    if (!ok) goto fail;
-    if (blockIdx.x == 0)
-      for (uint32_t b = t; b < 2048; b += kPThreads) a.hist[kPHistBins + b] = 0;
-
-    // ---- phase D: fix digit 2 -> tau; count (key < tau, key == tau) in the slice ----
-    pick_bin(a.hist + 2 * kPHistBins, 1024, k_rem, s_warp, s_pick, bin, before);
-    const bool found = found0 && found1 && bin != 0xFFFFFFFFu;
-    const uint32_t tau = prefix | (bin & 1023u);
-    const unsigned long long need_eq = k_rem - before;
+    // ---- phase D: tau is known; count (key < tau, key == tau) in the slice ----
+    const uint32_t tau = base;
+    const unsigned long long need_eq = k_rem;
     {
       uint32_t n_less = 0, n_eq = 0;
       for_each_key([&](uint32_t key) {
@@ -354,11 +404,10 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(tot_less, tot_eq);
     }
     stamp(5);
-    ok = grid_barrier(bar, 4 * G);
+    ok = grid_barrier(bar, ++nbar * G);
     stamp(6);
     if (!ok) goto fail;
-    if (blockIdx.x == 0)
-      for (uint32_t b = t; b < 2048; b += kPThreads) a.hist[2 * kPHistBins + b] = 0;
+    retire(h);
 
     // ---- phase E: ordered write ----
     unsigned long long less_before, eq_before;
@@ -433,6 +482,10 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       if (!found || got != a.k) atomicOr(a.status, KV_DEV_SELECT_MISMATCH);
       a.sel->tau = tau;
       a.sel->need_eq = need_eq;
+      // hint for the next selection over the same keys
+      a.sel->hint_tau = tau;
+      a.sel->hint_n = a.n;
+      a.sel->hint_valid = (found && got == a.k) ? 1u : 0u;
     }
   }
   stamp(7);
