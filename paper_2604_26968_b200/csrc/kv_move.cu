@@ -299,7 +299,7 @@ __global__ void init_scalars_kernel(uint64_t* hits, uint64_t* misses, float* P, 
   if (t == 0) {
     *ws.status = 0;
     ws.sel->prefix = 0; ws.sel->tau = 0; ws.sel->k_rem = 0; ws.sel->need_eq = 0;
-    ws.sel->bar_arrive = 0; ws.sel->bar_done = 0; ws.sel->update_ticket = 0; ws.sel->pad = 0;
+    ws.sel->bar_arrive = 0; ws.sel->bar_done = 0; ws.sel->update_ticket = 0; ws.sel->hint_last = 0;
     ws.sel->hint_valid = 0; ws.sel->hint_tau = 0; ws.sel->hint_n = 0; ws.sel->below = 0;
   }
 }

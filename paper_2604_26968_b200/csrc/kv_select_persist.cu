@@ -483,8 +483,16 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       if (!found || got != a.k) atomicOr(a.status, KV_DEV_SELECT_MISMATCH);
       a.sel->tau = tau;
       a.sel->need_eq = need_eq;
-      // hint for the next selection over the same keys
-      a.sel->hint_tau = tau;
+      // hint for the next selection over the same keys: this tau moved on by as much as it
+      // moved since the selection before (while a pool warms up its scores grow epoch after
+      // epoch, and the trend is a better centre for the bracket than the last value)
+      const bool had = a.sel->hint_valid != 0 && a.sel->hint_n == a.n;
+      const long long step = had ? (long long)tau - (long long)a.sel->hint_last : 0ll;
+      long long guess = (long long)tau + step;
+      if (guess < 0) guess = 0;
+      if (guess > 0xFFFFFFFEll) guess = 0xFFFFFFFEll;
+      a.sel->hint_last = tau;
+      a.sel->hint_tau = (uint32_t)guess;
       a.sel->hint_n = a.n;
       a.sel->hint_valid = (found && got == a.k) ? 1u : 0u;
     }

@@ -79,8 +79,8 @@ struct SelectScalars {
   unsigned int bar_done;       // ... and CTAs that have left (the last one resets both)
   unsigned int update_ticket;  // blocks of the entry pass that have finished (the last one commits)
   unsigned int hint_valid;     // the persistent selection left a usable hint
-  uint32_t hint_tau;           // tau of the last persistent selection ...
-  uint32_t pad;
+  uint32_t hint_tau;           // where the next persistent selection centres its bracket ...
+  uint32_t hint_last;          // (tau of the last one)
   unsigned long long hint_n;   // ... and the number of keys it ran over
   unsigned long long below;    // keys below the bracket (accumulated per launch, cleared inside it)
   unsigned long long phase_ns[8];  // %globaltimer at the phase boundaries of the last persistent selection (CTA 0)
