@@ -155,6 +155,7 @@ template <bool FUSED>
 __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const PArgs a) {
   extern __shared__ __align__(16) uint32_t s_keys[];  // a.cap keys
   __shared__ uint32_t s_hist[kPHistBins];
+  __shared__ uint32_t s_hist_first[kPHistBins];  // the CTA's own first (bracket) histogram
   __shared__ uint32_t s_warp[32];
   __shared__ uint32_t s_pick[2];
   __shared__ float sP[16];
@@ -313,10 +314,10 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     for_each_key(first_pass);
   }
   flush_hist(a.hist, kPHistBins);
+  uint32_t cta_below0 = 0;  // keys of this CTA's slice below the bracket
   if (hint) {
-    uint32_t tot;
-    (void)block_scan_excl(n_below0, s_warp, tot);
-    if (t == 0 && tot) atomicAdd(&a.sel->below, (unsigned long long)tot);
+    (void)block_scan_excl(n_below0, s_warp, cta_below0);
+    if (t == 0 && cta_below0) atomicAdd(&a.sel->below, (unsigned long long)cta_below0);
   }
   stamp(1);
   ok = grid_barrier(bar, G);
@@ -336,6 +337,8 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     uint32_t bin, before;
     bool found = true;
     bool clear_below = hint;
+    bool bracket_hit = false;   // rank k was inside the bracket: two histograms in all
+    uint32_t bin_first = 0;     // ... and this was its bin of the first one
     auto hist_pass = [&](uint32_t width_log2, uint32_t new_shift, uint32_t h_new) {
       // histogram of ((key - base) >> new_shift) over the keys in [base, base + 2^width_log2)
       clear_hist();
@@ -359,6 +362,12 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       pick_bin(a.hist, kPHistBins, above ? a.k - below : 1ull, s_warp, s_pick, bin, before);
       if (above && bin != 0xFFFFFFFFu) {
         k_rem = a.k - below;
+        // The CTA's own first histogram is still in s_hist: keep it.  Together with its own
+        // second histogram it gives this slice's counts below and at tau without another
+        // pass over the keys.
+        bracket_hit = true;
+        bin_first = bin;
+        for (uint32_t b = t; b < kPHistBins; b += kPThreads) s_hist_first[b] = s_hist[b];
       } else {
         // rank k is outside the bracket: digit 0 of the plain radix select, from the cached keys
         base = 0;
@@ -393,7 +402,17 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     // ---- phase D: tau is known; count (key < tau, key == tau) in the slice ----
     const uint32_t tau = base;
     const unsigned long long need_eq = k_rem;
-    {
+    if (bracket_hit) {
+      // below tau = below the bracket + bins of the first histogram before rank k's bin +
+      // bins of the second (single keys, still in s_hist) before tau; at tau = tau's bin
+      const uint32_t bin_tau = tau - (base0 + (bin_first << kBracketShift));
+      uint32_t v = 0;
+      for (uint32_t b = t; b < kPHistBins; b += kPThreads)
+        v += (b < bin_first ? s_hist_first[b] : 0u) + (b < bin_tau ? s_hist[b] : 0u);
+      uint32_t tot_less;
+      (void)block_scan_excl(v, s_warp, tot_less);
+      if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(cta_below0 + tot_less, s_hist[bin_tau]);
+    } else {
       uint32_t n_less = 0, n_eq = 0;
       for_each_key([&](uint32_t key) {
         n_less += (key != kExcluded && key < tau);
