@@ -442,18 +442,30 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       (void)block_scan_excl(ea, s_warp, te);
       less_before = tl; eq_before = te;
     }
-    auto emit = [&](uint32_t key, unsigned long long id, unsigned long long& n1, unsigned long long& n2) {
-      if (key == kExcluded) return;
+    // Position of a victim.  With L entries below tau and E entries equal to tau before it
+    // in id order, an entry below tau goes to L + min(E, need_eq) and an entry equal to tau,
+    // taken while E < need_eq, to L + E.  Everything before the current piece of the slice is
+    // folded into pos0 and room once per piece, so the per-key arithmetic is 32-bit: ml and me
+    // count inside the piece.
+    unsigned long long pos0 = 0;
+    uint32_t room = 0;
+    auto set_piece = [&]() {
+      pos0 = less_before + (eq_before < need_eq ? eq_before : need_eq);
+      const unsigned long long left = need_eq > eq_before ? need_eq - eq_before : 0ull;
+      room = left > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)left;
+    };
+    auto emit = [&](uint32_t key, unsigned long long id, uint32_t& ml, uint32_t& me) {
+      if (key > tau) return;   // most keys (an excluded key is 0xFFFFFFFF)
       if (key < tau) {
-        const unsigned long long pos = n1 + (n2 < need_eq ? n2 : need_eq);
+        const unsigned long long pos = pos0 + ml + (me < room ? me : room);
         if (pos < a.k) a.victims[pos] = (uint32_t)id;
-        ++n1;
-      } else if (key == tau) {
-        if (n2 < need_eq) {
-          const unsigned long long pos = n1 + n2;
+        ++ml;
+      } else if (key != kExcluded) {
+        if (me < room) {
+          const unsigned long long pos = pos0 + ml + me;
           if (pos < a.k) a.victims[pos] = (uint32_t)id;
         }
-        ++n2;
+        ++me;
       }
     };
     if (found) {
@@ -467,12 +479,13 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         uint32_t v = 0;
         for (uint32_t j = j0; j < j1; ++j) {
           const uint32_t key = s_keys[j];
-          v += (key != kExcluded && key < tau) + ((uint32_t)(key != kExcluded && key == tau) << 16);
+          v += (key < tau) + ((uint32_t)(key == tau && key != kExcluded) << 16);
         }
         uint32_t total;
         const uint32_t excl = block_scan_excl(v, s_warp, total);
-        unsigned long long n1 = less_before + (excl & 0xFFFFu), n2 = eq_before + (excl >> 16);
-        for (uint32_t j = j0; j < j1; ++j) emit(s_keys[j], s0 + j, n1, n2);
+        set_piece();
+        uint32_t ml = excl & 0xFFFFu, me = excl >> 16;
+        for (uint32_t j = j0; j < j1; ++j) emit(s_keys[j], s0 + j, ml, me);
         less_before += total & 0xFFFFu;
         eq_before += total >> 16;
       }
@@ -483,13 +496,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         uint32_t v = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-          v += (key[j] != kExcluded && key[j] < tau) + ((uint32_t)(key[j] != kExcluded && key[j] == tau) << 16);
+          v += (key[j] < tau) + ((uint32_t)(key[j] == tau && key[j] != kExcluded) << 16);
         uint32_t total;
         const uint32_t excl = block_scan_excl(v, s_warp, total);
-        unsigned long long n1 = less_before + (excl & 0xFFFFu), n2 = eq_before + (excl >> 16);
+        set_piece();
+        uint32_t ml = excl & 0xFFFFu, me = excl >> 16;
         const unsigned long long i0 = s0 + (unsigned long long)c * kPChunk + 4ull * t;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) emit(key[j], i0 + j, n1, n2);
+        for (int j = 0; j < 4; ++j) emit(key[j], i0 + j, ml, me);
         less_before += total & 0xFFFFu;
         eq_before += total >> 16;
       }
