@@ -555,6 +555,9 @@ def main():
     if link:
         line["phases"]["demote_frac_of_d2h_link"] = line["phases"]["demote_gbs"] / link["d2h_gbs"]
         line["phases"]["promote_frac_of_h2d_link"] = line["phases"]["promote_gbs"] / link["h2d_gbs"]
+        # the promotion's copies run while the demotion's do: the link's rate per direction with both busy
+        line["phases"]["promote_frac_of_link_with_both_directions_busy"] = \
+            line["phases"]["promote_gbs"] / link["bidir_gbs_per_dir"]
     if dedup:
         line["phases"].update(dedup)
     if breakdown:

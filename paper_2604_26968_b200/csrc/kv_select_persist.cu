@@ -19,9 +19,9 @@
 // true): every CTA first updates the entries of its own slice (posterior, EMA,
 // score) and turns the fresh scores straight into keys -- the score array is
 // written for the caller but never read back, and a kernel boundary disappears.
-// The event reduction stays a launch of its own ahead of it: it is bound by the
-// latency of scattered accesses and wants twice the threads per SM that this
-// kernel's shared-memory footprint allows (measured: 2.5x slower inside it).
+// The event reduction stays a launch of its own ahead of it: its scattered gathers
+// and atomics ran 2.5x slower inside this kernel when that was tried, and a grid
+// barrier costs about what the launch boundary does.
 #include "kv_score_device.cuh"
 
 namespace kvt {
