@@ -34,10 +34,10 @@ UNIT = "head-blocks/s"
 
 # DRAM traffic from ncu (dram__bytes_read.sum + dram__bytes_write.sum) per payload
 # byte of a launch, keyed by move variant: captured on a 256 MiB payload-only
-# launch of a 3 GiB pool (488.15 MB of traffic for 268.44 MB of payload) and
+# launch of a 3 GiB pool (487.35 MB of traffic for 268.44 MB of payload) and
 # scaled to the benchmark's launch size in proportion to the payload.  None = no
 # capture of that kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE = {1: 488.15 / 268.44, 0: None}
+NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE = {1: 487.35 / 268.44, 0: None}
 PACK_KERNEL_NAME = {1: "move_tma_kernel<true> (pack)", 0: "pack_kernel"}
 
 
