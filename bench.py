@@ -310,6 +310,10 @@ def main():
     dev = torch.device("cuda", local)
     dist_on = world > 1 or args.sharded    # --sharded: take the multi-GPU code path even on one rank
     if dist_on:
+        if "RANK" not in os.environ:      # --sharded started without a launcher: a group of one
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29533")
+            os.environ["RANK"], os.environ["WORLD_SIZE"] = "0", "1"
         dist.init_process_group("nccl", device_id=dev)
 
     w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries)
