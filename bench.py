@@ -50,7 +50,9 @@ def parse():
     ap.add_argument("--config", type=int, default=2, help="pool 1..5")
     ap.add_argument("--scale", type=float, default=1.0, help="shrinks blocks per layer")
     ap.add_argument("--ring-slots", type=int, default=None)
-    ap.add_argument("--batch-mb", type=int, default=1024, help="demote/promote chunk (staging buffer) size")
+    ap.add_argument("--batch-mb", type=int, default=1320,
+                    help="demote/promote chunk (staging buffer) size; the default lets the default pool's demotion "
+                         "(2.58 GB) take two chunks, so that both pack launches run back to back")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-hostlink", action="store_true", help="skip the 1 GiB host-link probe")
