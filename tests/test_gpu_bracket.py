@@ -96,11 +96,14 @@ def test_threshold_on_and_beside_the_bracket_edges(offset):
     s.close()
 
 
-def test_entry_and_block_selections_share_the_scratch():
-    """A block-granular selection between two entry selections runs over another number of
-    keys: the hint of one must not be used for the other."""
+@pytest.mark.parametrize("kind", ["gqa", "mla"])
+def test_entry_and_block_selections_share_the_scratch(kind):
+    """A block-granular selection between two entry selections runs over other keys (and, except
+    for MLA, whose blocks have one entry each, over another number of them): a hint left by one
+    kind of selection must not spoil the other."""
     from lockstep import Lockstep
-    w = W.Workload("mix", [W.gqa(2, 8, 4, 16, 8, 3000, 4000, "entry")], 0.05, 0.02, seed=13, promote_style="recent")
+    part = W.gqa(2, 8, 4, 16, 8, 3000, 4000, "entry") if kind == "gqa" else W.mla(3, 64, 16, 8, 5000, 4000, "entry")
+    w = W.Workload("mix", [part], 0.05, 0.02, seed=13, promote_style="recent")
     ls = Lockstep(w, payload=False, batch_bytes=1 << 20, fused=True)
     for e in range(3):
         ls.epoch(e)
