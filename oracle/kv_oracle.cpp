@@ -16,10 +16,16 @@
 //   * the EMA recurrence, the product score, the per-(layer, head) importance
 //     weighting (recurrence, group maximum, multipliers: okv_head_importance_update),
 //     the ring organisation of the host
-//     tier and the free-slot rule of promotion are NOT printed in the paper
-//     (it withholds them): they are this build's readings, so their agreement
-//     with the paper is "parity unpinned"; their internal consistency (closed
-//     forms, brute force, conservation) is what the tests pin.
+//     tier, the free-slot rule of promotion and the lazy decay of promoted
+//     entries (okv_set_lazy_decay) are NOT printed in the paper (it withholds
+//     them): they are this build's readings, so their agreement with the paper
+//     is "parity unpinned"; their internal consistency (closed forms, brute
+//     force, conservation, equality with a resident twin) is what the tests pin.
+//   * content hashing (okv_entry_image + SHA-256 in kv_oracle.py) follows the
+//     content-addressable deduplication section: the hash is FIPS 180-4's and is
+//     pinned to the standard's published digests; what counts as a block's
+//     content (the entry image) and the list-order rule of the reference counts
+//     are readings, pinned by a hand-built slab and a quadratic brute force.
 //
 // Floating point is IEEE binary32 with every operation rounded once
 // (build with -O2 -ffp-contract=off -fno-fast-math; no flush-to-zero).
