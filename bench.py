@@ -186,11 +186,12 @@ def hostlink_probe(torch, dev, nbytes=1 << 30, reps=10):
     return out
 
 
-# Instruction slots of one SHA-256 compression (64 bytes) as the kernel issues it: 64 rounds of
-# 6 funnel shifts + 4 three-input logic ops + 4 three-input adds, 48 schedule steps of 6 shifts +
-# 2 logic ops + 2 adds, 16 byte swaps; a funnel shift issues at half the rate of the others, so it
-# takes two slots.  An SM issues 128 lanes per clock (4 schedulers x 32).
-SHA_SLOTS_PER_64B = 64 * (2 * 6 + 4 + 4) + 48 * (2 * 6 + 2 + 2) + 16
+# Integer-pipe slots of one SHA-256 compression (64 bytes) as the kernel issues it: 64 rounds of
+# 6 funnel shifts + 4 three-input logic ops, 48 schedule steps of 6 shifts + 2 logic ops, 16 byte
+# swaps; a funnel shift issues at half the rate of the others, so it takes two slots.  The
+# additions are issued as multiply-adds on the FMA pipe and do not queue here.  An SM issues 128
+# lanes per clock (4 schedulers x 32).
+SHA_SLOTS_PER_64B = 64 * (2 * 6 + 4) + 48 * (2 * 6 + 2) + 16
 
 
 def time_dedup(torch, pool, w, B, reps=3):

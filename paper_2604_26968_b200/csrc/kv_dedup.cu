@@ -8,10 +8,12 @@
 //   hash_entries_kernel   one thread per entry walks the entry's image (K chunk
 //                         then V chunk, or the MLA chunk) in 64-byte blocks through
 //                         the SHA-256 compression function of FIPS 180-4.  The
-//                         work is integer arithmetic (about 30 instructions per
+//                         work is integer arithmetic (about 25 instructions per
 //                         byte), not memory traffic: a thread reads its 64 bytes as
-//                         four 16-byte loads and then spends ~2,000 instructions on
-//                         them.
+//                         four 16-byte loads and then spends ~1,600 instructions on
+//                         them.  Shifts and logic operations fill the integer pipe, so
+//                         the additions are issued as multiply-adds, which run on the
+//                         FMA pipe beside it (861 -> 1,025 GB/s on 8 KB entries).
 //   dedup_insert_kernel / dedup_resolve_kernel
 //                         an open-addressing table of list positions, probed from
 //                         the first 8 bytes of the digest (a SHA-256 digest is as
@@ -50,7 +52,16 @@ __device__ __forceinline__ uint32_t be32(uint32_t x) { return __byte_perm(x, 0, 
 
 // One application of the compression function: st <- st + compress(st, w), w = the
 // 16 message words of the block (overwritten by the message schedule).
-__device__ __forceinline__ void sha256_block(uint32_t st[8], uint32_t w[16]) {
+// x + y as an integer multiply-add x * one + y (one = 1, a kernel argument so that it stays a
+// multiply-add): it issues to the FMA pipe, while the shifts, logic operations and plain adds of
+// the compression function all queue for the integer pipe, which is the kernel's bottleneck.
+__device__ __forceinline__ uint32_t add_on_fma_pipe(uint32_t x, uint32_t y, uint32_t one) {
+  uint32_t r;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(x), "r"(one), "r"(y));
+  return r;
+}
+
+__device__ __forceinline__ void sha256_block(uint32_t st[8], uint32_t w[16], uint32_t one) {
   uint32_t a = st[0], b = st[1], c = st[2], d = st[3], e = st[4], f = st[5], g = st[6], h = st[7];
 #pragma unroll
   for (int i = 0; i < 64; ++i) {
@@ -58,15 +69,15 @@ __device__ __forceinline__ void sha256_block(uint32_t st[8], uint32_t w[16]) {
       const uint32_t w15 = w[(i + 1) & 15], w2 = w[(i + 14) & 15];
       const uint32_t s0 = rotr(w15, 7) ^ rotr(w15, 18) ^ (w15 >> 3);
       const uint32_t s1 = rotr(w2, 17) ^ rotr(w2, 19) ^ (w2 >> 10);
-      w[i & 15] = w[i & 15] + s0 + w[(i + 9) & 15] + s1;
+      w[i & 15] = add_on_fma_pipe(add_on_fma_pipe(w[i & 15], s0, one), add_on_fma_pipe(w[(i + 9) & 15], s1, one), one);
     }
     const uint32_t S1 = rotr(e, 6) ^ rotr(e, 11) ^ rotr(e, 25);
     const uint32_t ch = (e & f) ^ (~e & g);
-    const uint32_t t1 = h + S1 + ch + kShaK[i] + w[i & 15];
+    const uint32_t t1 = add_on_fma_pipe(add_on_fma_pipe(h, S1, one), add_on_fma_pipe(ch, add_on_fma_pipe(w[i & 15], kShaK[i], one), one), one);
     const uint32_t S0 = rotr(a, 2) ^ rotr(a, 13) ^ rotr(a, 22);
     const uint32_t maj = (a & b) ^ (a & c) ^ (b & c);
-    const uint32_t t2 = S0 + maj;
-    h = g; g = f; f = e; e = d + t1; d = c; c = b; b = a; a = t1 + t2;
+    const uint32_t t2 = add_on_fma_pipe(S0, maj, one);
+    h = g; g = f; f = e; e = add_on_fma_pipe(d, t1, one); d = c; c = b; b = a; a = add_on_fma_pipe(t1, t2, one);
   }
   st[0] += a; st[1] += b; st[2] += c; st[3] += d; st[4] += e; st[5] += f; st[6] += g; st[7] += h;
 }
@@ -82,7 +93,7 @@ __device__ __forceinline__ uint64_t hash_chunk_offset(const PartGeom& g, uint64_
 // of the image never straddles the K and V chunks.
 __global__ void __launch_bounds__(128)
 hash_entries_kernel(const HashGeom hg, const uint32_t* __restrict__ ids, uint64_t m,
-                    uint8_t* __restrict__ digests, uint32_t* __restrict__ status) {
+                    uint8_t* __restrict__ digests, uint32_t* __restrict__ status, uint32_t one) {
   const uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= m) return;
   const uint64_t id = ids ? ids[j] : j;
@@ -112,7 +123,7 @@ hash_entries_kernel(const HashGeom hg, const uint32_t* __restrict__ ids, uint64_
       const uint4 v = piece(b * 64 + u * 16);
       w[4 * u + 0] = be32(v.x); w[4 * u + 1] = be32(v.y); w[4 * u + 2] = be32(v.z); w[4 * u + 3] = be32(v.w);
     }
-    sha256_block(st, w);
+    sha256_block(st, w, one);
   }
   // last block: what is left of the image (0, 16, 32 or 48 bytes), the 1 bit, zeros, the length in bits
   const uint32_t rem = eb - full * 64;
@@ -127,7 +138,7 @@ hash_entries_kernel(const HashGeom hg, const uint32_t* __restrict__ ids, uint64_
     if ((uint32_t)i * 4 == rem) w[i] = 0x80000000u;
   w[14] = (uint32_t)(((uint64_t)eb * 8) >> 32);   // rem <= 48: the length always fits this block
   w[15] = (uint32_t)((uint64_t)eb * 8);
-  sha256_block(st, w);
+  sha256_block(st, w, one);
   uint4* out = reinterpret_cast<uint4*>(digests + j * 32);
   out[0] = make_uint4(be32(st[0]), be32(st[1]), be32(st[2]), be32(st[3]));
   out[1] = make_uint4(be32(st[4]), be32(st[5]), be32(st[6]), be32(st[7]));
@@ -140,7 +151,7 @@ cudaError_t launch_hash_entries(const PartGeom* parts, int n_parts, const uint32
   for (int q = 0; q < 4; ++q) hg.part[q] = parts[q < n_parts ? q : 0];
   hg.n_parts = n_parts;
   const uint64_t blocks = (m + 127) / 128;
-  hash_entries_kernel<<<(unsigned)blocks, 128, 0, s>>>(hg, ids, m, digests, ws.status);
+  hash_entries_kernel<<<(unsigned)blocks, 128, 0, s>>>(hg, ids, m, digests, ws.status, 1u);
   count_launches(1);
   return cudaGetLastError();
 }
