@@ -123,3 +123,25 @@ def test_bad_descriptions_are_refused_without_cuda():
                  lambda: lib.kv_promote(None, 0, None, 1, 1, None, None)):
         assert call() == B.KV_ERR_INVALID_ARG
     assert lib.kv_status_string(B.KV_ERR_K_TOO_LARGE).decode().startswith("k exceeds")
+
+
+def test_dedup_table_size_and_argument_checks_need_no_gpu():
+    """The scratch table of kv_dedup_digests: a power of two, at least twice the list (so that a
+    probe always ends) and at least 16; null and misaligned arguments are refused on the host."""
+    for m, want in [(0, 16), (1, 16), (8, 16), (9, 32), (1000, 2048), (1024, 2048), (1025, 4096),
+                    (3_145_728, 8_388_608)]:
+        s = B.kv_dedup_table_slots(m)
+        assert s == want and s >= 2 * m and s & (s - 1) == 0, (m, s)
+    lib = B.load()
+    fake = C.c_void_p(0x1000)      # aligned, never dereferenced: every call below fails its checks first
+    bad = C.c_void_p(0x1004)
+    args = lambda **kw: [kw.get("dig", fake), kw.get("m", 8), fake, fake, kw.get("table", fake),
+                         kw.get("slots", 16), None, kw.get("status", fake), None]
+    assert lib.kv_dedup_digests(*args(table=None)) == B.KV_ERR_INVALID_ARG
+    assert lib.kv_dedup_digests(*args(table=bad)) == B.KV_ERR_INVALID_ARG
+    assert lib.kv_dedup_digests(*args(slots=8)) == B.KV_ERR_INVALID_ARG        # fewer than 2 * m
+    assert lib.kv_dedup_digests(*args(slots=24)) == B.KV_ERR_INVALID_ARG       # not a power of two
+    assert lib.kv_dedup_digests(*args(status=None)) == B.KV_ERR_INVALID_ARG
+    assert lib.kv_dedup_digests(*args(dig=None)) == B.KV_ERR_INVALID_ARG
+    assert lib.kv_dedup_digests(*args(dig=bad)) == B.KV_ERR_INVALID_ARG
+    assert lib.kv_dedup_digests(*args(m=0xFFFFFFFF, slots=1 << 34)) == B.KV_ERR_INVALID_ARG
