@@ -61,7 +61,10 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
   const unsigned lane = threadIdx.x & 31u;
   EventCounter ec;
   ec.init(lane);
+  // ids are 32-bit, so the bound is too (an id can never reach 2^32 - 1 = "no entry")
+  const uint32_t n32 = n > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)n;
   uint32_t bad = 0;
+  bool bad_id = false, not_resident = false;
   for (uint64_t it = 0; it < iters; ++it) {
     uint32_t ids[kEventVecs][4], hit[kEventVecs][4], pr[kEventVecs][4];
     bool valid[kEventVecs];
@@ -69,7 +72,7 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
     for (uint32_t u = 0; u < kEventVecs; ++u) {  // all event loads first
       const uint64_t v = (it * kEventVecs + u) * stride + gtid;
       valid[u] = v < n4;
-      uint4 id4 = make_uint4(0, 0, 0, 0);
+      uint4 id4 = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);  // past the end: out of range
       uchar4 h4 = make_uchar4(0, 0, 0, 0);
       if (valid[u]) {
         id4 = reinterpret_cast<const uint4*>(ev_entry)[v];
@@ -82,14 +85,16 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
     for (uint32_t u = 0; u < kEventVecs; ++u)
 #pragma unroll
       for (int j = 0; j < 4; ++j)  // then all gathers, before any is used
-        pr[u][j] = (valid[u] && ids[u][j] < n) ? pair[ids[u][j]] : kPairFree;
+        pr[u][j] = ids[u][j] < n32 ? pair[ids[u][j]] : kPairFree;
 #pragma unroll
     for (uint32_t u = 0; u < kEventVecs; ++u) {
       bool ok[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        ok[j] = valid[u] && ids[u][j] < n && !(pr[u][j] & kPairFree);
-        if (valid[u] && !ok[j]) bad |= ids[u][j] >= n ? KV_DEV_EVENT_BAD_ID : KV_DEV_EVENT_NOT_RESIDENT;
+        const bool in = ids[u][j] < n32;
+        ok[j] = !(pr[u][j] & kPairFree);   // (out of range gathered nothing: FREE)
+        bad_id |= valid[u] && !in;
+        not_resident |= in && !ok[j];
       }
 #pragma unroll
       for (int j = 0; j < 4; j += 2) {
@@ -104,6 +109,8 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
       for (int j = 0; j < 4; ++j) ec.add(ok[j], (pr[u][j] & 15u) * 2u + hit[u][j]);
     }
   }
+  if (bad_id) bad |= KV_DEV_EVENT_BAD_ID;
+  if (not_resident) bad |= KV_DEV_EVENT_NOT_RESIDENT;
   // ragged tail (n_events not a multiple of 4): first warp of the grid
   if (gtid < 32) {
     const uint64_t e = n4 * 4 + gtid;
