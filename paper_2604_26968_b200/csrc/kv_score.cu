@@ -11,16 +11,13 @@ event_reduce_kernel(const uint32_t* __restrict__ ev_entry, const uint8_t* __rest
                     uint64_t n_events, const uint8_t* __restrict__ pair,
                     uint32_t* __restrict__ touch, uint64_t n,
                     unsigned long long* __restrict__ delta, uint32_t* __restrict__ status) {
-  __shared__ uint32_t s_cnt[32];
-  if (threadIdx.x < 32) s_cnt[threadIdx.x] = 0;
+  __shared__ uint32_t s_cnt[16 * kThreads];   // [pair][thread]: events | hits << 16
+  for (uint32_t i = threadIdx.x; i < 16 * kThreads; i += kThreads) s_cnt[i] = 0;
   __syncthreads();
   const uint32_t bad = reduce_events(ev_entry, ev_hit, n_events, pair, touch, n,
                                      (uint64_t)blockIdx.x * blockDim.x + threadIdx.x,
-                                     (uint64_t)gridDim.x * blockDim.x, s_cnt);
+                                     (uint64_t)gridDim.x * blockDim.x, s_cnt, delta);
   if (bad) atomicOr(status, bad);
-  __syncthreads();
-  if (threadIdx.x < 32 && s_cnt[threadIdx.x])
-    atomicAdd(&delta[threadIdx.x], (unsigned long long)s_cnt[threadIdx.x]);
 }
 
 cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit, uint64_t n_events,

@@ -13,125 +13,181 @@ namespace kvt {
 // ---- event reduction ---------------------------------------------------------
 // Each event adds one to the (pair, hit) counter of its entry's pair -- the
 // alpha += 1 / beta += 1 update of the Bayesian reuse section -- and one to the
-// entry's touch count.  Counters are integers, so the order of the atomics does
-// not matter.
+// entry's touch count.  Counters are integers, so the order of the additions
+// does not matter.
 //
-// The 32 (pair, hit) counters are kept one per lane: for every event slot the
-// warp takes six votes (valid, and the five bits of key = 2*pair + hit); lane L
-// combines them into the mask of lanes whose key is L and adds its population
-// count to a register.  No shared-memory atomics and no match instruction in the
-// loop; a warp's 32 registers go to 32 shared counters once, at the end, and a
-// block issues one 64-bit global atomic per non-zero counter.
-constexpr uint32_t kEventVecs = 2;  // 4-event vectors a thread has in flight per iteration
+// Pair counters: every thread owns 16 packed counters in shared memory (one per
+// pair: events in the low half, hits in the high half), laid out pair-major so
+// that the threads of a warp always fall into 32 different banks.  Counting an
+// event is a plain read-add-write of the thread's own word: no vote, no atomic.
+// The block adds its columns up once at the end.
+//
+// Touch counts: every update is a 64-bit atomic on the aligned pair of 32-bit
+// counts (touch[2i], touch[2i+1]) -- adding 1, 1 << 32 or both -- so that all
+// atomics on a word have one size.  (A carry out of the low count would need
+// 2^32 touches of one entry in one epoch, where the count wraps anyway.)  The
+// one exception is the last entry of an array of odd length, whose partner
+// would lie outside the array: it takes 32-bit atomics, and only those.
+//
+// Traces in which a touched block reports all its heads hand every thread four
+// consecutive entries (an aligned group of four ids): one 4-byte load then
+// fetches their pairs and FREE bits, and two atomics count the four touches.
+constexpr uint32_t kEventVecs = 2;          // 4-event vectors a thread has in flight per iteration
+constexpr uint32_t kEventFlushIters = 4096; // iterations between flushes: 8 events each, below 2^16
 
-struct EventCounter {
-  uint32_t flip[5];  // bit b of the lane id clear -> all ones (selects lanes whose key bit b is clear)
-  uint32_t cnt;      // events seen with key == lane id
-  __device__ __forceinline__ void init(unsigned lane) {
-#pragma unroll
-    for (int b = 0; b < 5; ++b) flip[b] = ((lane >> b) & 1u) ? 0u : 0xFFFFFFFFu;
-    cnt = 0;
-  }
-  // every lane of the warp must call it
-  __device__ __forceinline__ void add(bool counted, uint32_t key) {
-    uint32_t m = __ballot_sync(0xFFFFFFFFu, counted);
-#pragma unroll
-    for (int b = 0; b < 5; ++b) m &= __ballot_sync(0xFFFFFFFFu, (key >> b) & 1u) ^ flip[b];
-    cnt += __popc(m);
-  }
+struct EventVec {
+  uint32_t id[4];
+  uint32_t hit4;   // bit 8j+7 set: event j carried a hit flag
+  uint32_t pr4;    // byte j: pair byte of event j's entry (bit 7 = FREE or out of range)
+  bool valid, run; // vector inside the trace; ids are an aligned run of four inside the pool
 };
 
-// The calling block's share of the events: thread `gtid` of `stride` takes
-// kEventVecs vectors of four consecutive events at a time, so that all their
-// scattered gathers are in flight together.  One byte per event is gathered: the entry's pair, whose bit 7 says
-// that the entry is FREE.  Two consecutive events on the two entries of an
-// aligned pair (2i, 2i+1) -- the normal case when a touched block reports all its
-// heads -- share one 64-bit atomic on the two 32-bit touch counts (a carry out of
-// the low count would need 2^32 touches, where the count wraps anyway).  Every
-// thread of the block must call it (the votes need all lanes).  s_cnt: 32 zeroed
-// shared-memory counters, index 2*pair + hit; returns the KV_DEV_* bits of
-// refused events.
+// bit 7 of every non-zero byte
+__device__ __forceinline__ uint32_t nonzero_bytes(uint32_t x) {
+  return (((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x) & 0x80808080u;
+}
+
+__device__ __forceinline__ void touch_add(uint32_t* __restrict__ touch, uint32_t i, uint32_t n32,
+                                          unsigned long long inc_pair) {
+  // inc_pair: what to add to the aligned pair that contains entry i
+  if ((i | 1u) < n32)
+    atomicAdd(reinterpret_cast<unsigned long long*>(touch + (i & ~1u)), inc_pair);
+  else
+    atomicAdd(&touch[i], 1u);   // last entry of an odd-length array (i is even, inc_pair is 1)
+}
+
+// The calling block's share of the events.  s_cnt: kThreads * 16 words of shared
+// memory, zero on entry; on return word [p * blockDim.x + t] holds thread t's
+// counts for pair p (events | hits << 16) since the last flush.  delta: the 32
+// global epoch counters (index 2 * pair + hit).  Returns the KV_DEV_* bits of
+// refused events.  Every thread of the block must call it.
 __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ ev_entry,
                                                   const uint8_t* __restrict__ ev_hit, uint64_t n_events,
                                                   const uint8_t* __restrict__ pair,
                                                   uint32_t* __restrict__ touch, uint64_t n, uint64_t gtid,
-                                                  uint64_t stride, uint32_t* s_cnt) {
+                                                  uint64_t stride, uint32_t* s_cnt,
+                                                  unsigned long long* __restrict__ delta) {
   const uint64_t n4 = n_events / 4;
   const uint64_t iters = (n4 + stride * kEventVecs - 1) / (stride * kEventVecs);  // same for every thread
-  const unsigned lane = threadIdx.x & 31u;
-  EventCounter ec;
-  ec.init(lane);
   // ids are 32-bit, so the bound is too (an id can never reach 2^32 - 1 = "no entry")
   const uint32_t n32 = n > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)n;
-  uint32_t bad = 0;
+  uint32_t* my = s_cnt + threadIdx.x;
+  const uint32_t col = blockDim.x;
   bool bad_id = false, not_resident = false;
+
+  // adds the block's columns to the global counters and clears them
+  auto flush = [&]() {
+    __syncthreads();
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
+    for (uint32_t p = warp; p < 16; p += n_warps) {
+      uint32_t ev = 0, hi = 0;
+      for (uint32_t t = lane; t < col; t += 32) {
+        const uint32_t c = s_cnt[p * col + t];
+        s_cnt[p * col + t] = 0;
+        ev += c & 0xFFFFu;
+        hi += c >> 16;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        ev += __shfl_xor_sync(0xFFFFFFFFu, ev, o);
+        hi += __shfl_xor_sync(0xFFFFFFFFu, hi, o);
+      }
+      if (lane == 0) {
+        if (hi) atomicAdd(&delta[2 * p + 1], (unsigned long long)hi);
+        if (ev - hi) atomicAdd(&delta[2 * p], (unsigned long long)(ev - hi));
+      }
+    }
+    __syncthreads();
+  };
+  // counts event j of a vector (pair byte and hit bit already extracted)
+  auto count = [&](uint32_t prj, uint32_t hitbit) { my[(prj & 15u) * col] += 1u + (hitbit << 16); };
+
   for (uint64_t it = 0; it < iters; ++it) {
-    uint32_t ids[kEventVecs][4], hit[kEventVecs][4], pr[kEventVecs][4];
-    bool valid[kEventVecs];
+    EventVec x[kEventVecs];
 #pragma unroll
     for (uint32_t u = 0; u < kEventVecs; ++u) {  // all event loads first
       const uint64_t v = (it * kEventVecs + u) * stride + gtid;
-      valid[u] = v < n4;
+      x[u].valid = v < n4;
       uint4 id4 = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);  // past the end: out of range
-      uchar4 h4 = make_uchar4(0, 0, 0, 0);
-      if (valid[u]) {
+      uint32_t h4 = 0;
+      if (x[u].valid) {
         id4 = reinterpret_cast<const uint4*>(ev_entry)[v];
-        h4 = reinterpret_cast<const uchar4*>(ev_hit)[v];
+        h4 = reinterpret_cast<const uint32_t*>(ev_hit)[v];
       }
-      ids[u][0] = id4.x; ids[u][1] = id4.y; ids[u][2] = id4.z; ids[u][3] = id4.w;
-      hit[u][0] = h4.x != 0; hit[u][1] = h4.y != 0; hit[u][2] = h4.z != 0; hit[u][3] = h4.w != 0;
+      x[u].id[0] = id4.x; x[u].id[1] = id4.y; x[u].id[2] = id4.z; x[u].id[3] = id4.w;
+      x[u].hit4 = nonzero_bytes(h4);
+      x[u].run = !(id4.x & 3u) && id4.y == id4.x + 1u && id4.z == id4.x + 2u && id4.w == id4.x + 3u &&
+                 id4.w < n32;
     }
 #pragma unroll
-    for (uint32_t u = 0; u < kEventVecs; ++u)
+    for (uint32_t u = 0; u < kEventVecs; ++u) {  // then all gathers, before any is used
+      if (x[u].run) {
+        x[u].pr4 = *reinterpret_cast<const uint32_t*>(pair + x[u].id[0]);
+      } else {
+        uint32_t pr4 = 0;
 #pragma unroll
-      for (int j = 0; j < 4; ++j)  // then all gathers, before any is used
-        pr[u][j] = ids[u][j] < n32 ? pair[ids[u][j]] : kPairFree;
+        for (int j = 0; j < 4; ++j)
+          pr4 |= (uint32_t)(x[u].id[j] < n32 ? pair[x[u].id[j]] : (uint8_t)kPairFree) << (8 * j);
+        x[u].pr4 = pr4;
+      }
+    }
 #pragma unroll
     for (uint32_t u = 0; u < kEventVecs; ++u) {
+      const uint32_t pr4 = x[u].pr4, hit4 = x[u].hit4;
+      if (x[u].run && !(pr4 & 0x80808080u)) {
+        // four resident entries in a row: two atomics, four counts
+        unsigned long long* t2 = reinterpret_cast<unsigned long long*>(touch + x[u].id[0]);
+        atomicAdd(t2, 0x100000001ull);
+        atomicAdd(t2 + 1, 0x100000001ull);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) count(pr4 >> (8 * j), (hit4 >> (8 * j + 7)) & 1u);
+        continue;
+      }
+      if (!x[u].valid) continue;
       bool ok[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const bool in = ids[u][j] < n32;
-        ok[j] = !(pr[u][j] & kPairFree);   // (out of range gathered nothing: FREE)
-        bad_id |= valid[u] && !in;
+        const bool in = x[u].id[j] < n32;
+        ok[j] = !((pr4 >> (8 * j)) & kPairFree);   // (out of range gathered nothing: FREE)
+        bad_id |= !in;
         not_resident |= in && !ok[j];
       }
 #pragma unroll
       for (int j = 0; j < 4; j += 2) {
-        if (ok[j] && ok[j + 1] && ids[u][j + 1] == ids[u][j] + 1u && !(ids[u][j] & 1u)) {
-          atomicAdd(reinterpret_cast<unsigned long long*>(touch + ids[u][j]), 0x100000001ull);
+        const uint32_t i0 = x[u].id[j], i1 = x[u].id[j + 1];
+        if (ok[j] && ok[j + 1] && i1 == i0 + 1u && !(i0 & 1u)) {
+          atomicAdd(reinterpret_cast<unsigned long long*>(touch + i0), 0x100000001ull);
         } else {
-          if (ok[j]) atomicAdd(&touch[ids[u][j]], 1u);
-          if (ok[j + 1]) atomicAdd(&touch[ids[u][j + 1]], 1u);
+          if (ok[j]) touch_add(touch, i0, n32, (i0 & 1u) ? (1ull << 32) : 1ull);
+          if (ok[j + 1]) touch_add(touch, i1, n32, (i1 & 1u) ? (1ull << 32) : 1ull);
         }
       }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) ec.add(ok[j], (pr[u][j] & 15u) * 2u + hit[u][j]);
+      for (int j = 0; j < 4; ++j)
+        if (ok[j]) count(pr4 >> (8 * j), (hit4 >> (8 * j + 7)) & 1u);
     }
+    if ((it + 1) % kEventFlushIters == 0) flush();   // (uniform over the block)
   }
+  uint32_t bad = 0;
   if (bad_id) bad |= KV_DEV_EVENT_BAD_ID;
   if (not_resident) bad |= KV_DEV_EVENT_NOT_RESIDENT;
-  // ragged tail (n_events not a multiple of 4): first warp of the grid
-  if (gtid < 32) {
+  // ragged tail (n_events not a multiple of 4): first threads of the grid
+  if (gtid < 3) {
     const uint64_t e = n4 * 4 + gtid;
-    bool ok = false;
-    uint32_t key = 0;
     if (e < n_events) {
       const uint32_t i = ev_entry[e];
-      const uint32_t pr = i < n ? pair[i] : kPairFree;
-      if (i >= n) {
+      const uint32_t pr = i < n32 ? pair[i] : kPairFree;
+      if (i >= n32) {
         bad |= KV_DEV_EVENT_BAD_ID;
       } else if (pr & kPairFree) {
         bad |= KV_DEV_EVENT_NOT_RESIDENT;
       } else {
-        ok = true;
-        key = (pr & 15u) * 2u + (ev_hit[e] != 0);
-        atomicAdd(&touch[i], 1u);
+        count(pr, ev_hit[e] != 0);
+        touch_add(touch, i, n32, (i & 1u) ? (1ull << 32) : 1ull);
       }
     }
-    ec.add(ok, key);
   }
-  if (ec.cnt) atomicAdd(&s_cnt[lane], ec.cnt);
+  flush();
   return bad;
 }
 

@@ -108,6 +108,7 @@ struct kv_pool {
     const uint32_t* victims = nullptr;
     uint64_t off[4] = {0, 0, 0, 0}, kq[4] = {0, 0, 0, 0}, per[4] = {0, 0, 0, 0};
     uint64_t next[4] = {0, 0, 0, 0}, cursor0[4] = {0, 0, 0, 0};
+    uint64_t promoted[4] = {0, 0, 0, 0};  // entries promoted into the partition since this demotion began
     cudaStream_t compute = nullptr, copy = nullptr;
   };
   Pending pending;
@@ -756,6 +757,7 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
     pd.kq[q] = kq[q];
     pd.per[q] = per[q];
     pd.next[q] = 0;
+    pd.promoted[q] = 0;
     pd.cursor0[q] = q < p->n_parts ? p->host[q].cursor : 0;
     off += kq[q];
   }
@@ -866,12 +868,13 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
       j += len;
     }
     KV_CUDA(p, cudaEventRecord(p->ev_ready[b], copy));
-    // The entries of this chunk go to the (c0+cnt) lowest FREE slots of the partition.  Any of those
-    // that the pending demotion freed is among its first (c0+cnt) victims of the partition (victims and
-    // free slots are both in ascending id order), so their payload must have been packed: enqueue
-    // that much of the demotion first.
+    // With P entries promoted into the partition since the pending demotion began, this chunk
+    // fills FREE slots number P+c0 .. P+c0+cnt-1 of the free set as it was right after that
+    // demotion.  Any of those that the demotion freed is among its first P+c0+cnt victims of the
+    // partition (victims and free slots are both in ascending id order), so that much of its
+    // payload must have been packed: enqueue it first.
     if (p->pending.active) {
-      const int32_t rc = drain_pending(p, q, c0 + cnt, ~0ull);
+      const int32_t rc = drain_pending(p, q, p->pending.promoted[q] + c0 + cnt, ~0ull);
       if (rc != KV_OK) return rc;
     }
     KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_ready[b], 0));
@@ -886,6 +889,7 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
   KV_CUDA(p, cudaEventRecord(p->ev_list_free[li], compute));
   KV_CUDA(p, cudaEventRecord(p->ev_h2d_done, copy));
   p->h2d_valid = true;
+  if (p->pending.active) p->pending.promoted[q] += m;
   for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 0;
   h.n_live -= m;
   h.n_free -= m;

@@ -36,7 +36,8 @@ def oracle_admit(w, pool, epoch, key=None):
 
 class Lockstep:
     def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True,
-                 policy=0, blend=None, deferred=False, fused=False, heads=None, lazy=False):
+                 policy=0, blend=None, deferred=False, fused=False, heads=None, lazy=False,
+                 split_promote=1):
         self.w = w
         self.payload = payload
         self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
@@ -44,6 +45,7 @@ class Lockstep:
         self.options = (policy, blend)
         self.deferred = deferred
         self.fused = fused   # score and select through the single fused call
+        self.split_promote = split_promote   # each partition's promote list goes in this many calls
         # heads = (decay, every): importance matrices of all partitions updated before every
         # epoch's scoring, multipliers set on epochs divisible by `every` and reset on the next
         self.heads = heads
@@ -194,8 +196,10 @@ class Lockstep:
             self.compare_ring("epoch %d demote" % e)
         lists = g.promote_lists(e)
         for q, lst in enumerate(lists):
-            assert o.promote(q, lst) == O.OK
-            g.check(g.pool.kv_promote(q, lst, g.batch_bytes), "kv_promote")
+            pieces = np.array_split(lst, self.split_promote) if self.split_promote > 1 else [lst]
+            for piece in pieces:
+                assert o.promote(q, piece) == O.OK
+                g.check(g.pool.kv_promote(q, piece, g.batch_bytes), "kv_promote")
         self.compare_state("epoch %d promote" % e, scores=False)
         self.compare_ring("epoch %d promote" % e)
         self.fresh = oracle_admit(w, o, e)

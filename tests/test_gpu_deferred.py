@@ -42,3 +42,26 @@ def test_deferred_packing_with_promotions_of_just_demoted_slots_and_block_mode()
     for e in range(8, 12):
         ls.epoch(e, k_blocks=40)
     ls.close()
+
+
+@pytest.mark.parametrize("cfg,scale,batch_kb,pieces", [
+    (1, 1.0, 16, 3),         # 81 promotions in calls of 27: the later calls land beyond the first victims
+    (2, 1 / 64, 256, 4),
+    (5, 1 / 128, 512, 2),
+])
+def test_deferred_packing_with_several_promotions_per_partition(cfg, scale, batch_kb, pieces):
+    """A promote list longer than max_promote has to be split by the caller, so several
+    kv_promote calls on one partition between a demotion and the next draining call are
+    normal.  Every later call scatters into freed slots further up the victim list, whose
+    payload must have been packed by then: ring bytes of those victims and slab bytes of
+    the promoted blocks are compared in full."""
+    from lockstep import Lockstep
+    w = W.config(cfg, scale=scale)
+    if cfg == 5:
+        for p in w.parts:
+            p.ring_slots = w.k + 64
+    ls = Lockstep(w, payload=True, batch_bytes=batch_kb << 10, deferred=True, split_promote=pieces)
+    for e in range(6):
+        r = ls.epoch(e)
+        assert r["promoted"] > 0
+    ls.close()
