@@ -75,8 +75,10 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
   const uint32_t col = blockDim.x;
   bool bad_id = false, not_resident = false;
 
-  // adds the block's columns to the global counters and clears them
+  // adds the block's columns to the global counters and clears them; the 32 sums
+  // go out as one warp's 32 neighbouring atomics (a single request per cache line)
   auto flush = [&]() {
+    __shared__ uint32_t s_tot[32];
     __syncthreads();
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
     for (uint32_t p = warp; p < 16; p += n_warps) {
@@ -93,10 +95,13 @@ __device__ __forceinline__ uint32_t reduce_events(const uint32_t* __restrict__ e
         hi += __shfl_xor_sync(0xFFFFFFFFu, hi, o);
       }
       if (lane == 0) {
-        if (hi) atomicAdd(&delta[2 * p + 1], (unsigned long long)hi);
-        if (ev - hi) atomicAdd(&delta[2 * p], (unsigned long long)(ev - hi));
+        s_tot[2 * p + 1] = hi;
+        s_tot[2 * p] = ev - hi;
       }
     }
+    __syncthreads();
+    if (threadIdx.x < 32 && s_tot[threadIdx.x])
+      atomicAdd(&delta[threadIdx.x], (unsigned long long)s_tot[threadIdx.x]);
     __syncthreads();
   };
   // counts event j of a vector (pair byte and hit bit already extracted)

@@ -3,12 +3,30 @@
 // The multi-launch selection in kv_select.cu spends most of its time between
 // kernels when the pool has a few million entries: ten dependent launches of
 // 3-10 us each.  Here one CTA per SM stays resident for the whole selection.
-// Each CTA owns a contiguous slice of the entries, converts its slice's scores
-// to order-preserving keys ONCE and keeps them in shared memory (up to 40 K keys
-// per SM, i.e. 6 M entries on 148 SMs; the rest of a larger slice is re-read
-// from the score array, which then sits in L2), and the phases of the
-// selection -- the histograms, the count, the ordered write -- are separated
-// by grid-wide barriers instead of kernel boundaries.
+// Each CTA owns a contiguous slice of the entries; the phases of the selection
+// are separated by grid-wide barriers instead of kernel boundaries:
+//
+//   A  every score becomes an order-preserving key (fused form: the entry pass
+//      itself produces it) and enters the first histogram.  With a hint -- tau of
+//      the previous selection -- the histogram covers a bracket of 2^22 keys
+//      around it, and the pass also leaves in shared memory a bitmap "key below
+//      the bracket" and a list of the keys inside the bracket (index in the
+//      slice, bracket bin, low bits): typically 5-10 % of the slice.
+//   B  the remaining histograms of the radix select.  When rank k falls inside
+//      the bracket, ONE more histogram (the 2^11 single keys of the bracket bin
+//      that holds rank k) finishes it, and it is built from the list alone: no
+//      second pass over the scores.  Otherwise (no hint, a miss, a list that
+//      overflowed) the keys are re-read from the score array, which then sits
+//      mostly in L2; the last histogram of that path leaves the bitmaps "key
+//      below the final range" and "key inside the final range".
+//   C  tau picked: the keys of the final range are sorted into "below tau" and
+//      "equal to tau" -- from the list, or, on the other path, by fetching just
+//      the keys inside the range (not even those when the CTA's own histogram
+//      shows that all of them equal tau: a tie, the usual case when few distinct
+//      scores exist).
+//   D  per-CTA counts = population counts of the two bitmaps; after the last
+//      barrier every CTA knows how many victims precede its slice and writes its
+//      own victims in ascending id order straight from the bitmaps.
 //
 // The grid barrier is a counter in global memory that every CTA increments and
 // then polls.  A cooperative launch guarantees that all CTAs are resident, so
@@ -17,26 +35,31 @@
 //
 // The same kernel also exists fused with the per-entry scoring pass (FUSED =
 // true): every CTA first updates the entries of its own slice (posterior, EMA,
-// score) and turns the fresh scores straight into keys -- the score array is
-// written for the caller but never read back, and a kernel boundary disappears.
-// The event reduction stays a launch of its own ahead of it: its scattered gathers
-// and atomics ran 2.5x slower inside this kernel when that was tried, and a grid
-// barrier costs about what the launch boundary does.
+// score) and turns the fresh scores straight into keys -- a kernel boundary
+// disappears.  The event reduction stays a launch of its own ahead of it: its
+// scattered gathers and atomics ran 2.5x slower inside this kernel when that was
+// tried, and a grid barrier costs about what the launch boundary does.
+#include <cstdlib>
+#include <mutex>
+#include <type_traits>
+
 #include "kv_score_device.cuh"
 
 namespace kvt {
 
 constexpr uint32_t kPThreads = 1024;
 constexpr uint32_t kPChunk = kPThreads * 4;             // 4096 entries: one 16-byte vector per thread
-constexpr uint32_t kPKeyCap = 40960;                    // most keys kept in shared memory per CTA (160 KB)
 constexpr uint32_t kPHistBins = 2048;
 constexpr uint32_t kExcluded = 0xFFFFFFFFu;             // key of a non-candidate (FREE) entry
 constexpr uint32_t kBarrierSpins = 1u << 22;
 constexpr uint32_t kBracketShift = 11;                  // a bracket bin is 2^11 keys wide ...
 constexpr uint32_t kBracketHalf = 1u << 21;             // ... and the 2,048 bins reach 2^21 keys to either side of the hint
+constexpr uint32_t kBracketBits = 22;                   // log2 of the bracket's width in keys
+constexpr uint32_t kPIdxBits = 18;                      // index of an entry inside its slice
+constexpr uint32_t kPMaxSlice = 1u << kPIdxBits;        // entries per CTA the bitmaps are sized for (2 x 32 KB)
+constexpr uint32_t kPListCapMax = 16384;                // bracket keys remembered per CTA (6 bytes each)
 
-static_assert(kPKeyCap % kPChunk == 0, "the cached part of a slice is a whole number of chunks");
-static_assert(kPKeyCap < 65536, "per-CTA counts of the cached part are packed in 16 bits");
+static_assert(kPIdxBits + kBracketBits - kBracketShift <= 32, "index and bracket bin share one word");
 
 __device__ __forceinline__ uint32_t p_score_key(float s) {
   uint32_t b = __float_as_uint(s);
@@ -44,20 +67,38 @@ __device__ __forceinline__ uint32_t p_score_key(float s) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// Adds one to s_hist[bin] for every active lane; one atomic when the warp agrees
-// on the bin (the common case while most scores are equal).
-__device__ __forceinline__ void p_warp_hist_add(uint32_t* s_hist, bool active, uint32_t bin) {
-  const unsigned m = __ballot_sync(0xFFFFFFFFu, active);
-  if (m == 0) return;
-  const int leader = __ffs(m) - 1;
-  const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, bin, leader);
-  const bool same = !active || bin == b0;
-  if (__all_sync(0xFFFFFFFFu, same)) {
-    if ((int)(threadIdx.x & 31u) == leader) atomicAdd(&s_hist[b0], (uint32_t)__popc(m));
-  } else if (active) {
-    atomicAdd(&s_hist[bin], 1u);
+// Adds one to s_hist[bin] for every active lane.  When the warp agrees on the bin
+// (the common case while many scores are equal) the addition is not even issued:
+// the warp carries a pending (bin, count) pair, identical in all its lanes, and
+// only a change of bin sends the count to shared memory.  Atomics of different
+// warps on one hot address serialise at ~18 cycles each, which is what a pass
+// over a heavily tied slice used to spend its time on.
+struct WarpHist {
+  uint32_t bin = 0, cnt = 0;
+  // m = the warp's vote on `active` (every lane calls, with the same m)
+  __device__ __forceinline__ void add_voted(uint32_t* s_hist, unsigned m, bool active, uint32_t b) {
+    if (m == 0) return;
+    const int leader = __ffs(m) - 1;
+    const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, b, leader);
+    const bool same = !active || b == b0;
+    if (__all_sync(0xFFFFFFFFu, same)) {
+      if (b0 != bin) {
+        flush(s_hist);
+        bin = b0;
+      }
+      cnt += (uint32_t)__popc(m);
+    } else if (active) {
+      atomicAdd(&s_hist[b], 1u);
+    }
   }
-}
+  __device__ __forceinline__ void add(uint32_t* s_hist, bool active, uint32_t b) {
+    add_voted(s_hist, __ballot_sync(0xFFFFFFFFu, active), active, b);
+  }
+  __device__ __forceinline__ void flush(uint32_t* s_hist) {
+    if (cnt && (threadIdx.x & 31u) == 0) atomicAdd(&s_hist[bin], cnt);
+    cnt = 0;
+  }
+};
 
 struct PArgs {
   const float* score;
@@ -69,8 +110,9 @@ struct PArgs {
   SelectScalars* sel;
   uint2* cta_counts;      // [gridDim.x]
   uint32_t* status;
-  unsigned long long per; // entries per CTA slice (multiple of 4)
-  uint32_t cap;           // keys of a slice kept in shared memory (a multiple of kPChunk, at most kPKeyCap)
+  unsigned long long per; // entries per CTA slice (multiple of 4, at most kPMaxSlice)
+  uint32_t words;         // 32-bit words of one bitmap of a slice (a multiple of 4)
+  uint32_t list_cap;      // entries of the bracket list (a multiple of 8)
   // the scoring pass of the fused form
   EntryState st;
   Predictor pd;
@@ -153,20 +195,23 @@ __device__ __forceinline__ void pick_bin(const uint32_t* __restrict__ hist, uint
 
 template <bool FUSED>
 __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const PArgs a) {
-  extern __shared__ __align__(16) uint32_t s_keys[];  // a.cap keys
+  extern __shared__ __align__(16) uint32_t s_dyn[];
+  uint32_t* const s_bit_l = s_dyn;                    // bit j: key of local entry j is below tau
+  uint32_t* const s_bit_e = s_bit_l + a.words;        // bit j: key of local entry j equals tau
+  uint32_t* const s_list_jb = s_bit_e + a.words;      // bracket list: index in slice | bracket bin << kPIdxBits
+  uint16_t* const s_list_low = reinterpret_cast<uint16_t*>(s_list_jb + a.list_cap);  // ... and key bits below the bin
   __shared__ uint32_t s_hist[kPHistBins];
-  __shared__ uint32_t s_hist_first[kPHistBins];  // the CTA's own first (bracket) histogram
   __shared__ uint32_t s_warp[32];
   __shared__ uint32_t s_pick[2];
+  __shared__ uint32_t s_list_n;
   __shared__ float sP[16];
   const uint32_t t = threadIdx.x;
+  const uint32_t lane = t & 31u;
   unsigned int* bar = &a.sel->bar_arrive;
   const unsigned int G = gridDim.x;
   const unsigned long long s0 = (unsigned long long)blockIdx.x * a.per;
   const unsigned long long s1 = (s0 + a.per < a.n) ? s0 + a.per : a.n;
   const uint32_t len = s1 > s0 ? (uint32_t)(s1 - s0) : 0u;
-  const uint32_t cached = len < a.cap ? len : a.cap;               // local [0, cached) lives in s_keys
-  const uint32_t first_far = a.cap / kPChunk;                      // first chunk beyond the cache
   const uint32_t n_chunks = (len + kPChunk - 1) / kPChunk;
   bool ok = true;
   auto stamp = [&](int i) {
@@ -197,22 +242,53 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
                                                                         : kExcluded;
     }
   };
-
-  // Applies f(key) to every key of the slice, all threads in lock step (f may
-  // vote across the warp): the cached part with a stride of one block, the far
-  // part chunk by chunk from the arrays.
-  auto for_each_key = [&](auto f) {
-    const uint32_t iters = (cached + kPThreads - 1) / kPThreads;
-    for (uint32_t i = 0; i < iters; ++i) {
-      const uint32_t j = i * kPThreads + t;
-      f(j < cached ? s_keys[j] : kExcluded);
-    }
-    for (uint32_t c = first_far; c < n_chunks; ++c) {
-      uint32_t key[4];
-      keys_from_arrays(c, key);
+  // A pass over the slice's keys, re-read from the arrays: body(c, key) sees the thread's
+  // four keys of every chunk c, last chunk first (the end of the slice is what the cache
+  // hierarchy saw last), all threads in lock step (body may vote across the warp).  The
+  // loads of kAhead chunks are issued before the first of them is used.
+  constexpr uint32_t kAhead = 2;
+  auto for_chunks = [&](auto body) {
+    uint32_t c = n_chunks;
+    while (c > 0) {
+      const uint32_t nb = c < kAhead ? c : kAhead;
+      float4 sc[kAhead];
+      uchar4 st[kAhead];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) f(key[j]);
+      for (uint32_t u = 0; u < kAhead; ++u) {
+        const uint32_t j0 = (c - 1u - u) * kPChunk + 4u * t;
+        if (u < nb && j0 + 4 <= len) {
+          sc[u] = __ldcg(reinterpret_cast<const float4*>(a.score + s0 + j0));
+          st[u] = __ldcg(reinterpret_cast<const uchar4*>(a.state + s0 + j0));
+        }
+      }
+#pragma unroll
+      for (uint32_t u = 0; u < kAhead; ++u) {
+        if (u < nb) {
+          const uint32_t cc = c - 1u - u;
+          const uint32_t j0 = cc * kPChunk + 4u * t;
+          uint32_t key[4];
+          if (j0 + 4 <= len) {
+            key[0] = st[u].x == KV_STATE_RESIDENT ? p_score_key(sc[u].x) : kExcluded;
+            key[1] = st[u].y == KV_STATE_RESIDENT ? p_score_key(sc[u].y) : kExcluded;
+            key[2] = st[u].z == KV_STATE_RESIDENT ? p_score_key(sc[u].z) : kExcluded;
+            key[3] = st[u].w == KV_STATE_RESIDENT ? p_score_key(sc[u].w) : kExcluded;
+          } else {
+            keys_from_arrays(cc, key);   // the ragged end of the slice
+          }
+          body(cc, key);
+        }
+      }
+      c -= nb;
     }
+  };
+  // Eight lanes x four bits (a lane holds 4 consecutive entries) -> the bitmap word of
+  // the 32 entries starting at j0 of the lane with (lane & 7) == 0, which stores it.
+  auto store_word = [&](uint32_t* bits, uint32_t nib, uint32_t j0) {
+    uint32_t v = nib << (4u * (lane & 7u));
+    v |= __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+    v |= __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+    v |= __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+    if ((lane & 7u) == 0 && (j0 >> 5) < a.words) bits[j0 >> 5] = v;
   };
   auto clear_hist = [&]() {
     for (uint32_t b = t; b < kPHistBins; b += kPThreads) s_hist[b] = 0;
@@ -225,6 +301,10 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       if (c) atomicAdd(&g_hist[b], c);
     }
   };
+  // every thread owns a contiguous run of bitmap words
+  const uint32_t wpt = (a.words + kPThreads - 1) / kPThreads;
+  const uint32_t w0 = t * wpt < a.words ? t * wpt : a.words;
+  const uint32_t w1 = w0 + wpt < a.words ? w0 + wpt : a.words;
 
   if constexpr (FUSED) {
     // reuse estimates from the totals plus this epoch's counts (final: the event
@@ -235,30 +315,57 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       sP[t] = reuse_estimate(a.pd, t, P, h, m, wh, wm);
     }
   }
+  for (uint32_t w = t; w < 2 * a.words; w += kPThreads) s_bit_l[w] = 0;   // both bitmaps
+  if (t == 0) s_list_n = 0;
 
-  // ---- phase A: keys into shared memory, and the first histogram ----
+  // ---- phase A: keys and the first histogram ----
   // Without a hint the first histogram is digit 0 of a plain radix select (bits
-  // 31..21 of every key).  With a hint -- tau of the previous selection over the
-  // same number of keys -- it covers only the bracket [lo, lo + 2^22) around that
-  // tau in 2,048 bins of 2^11 keys, and keys below lo are merely counted: scores
+  // 31..21 of every key).  With a hint it covers only the bracket [base0, base0 +
+  // 2^22) around the hinted tau in 2,048 bins of 2^11 keys; keys below base0 set
+  // their bit in s_bit_l (and are counted), keys inside go on the list: scores
   // move little from one epoch to the next, so the k-th key is almost always
-  // inside, few keys need an atomic, and one later pass (2^11 keys wide) finishes
-  // the selection instead of two.  If rank k falls outside the bracket the plain
-  // radix select runs after all, from the cached keys.
+  // inside, and then nothing but the list is looked at again.
   const bool hint = a.sel->hint_valid != 0 && a.sel->hint_n == a.n;
   const uint32_t hint_tau = a.sel->hint_tau;
   const uint32_t base0 = hint ? (hint_tau > kBracketHalf ? hint_tau - kBracketHalf : 0u) : 0u;
   const uint32_t shift0 = hint ? kBracketShift : 21u;
-  uint32_t n_below0 = 0;  // keys of this thread below the bracket
-  auto first_pass = [&](uint32_t key) {
-    n_below0 += (key < base0);  // (an excluded key is 0xFFFFFFFF: never below)
-    const bool cand = key != kExcluded && key >= base0 && ((key - base0) >> shift0) < kPHistBins;
-    p_warp_hist_add(s_hist, cand, (key - base0) >> shift0);
+  WarpHist wh;
+  auto phase_a = [&](uint32_t c, const uint32_t key[4]) {
+    if (!hint) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) wh.add(s_hist, key[q] != kExcluded, key[q] >> 21);
+      return;
+    }
+    const uint32_t j0 = c * kPChunk + 4u * t;
+    uint32_t nib = 0, d[4], m[4], total = 0;
+    bool in[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      d[q] = key[q] - base0;
+      nib |= (uint32_t)(key[q] < base0) << q;   // (an excluded key is 0xFFFFFFFF: never below)
+      in[q] = key[q] != kExcluded && key[q] >= base0 && (d[q] >> kBracketBits) == 0u;
+      m[q] = __ballot_sync(0xFFFFFFFFu, in[q]);
+      total += (uint32_t)__popc(m[q]);
+    }
+    store_word(s_bit_l, nib, j0);
+    if (total == 0) return;   // (uniform over the warp)
+    uint32_t at = 0;
+    if (lane == 0) at = atomicAdd(&s_list_n, total);
+    at = __shfl_sync(0xFFFFFFFFu, at, 0);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      wh.add_voted(s_hist, m[q], in[q], d[q] >> kBracketShift);
+      const uint32_t pos = at + (uint32_t)__popc(m[q] & ((1u << lane) - 1u));
+      if (in[q] && pos < a.list_cap) {
+        s_list_jb[pos] = (j0 + q) | ((d[q] >> kBracketShift) << kPIdxBits);
+        s_list_low[pos] = (uint16_t)(d[q] & ((1u << kBracketShift) - 1u));
+      }
+      at += (uint32_t)__popc(m[q]);
+    }
   };
   clear_hist();
   if constexpr (FUSED) {
-    // the slice's entries go through the EMA and score update on the way; keys of
-    // the far part are histogrammed here too, from registers
+    // the slice's entries go through the EMA and score update on the way
     const int policy = a.pd.policy;
     const uint32_t jt = 4u * t;
     EntryVec cur;
@@ -289,34 +396,17 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         }
       }
       cur = nxt;
-      if (c < first_far) {
-        reinterpret_cast<uint4*>(s_keys)[c * kPThreads + t] = make_uint4(key[0], key[1], key[2], key[3]);
-      } else {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) first_pass(key[j]);
-      }
-    }
-    __syncthreads();
-    const uint32_t iters = (cached + kPThreads - 1) / kPThreads;
-    for (uint32_t i = 0; i < iters; ++i) {
-      const uint32_t j = i * kPThreads + t;
-      first_pass(j < cached ? s_keys[j] : kExcluded);
+      phase_a(c, key);
     }
   } else {
-    const uint32_t cached_chunks = (cached + kPChunk - 1) / kPChunk;
-#pragma unroll 4
-    for (uint32_t c = 0; c < cached_chunks; ++c) {
-      uint32_t key[4];
-      keys_from_arrays(c, key);
-      reinterpret_cast<uint4*>(s_keys)[c * kPThreads + t] = make_uint4(key[0], key[1], key[2], key[3]);
-    }
-    __syncthreads();
-    for_each_key(first_pass);
+    for_chunks(phase_a);
   }
-  flush_hist(a.hist, kPHistBins);
-  uint32_t cta_below0 = 0;  // keys of this CTA's slice below the bracket
+  wh.flush(s_hist);
+  flush_hist(a.hist, kPHistBins);   // (begins with a block barrier: the bitmap words are all written)
   if (hint) {
-    (void)block_scan_excl(n_below0, s_warp, cta_below0);
+    uint32_t below = 0, cta_below0;
+    for (uint32_t w = w0; w < w1; ++w) below += (uint32_t)__popc(s_bit_l[w]);
+    (void)block_scan_excl(below, s_warp, cta_below0);
     if (t == 0 && cta_below0) atomicAdd(&a.sel->below, (unsigned long long)cta_below0);
   }
   stamp(1);
@@ -329,7 +419,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   }
 
   {
-    // ---- phases B, C: narrow [base, base + 2^shift) around rank k, one histogram per step ----
+    // ---- phase B: narrow [base, base + 2^shift) around rank k, one histogram per step ----
     // The current histogram is a.hist[h]; it was built over [base, base + 2048 << shift).
     // Every CTA reads the same global data, so all of them take the same path.
     uint32_t h = 0, nbar = 1, base = base0, shift = shift0;
@@ -337,16 +427,57 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     uint32_t bin, before;
     bool found = true;
     bool clear_below = hint;
-    bool bracket_hit = false;   // rank k was inside the bracket: two histograms in all
-    uint32_t bin_first = 0;     // ... and this was its bin of the first one
+    bool use_list = false;   // rank k is inside the bracket and this CTA's list holds all its bracket keys
+    const uint32_t n_list = s_list_n;
     auto hist_pass = [&](uint32_t width_log2, uint32_t new_shift, uint32_t h_new) {
       // histogram of ((key - base) >> new_shift) over the keys in [base, base + 2^width_log2)
       clear_hist();
       const uint32_t top = width_log2 - new_shift;  // log2 of the number of bins
-      for_each_key([&](uint32_t key) {
-        const uint32_t d = key - base;
-        p_warp_hist_add(s_hist, key != kExcluded && key >= base && ((d >> new_shift) >> top) == 0u, d >> new_shift);
-      });
+      WarpHist w2;
+      if (new_shift != 0) {
+        for_chunks([&](uint32_t, const uint32_t key[4]) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t d = key[q] - base;
+            w2.add(s_hist, key[q] != kExcluded && key[q] >= base && ((d >> new_shift) >> top) == 0u,
+                   d >> new_shift);
+          }
+        });
+      } else if (use_list) {
+        // the last histogram (single keys of the bracket bin that holds rank k) from the
+        // list; listed keys of earlier bins are below the range: their bit joins s_bit_l
+        const uint32_t bin_k = (base - base0) >> kBracketShift;
+        const uint32_t iters = (n_list + kPThreads - 1) / kPThreads;
+        for (uint32_t i = 0; i < iters; ++i) {
+          const uint32_t e = i * kPThreads + t;
+          uint32_t b = 0xFFFFFFFFu, j = 0, low = 0;
+          if (e < n_list) {
+            const uint32_t v = s_list_jb[e];
+            b = v >> kPIdxBits;
+            j = v & (kPMaxSlice - 1u);
+            low = s_list_low[e];
+          }
+          if (b < bin_k) atomicOr(&s_bit_l[j >> 5], 1u << (j & 31u));
+          w2.add(s_hist, b == bin_k, low);
+        }
+      } else {
+        // the last histogram (single keys) from the arrays; it also leaves the bitmaps "key
+        // below the range" in s_bit_l and "key inside the range" in s_bit_e
+        for_chunks([&](uint32_t c, const uint32_t key[4]) {
+          uint32_t nl = 0, ne = 0;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t d = key[q] - base;
+            const bool in = key[q] != kExcluded && key[q] >= base && (d >> top) == 0u;
+            nl |= (uint32_t)(key[q] < base) << q;
+            ne |= (uint32_t)in << q;
+            w2.add(s_hist, in, d);
+          }
+          store_word(s_bit_l, nl, c * kPChunk + 4u * t);
+          store_word(s_bit_e, ne, c * kPChunk + 4u * t);
+        });
+      }
+      w2.flush(s_hist);
       flush_hist(a.hist + h_new * kPHistBins, 1u << top);
     };
     auto retire = [&](uint32_t h_old) {   // after a barrier: nobody reads histogram h_old any more
@@ -362,14 +493,9 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       pick_bin(a.hist, kPHistBins, above ? a.k - below : 1ull, s_warp, s_pick, bin, before);
       if (above && bin != 0xFFFFFFFFu) {
         k_rem = a.k - below;
-        // The CTA's own first histogram is still in s_hist: keep it.  Together with its own
-        // second histogram it gives this slice's counts below and at tau without another
-        // pass over the keys.
-        bracket_hit = true;
-        bin_first = bin;
-        for (uint32_t b = t; b < kPHistBins; b += kPThreads) s_hist_first[b] = s_hist[b];
+        use_list = n_list <= a.list_cap;
       } else {
-        // rank k is outside the bracket: digit 0 of the plain radix select, from the cached keys
+        // rank k is outside the bracket: digit 0 of the plain radix select
         base = 0;
         shift = 21;
         hist_pass(32, 21, 1);
@@ -386,7 +512,6 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       found = found && bin != 0xFFFFFFFFu;
       k_rem -= before;
       base += (bin & (kPHistBins - 1u)) << shift;   // rank k lies in [base, base + 2^shift)
-      if (shift == 0) break;
       const uint32_t new_shift = shift > 11u ? shift - 11u : 0u;
       const uint32_t h_new = (h + 1u) % 3u;
       hist_pass(shift, new_shift, h_new);
@@ -396,116 +521,105 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       retire(h);
       pick_bin(a.hist + h_new * kPHistBins, 1u << (shift - new_shift), k_rem, s_warp, s_pick, bin, before);
       h = h_new;
+      if (new_shift == 0) break;   // bin is tau's offset inside the final range [base, base + 2^shift)
       shift = new_shift;
     }
+    found = found && bin != 0xFFFFFFFFu;
+    k_rem -= before;
 
-    // ---- phase D: tau is known; count (key < tau, key == tau) in the slice ----
-    const uint32_t tau = base;
+    // ---- phases C, D: tau is known; complete the bitmaps and count ----
+    const uint32_t tau_low = found ? bin : 0u;          // tau - base
+    const uint32_t tau = base + tau_low;
     const unsigned long long need_eq = k_rem;
-    if (bracket_hit) {
-      // below tau = below the bracket + bins of the first histogram before rank k's bin +
-      // bins of the second (single keys, still in s_hist) before tau; at tau = tau's bin
-      const uint32_t bin_tau = tau - (base0 + (bin_first << kBracketShift));
-      uint32_t v = 0;
-      for (uint32_t b = t; b < kPHistBins; b += kPThreads)
-        v += (b < bin_first ? s_hist_first[b] : 0u) + (b < bin_tau ? s_hist[b] : 0u);
-      uint32_t tot_less;
-      (void)block_scan_excl(v, s_warp, tot_less);
-      if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(cta_below0 + tot_less, s_hist[bin_tau]);
+    uint32_t c_l = 0, c_e = 0;
+    if (use_list) {
+      const uint32_t bin_k = (base - base0) >> kBracketShift;
+      for (uint32_t e = t; e < n_list; e += kPThreads) {
+        const uint32_t v = s_list_jb[e];
+        if ((v >> kPIdxBits) != bin_k) continue;
+        const uint32_t j = v & (kPMaxSlice - 1u), low = s_list_low[e];
+        if (low < tau_low) atomicOr(&s_bit_l[j >> 5], 1u << (j & 31u));
+        else if (low == tau_low) atomicOr(&s_bit_e[j >> 5], 1u << (j & 31u));
+      }
+      __syncthreads();
+      for (uint32_t w = w0; w < w1; ++w) {
+        c_l += (uint32_t)__popc(s_bit_l[w]);
+        c_e += (uint32_t)__popc(s_bit_e[w]);
+      }
     } else {
-      uint32_t n_less = 0, n_eq = 0;
-      for_each_key([&](uint32_t key) {
-        n_less += (key != kExcluded && key < tau);
-        n_eq += (key != kExcluded && key == tau);
-      });
-      uint32_t tot_less, tot_eq;
-      (void)block_scan_excl(n_less, s_warp, tot_less);
-      (void)block_scan_excl(n_eq, s_warp, tot_eq);
-      if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(tot_less, tot_eq);
+      // s_bit_e holds the keys inside the final range; the ones below tau move to s_bit_l,
+      // the ones above tau drop out.  The CTA's own last histogram is still in s_hist: when
+      // all its keys of the range equal tau nothing has to be looked at again, otherwise
+      // only the keys inside the range are fetched.
+      uint32_t in_range = 0, cta_in_range;
+      for (uint32_t w = w0; w < w1; ++w) in_range += (uint32_t)__popc(s_bit_e[w]);
+      (void)block_scan_excl(in_range, s_warp, cta_in_range);
+      const bool all_tau = s_hist[tau_low] == cta_in_range;
+      for (uint32_t w = w0; w < w1; ++w) {
+        uint32_t bl = s_bit_l[w], be = s_bit_e[w];
+        if (!all_tau) {
+          uint32_t bits = be;
+          while (bits) {
+            const uint32_t b = (uint32_t)__ffs(bits) - 1u;
+            bits &= bits - 1u;
+            const uint32_t key = p_score_key(__ldcg(a.score + s0 + 32u * w + b));
+            if (key != tau) be &= ~(1u << b);
+            if (key < tau) bl |= 1u << b;
+          }
+          s_bit_l[w] = bl;
+          s_bit_e[w] = be;
+        }
+        c_l += (uint32_t)__popc(bl);
+        c_e += (uint32_t)__popc(be);
+      }
     }
+    uint32_t tot_l, tot_e;
+    const uint32_t ex_l = block_scan_excl(c_l, s_warp, tot_l);
+    const uint32_t ex_e = block_scan_excl(c_e, s_warp, tot_e);
+    if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(tot_l, tot_e);
     stamp(5);
     ok = grid_barrier(bar, ++nbar * G);
     stamp(6);
     if (!ok) goto fail;
     retire(h);
 
-    // ---- phase E: ordered write ----
     unsigned long long less_before, eq_before;
     {
-      uint32_t la = 0, ea = 0;  // partial sums over the CTAs before this one
+      unsigned long long la = 0, ea = 0;  // sums over the CTAs before this one
       for (uint32_t g = t; g < blockIdx.x; g += kPThreads) {
         const uint2 cc = __ldcg(&a.cta_counts[g]);
         la += cc.x; ea += cc.y;
       }
+      // (G <= 1024: one value per thread at most, each below 2^18)
       uint32_t tl, te;
-      (void)block_scan_excl(la, s_warp, tl);
-      (void)block_scan_excl(ea, s_warp, te);
+      (void)block_scan_excl((uint32_t)la, s_warp, tl);
+      (void)block_scan_excl((uint32_t)ea, s_warp, te);
       less_before = tl; eq_before = te;
     }
-    // Position of a victim.  With L entries below tau and E entries equal to tau before it
-    // in id order, an entry below tau goes to L + min(E, need_eq) and an entry equal to tau,
-    // taken while E < need_eq, to L + E.  Everything before the current piece of the slice is
-    // folded into pos0 and room once per piece, so the per-key arithmetic is 32-bit: ml and me
-    // count inside the piece.
-    unsigned long long pos0 = 0;
-    uint32_t room = 0;
-    auto set_piece = [&]() {
-      pos0 = less_before + (eq_before < need_eq ? eq_before : need_eq);
-      const unsigned long long left = need_eq > eq_before ? need_eq - eq_before : 0ull;
-      room = left > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)left;
-    };
-    auto emit = [&](uint32_t key, unsigned long long id, uint32_t& ml, uint32_t& me) {
-      if (key > tau) return;   // most keys (an excluded key is 0xFFFFFFFF)
-      if (key < tau) {
-        const unsigned long long pos = pos0 + ml + (me < room ? me : room);
-        if (pos < a.k) a.victims[pos] = (uint32_t)id;
-        ++ml;
-      } else if (key != kExcluded) {
-        if (me < room) {
-          const unsigned long long pos = pos0 + ml + me;
-          if (pos < a.k) a.victims[pos] = (uint32_t)id;
-        }
-        ++me;
-      }
-    };
     if (found) {
-      // cached part: every thread owns a contiguous run of L keys (L odd: the
-      // strided shared-memory reads of a warp then fall into distinct banks)
-      {
-        uint32_t L = (cached + kPThreads - 1) / kPThreads;
-        L |= 1u;
-        const uint32_t j0 = t * L;
-        const uint32_t j1 = (j0 + L < cached) ? j0 + L : cached;
-        uint32_t v = 0;
-        for (uint32_t j = j0; j < j1; ++j) {
-          const uint32_t key = s_keys[j];
-          v += (key < tau) + ((uint32_t)(key == tau && key != kExcluded) << 16);
+      // Position of a victim.  With L entries below tau and E entries equal to tau before it
+      // in id order, an entry below tau goes to L + min(E, need_eq) and an entry equal to tau,
+      // taken while E < need_eq, to L + E.
+      unsigned long long n_l = less_before + ex_l, n_e = eq_before + ex_e;
+      for (uint32_t w = w0; w < w1; ++w) {
+        const uint32_t bl = s_bit_l[w], be = s_bit_e[w];
+        uint32_t bits = bl | be;
+        while (bits) {
+          const uint32_t b = (uint32_t)__ffs(bits) - 1u;
+          bits &= bits - 1u;
+          const unsigned long long id = s0 + 32ull * w + b;
+          if ((bl >> b) & 1u) {
+            const unsigned long long pos = n_l + (n_e < need_eq ? n_e : need_eq);
+            if (pos < a.k) a.victims[pos] = (uint32_t)id;
+            ++n_l;
+          } else {
+            if (n_e < need_eq) {
+              const unsigned long long pos = n_l + n_e;
+              if (pos < a.k) a.victims[pos] = (uint32_t)id;
+            }
+            ++n_e;
+          }
         }
-        uint32_t total;
-        const uint32_t excl = block_scan_excl(v, s_warp, total);
-        set_piece();
-        uint32_t ml = excl & 0xFFFFu, me = excl >> 16;
-        for (uint32_t j = j0; j < j1; ++j) emit(s_keys[j], s0 + j, ml, me);
-        less_before += total & 0xFFFFu;
-        eq_before += total >> 16;
-      }
-      // far part: chunk by chunk, a vector per thread
-      for (uint32_t c = first_far; c < n_chunks; ++c) {
-        uint32_t key[4];
-        keys_from_arrays(c, key);
-        uint32_t v = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          v += (key[j] < tau) + ((uint32_t)(key[j] == tau && key[j] != kExcluded) << 16);
-        uint32_t total;
-        const uint32_t excl = block_scan_excl(v, s_warp, total);
-        set_piece();
-        uint32_t ml = excl & 0xFFFFu, me = excl >> 16;
-        const unsigned long long i0 = s0 + (unsigned long long)c * kPChunk + 4ull * t;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) emit(key[j], i0 + j, ml, me);
-        less_before += total & 0xFFFFu;
-        eq_before += total >> 16;
       }
     }
     if (blockIdx.x == G - 1 && t == 0) {
@@ -549,36 +663,70 @@ done:
   }
 }
 
+// What one device can do with the persistent kernels, probed once per device
+// (with that device current) under a lock.
+namespace {
+struct PersistDevice {
+  int state = 0;   // 0 = not probed, 1 = usable, -1 = not usable
+  int n_sm = 0;
+  size_t smem_max = 0;   // dynamic shared memory the kernels were opted in for
+};
+constexpr int kPMaxDevices = 64;
+std::mutex g_persist_mutex;
+PersistDevice g_persist[kPMaxDevices];
+
+// Dynamic shared memory of a launch: two bitmaps and the bracket list.
+inline size_t persist_smem(uint32_t words, uint32_t list_cap) {
+  return (size_t)words * 8u + (size_t)list_cap * 6u;
+}
+}  // namespace
+
 // Launches the persistent selection (fused with the entry pass when fs is given)
-// if the device can hold one CTA per SM of it co-resident; *used = false (and
-// nothing launched) otherwise.
+// if the device can hold one CTA per SM of it co-resident and the slices fit the
+// bitmaps; *used = false (and nothing launched) otherwise.
 cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
                                      const Workspace& ws, cudaStream_t s, bool* used, const FusedScore* fs) {
   *used = false;
-  static int state = 0;  // 0 = not probed, 1 = usable, -1 = not usable
-  static int n_sm = 0;
-  const size_t smem_max = (size_t)kPKeyCap * 4;
-  if (state == 0) {
-    int dev = 0, coop = 0, blocks = 0, blocks_f = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
-    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(select_persistent_kernel<false>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(select_persistent_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)smem_max);
-    if (e == cudaSuccess)
-      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, select_persistent_kernel<false>,
-                                                        (int)kPThreads, smem_max);
-    if (e == cudaSuccess)
-      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_f, select_persistent_kernel<true>,
-                                                        (int)kPThreads, smem_max);
-    state = (e == cudaSuccess && coop && blocks >= 1 && blocks_f >= 1 && n_sm > 0) ? 1 : -1;
-    (void)cudaGetLastError();
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
+  if (dev < 0 || dev >= kPMaxDevices) return cudaSuccess;
+  PersistDevice pd;
+  {
+    std::lock_guard<std::mutex> lock(g_persist_mutex);
+    PersistDevice& d = g_persist[dev];
+    if (d.state == 0) {
+      int coop = 0, blocks = 0, blocks_f = 0, optin = 0;
+      cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+      cudaDeviceGetAttribute(&d.n_sm, cudaDevAttrMultiProcessorCount, dev);
+      cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+      cudaFuncAttributes fa{}, fb{};
+      cudaError_t e = cudaFuncGetAttributes(&fa, select_persistent_kernel<false>);
+      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, select_persistent_kernel<true>);
+      const size_t fixed = fa.sharedSizeBytes > fb.sharedSizeBytes ? fa.sharedSizeBytes : fb.sharedSizeBytes;
+      // the most a launch asks for: the largest bitmaps and the longest list
+      const size_t want = persist_smem(kPMaxSlice / 32, kPListCapMax);
+      if ((size_t)optin < fixed + want) e = cudaErrorInvalidValue;
+      d.smem_max = want;
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(select_persistent_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)want);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(select_persistent_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)want);
+      if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, select_persistent_kernel<false>,
+                                                          (int)kPThreads, want);
+      if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_f, select_persistent_kernel<true>,
+                                                          (int)kPThreads, want);
+      d.state = (e == cudaSuccess && coop && blocks >= 1 && blocks_f >= 1 && d.n_sm > 0) ? 1 : -1;
+      (void)cudaGetLastError();
+    }
+    pd = d;
   }
-  if (state != 1) return cudaSuccess;
-  unsigned int G = (unsigned int)n_sm;
+  if (pd.state != 1) return cudaSuccess;
+  unsigned int G = (unsigned int)pd.n_sm;
+  if (G > kPThreads) G = kPThreads;  // the prefix over the per-CTA counts takes one CTA per thread
   const uint64_t min_per = kPChunk;  // do not spread tiny pools over more CTAs than they have chunks
   if ((st.n + min_per - 1) / min_per < G) G = (unsigned int)((st.n + min_per - 1) / min_per);
   if (G == 0) G = 1;
@@ -594,14 +742,18 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   a.cta_counts = ws.tile_counts;
   a.status = ws.status;
   a.per = ((st.n + G - 1) / G + 3) / 4 * 4;
-  // Shared memory only for the keys a slice has, and never all of it: what the key cache
-  // does not take stays with the L1, whose lines hold the loads in flight.  Measured on
-  // 11.8 M entries: with 192 KB of keys per SM the streaming entry pass of this kernel took
-  // 68 us, with 160 KB 61 us (and the whole call 227 -> 213 us) although more keys are then
-  // re-read from L2; a 3.1 M pool, whose slices need 96 KB, went from 66.7 to 63.5 us.
-  const uint64_t want = (a.per + kPChunk - 1) / kPChunk * kPChunk;
-  a.cap = (uint32_t)(want < kPKeyCap ? want : kPKeyCap);
-  const size_t smem = (size_t)a.cap * 4;
+  if (a.per > kPMaxSlice) return cudaSuccess;  // slices beyond the bitmaps: the multi-launch selection runs
+  a.words = (uint32_t)((a.per + 31) / 32 + 3) / 4 * 4;
+  // The list holds the keys inside the hint's bracket, typically 5-10 % of a slice; a CTA whose
+  // list overflows re-reads its keys instead.  What this kernel does not take of the shared
+  // memory stays with the L1, whose lines hold the loads in flight of the streaming entry pass.
+  uint64_t list_cap = (a.per / 4 + 7) / 8 * 8;
+  if (const char* e = std::getenv("KVTIER_SELECT_LIST")) list_cap = (uint64_t)std::atoi(e) / 8 * 8;
+  if (list_cap < 8) list_cap = 8;
+  if (list_cap > kPListCapMax) list_cap = kPListCapMax;
+  a.list_cap = (uint32_t)list_cap;
+  const size_t smem = persist_smem(a.words, a.list_cap);
+  if (smem > pd.smem_max) return cudaSuccess;
   a.st = st;
   a.pd = Predictor{};
   a.hw = HeadWeights{};
