@@ -9,11 +9,16 @@ pack + D2H to the pinned host ring (kv_demote), H2D + unpack of prefetched
 entries (kv_promote).  Admission of fresh blocks, which keeps the pool full, is
 a harness step and runs untimed between steps, as does an L2 flush.
 
+By default the pool is the largest of the five that fits the device and the
+pinned host tier (the mixed fleet of 150 GiB, else the 90 GiB long-context pool,
+scaled down by a recorded factor only when free memory says so); --config picks
+one by number.
+
 Prints ONE JSON line.  `value` is KV head-blocks scored + selected per second,
-N / t(scoring + selection), measured inside full steps; the line
-also carries the whole-step rate, per-phase bandwidths, the roofline of the
-dominant kernel, the host-link peak measured in the same run, and the CPU
-oracle timed on the host cores.
+N / t(scoring + selection), measured inside full steps; `roofline` is that
+pass against the HBM peak; the line also carries the whole-step rate, per-phase
+bandwidths (pack / unpack kernels against HBM, copies against the host link
+measured in the same run), and the CPU oracle timed on the host cores.
 """
 import argparse
 import json
@@ -33,12 +38,17 @@ METRIC = "KV head-blocks scored+selected/s"
 UNIT = "head-blocks/s"
 
 # DRAM traffic from ncu (dram__bytes_read.sum + dram__bytes_write.sum) per payload
-# byte of a launch, keyed by move variant: captured on a 256 MiB payload-only
+# byte of a pack launch: captured on a 256 MiB payload-only
 # launch of a 3 GiB pool (487.35 MB of traffic for 268.44 MB of payload) and
-# scaled to the benchmark's launch size in proportion to the payload.  None = no
-# capture of that kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE = {1: 487.35 / 268.44, 0: None}
-PACK_KERNEL_NAME = {1: "move_tma_kernel<true> (pack)", 0: "pack_kernel"}
+# scaled to the benchmark's launch size in proportion to the payload.
+NCU_PACK_TRAFFIC_BYTES_PER_PAYLOAD_BYTE = 487.35 / 268.44
+PACK_KERNEL_NAME = "move_tma_kernel<true> (pack)"
+
+# DRAM traffic of the scoring + selection pass (event_reduce_kernel followed by
+# select_persistent_kernel<true>) from ncu, bytes per launch pair, keyed by pool number: captured
+# at the pool's full entry count with --tiny-entries (these kernels never touch block payload).
+# None = no capture of the kernels as they stand.
+NCU_SCORE_SELECT_TRAFFIC = {}
 
 
 def parse():
@@ -47,8 +57,10 @@ def parse():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, help="pool 1..5")
-    ap.add_argument("--scale", type=float, default=1.0, help="shrinks blocks per layer")
+    ap.add_argument("--config", type=int, default=None,
+                    help="pool 1..5 (default: the largest that fits device memory and the pinned host tier)")
+    ap.add_argument("--scale", type=float, default=None,
+                    help="shrinks blocks per layer (default: 1, or what free memory allows)")
     ap.add_argument("--ring-slots", type=int, default=None)
     ap.add_argument("--batch-mb", type=int, default=1320,
                     help="demote/promote chunk (staging buffer) size; the default lets the default pool's demotion "
@@ -56,8 +68,6 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-hostlink", action="store_true", help="skip the 1 GiB host-link probe")
-    ap.add_argument("--move-variant", type=int, default=1, choices=[0, 1],
-                    help="pack/unpack kernels: 1 = bulk-copy engine, 0 = register path")
     ap.add_argument("--no-deferred-packing", action="store_true",
                     help="enqueue the whole demotion before the promotion instead of interleaving their chunks")
     ap.add_argument("--sharded", action="store_true",
@@ -76,6 +86,50 @@ def parse():
     ap.add_argument("--select-variant", type=int, default=1, choices=[0, 1],
                     help="selection: 1 = one persistent cooperative launch, 0 = one launch per phase")
     return ap.parse_args()
+
+
+def device_need_bytes(w, batch_bytes):
+    """Device memory a pool of this workload takes in the benchmark (slabs, four staging
+    buffers, per-entry state and workspace, block table, the L2-flush buffer, victims)."""
+    per_entry = 26 + 4 + 8 + 4      # state arrays, free list, tile scratch, victim list
+    return (sum(p.slab_bytes for p in w.parts) + 4 * (batch_bytes + (batch_bytes // 8192 + 2) * 24 + 64)
+            + w.N * per_entry + w.n_tags * 4 + sum(p.ring_slots for p in w.parts) * 21 + (256 << 20) + (1 << 30))
+
+
+def host_need_bytes(w):
+    return sum(p.ring_slots * (p.entry_bytes + 24) for p in w.parts) + (2 << 30)
+
+
+def choose_workload(args, torch, W, dev):
+    """The workload to run: --config / --scale if given, else the largest pool that fits."""
+    def make(cfg, scale):
+        return W.config(cfg, scale=scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries)
+    if args.config is not None:
+        scale = 1.0 if args.scale is None else args.scale
+        return args.config, scale, make(args.config, scale), "--config"
+    free_dev, _ = torch.cuda.mem_get_info(dev)
+    try:
+        import psutil
+        free_host = psutil.virtual_memory().available
+    except Exception:
+        free_host = os.sysconf("SC_PAGE_SIZE") * os.sysconf("SC_AVPHYS_PAGES")
+    batch = args.batch_mb << 20
+    why = ""
+    for cfg in (5, 3, 2):
+        scale = 1.0 if args.scale is None else args.scale
+        w = make(cfg, scale)
+        fit = min(1.0, 0.97 * free_dev / device_need_bytes(w, batch), 0.6 * free_host / host_need_bytes(w))
+        if fit >= 1.0:
+            return cfg, scale, w, why + "pool %d fits: %.0f GiB free on the device, %.0f GiB free on the host" % (
+                cfg, free_dev / 2**30, free_host / 2**30)
+        if args.scale is None and fit >= 0.5:
+            scale = int(fit * 20) / 20.0      # in steps of 0.05, rounded down
+            return cfg, scale, make(cfg, scale), why + (
+                "pool %d scaled by %.2f: %.0f GiB free on the device, %.0f GiB free on the host" % (
+                    cfg, scale, free_dev / 2**30, free_host / 2**30))
+        why += "pool %d does not fit (needs %.0f GiB device, %.0f GiB pinned host); " % (
+            cfg, device_need_bytes(w, batch) / 2**30, host_need_bytes(w) / 2**30)
+    return 2, 1.0, make(2, 1.0), why
 
 
 def measured_peaks():
@@ -270,25 +324,97 @@ def oracle_epochs(w, n_epochs, warm=0):
     return t_ss, t_all, done
 
 
+def oracle_movement(W, cfg, target_bytes=1 << 30, epochs=3):
+    """GB/s of the oracle's memcpy-based demotion and promotion (payload mode, 1 thread)
+    on the workload scaled down to about target_bytes of slab."""
+    from paper_2604_26968_b200.harness import INITIAL_EPOCH_KEY
+    full = W.config(cfg)
+    scale = min(1.0, target_bytes / sum(p.slab_bytes for p in full.parts))
+    w = W.config(cfg, scale=scale)
+    O, _ = None, None
+    from oracle import kv_oracle as O
+    parts = [dict(model=O.Model(p.variant, p.n_layers, p.n_q_heads, p.n_kv_heads, p.head_dim,
+                                p.d_latent, p.d_rope, p.dtype_bits),
+                  block_tokens=p.block_tokens, blocks_per_layer=p.blocks_per_layer,
+                  ring_slots=p.ring_slots) for p in w.parts]
+    pool = O.OraclePool(parts, w.alpha0, w.beta0, n_tags=w.n_tags, payload=True)
+
+    def admit(e, key):
+        fresh = np.flatnonzero(pool.state == O.FREE).astype(np.uint32)
+        nbytes = 0
+        for q in range(pool.n_parts):
+            inf = pool.info(q)
+            nbytes += int((pool.state[inf["base"]:inf["base"] + inf["n"]] == O.FREE).sum()) * inf["entry_bytes"]
+        pool.admit(e, w.decay, w.new_pairs(key, fresh.size), np.zeros(nbytes, np.uint8))
+        return fresh
+
+    fresh = admit(0, INITIAL_EPOCH_KEY)
+    t_dem = t_pro = 0.0
+    b_dem = b_pro = 0
+    for e in range(epochs):
+        ev_entry, ev_hit = w.events(e, pool.pair, fresh)
+        assert pool.epoch_score(e, ev_entry, ev_hit) == O.OK
+        rc, v = pool.select_victims(w.k)
+        assert rc == O.OK
+        s0 = pool.stats()
+        t0 = time.perf_counter()
+        assert pool.demote(v) == O.OK
+        t_dem += time.perf_counter() - t0
+        for q, p in enumerate(w.parts):
+            inf = pool.info(q)
+            live = pool.part_array(q, "r_live")
+            n_fq = int((pool.state[inf["base"]:inf["base"] + inf["n"]] == O.FREE).sum())
+            m_q = min(int(w.promote_frac * p.n_entries), n_fq, int(live.sum()))
+            lst = w.promote_list(e, q, m_q, inf["cursor"], live, just_written=n_fq)
+            t0 = time.perf_counter()
+            assert pool.promote(q, lst) == O.OK
+            t_pro += time.perf_counter() - t0
+        s1 = pool.stats()
+        b_dem += s1["bytes_demoted"] - s0["bytes_demoted"]
+        b_pro += s1["bytes_promoted"] - s0["bytes_promoted"]
+        fresh = admit(e, e)
+    pool.close()
+    return {"demote_gbs": b_dem / max(t_dem, 1e-12) / 1e9, "promote_gbs": b_pro / max(t_pro, 1e-12) / 1e9,
+            "pool_bytes": sum(p.slab_bytes for p in w.parts), "scale": scale, "epochs": epochs}
+
+
+def reference_workload(args, W):
+    """The pool the CUDA arm would choose on this machine (asks the device for its free
+    memory when one is there; no kernel is launched)."""
+    try:
+        import torch
+        if torch.cuda.is_available():
+            local = int(os.environ.get("LOCAL_RANK", "0"))
+            return choose_workload(args, torch, W, torch.device("cuda", local))
+    except Exception:
+        pass
+    cfg = args.config if args.config is not None else 5
+    scale = args.scale if args.scale is not None else 1.0
+    return cfg, scale, W.config(cfg, scale=scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries), \
+        "no CUDA device to ask"
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle, as it stands, on the host cores."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2604_26968_b200 import workloads as W
-    w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries)
+    cfg, scale, w, why = reference_workload(args, W)
     t_ss, t_all, done = oracle_epochs(w, args.steps, warm=args.warmup)
     value = w.N * done / t_ss
     sample = "%d full epochs of pool %d (N=%d) in metadata mode (no payload bytes), 1 thread" % (
-        done, args.config, w.N)
+        done, cfg, w.N)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_ss / done,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": w.name, "pool": args.config, "n_entries": w.N,
-                                        "k": w.k, "scale": args.scale},
+        "data": "synthetic", "config": {"workload": w.name, "pool": cfg, "n_entries": w.N,
+                                        "k": w.k, "scale": scale, "chosen_because": why},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "e2e": {"value": w.N * done / t_all, "unit": UNIT, "scope": "whole epoch (score, select, demote, "
+                "promote) in metadata mode: no payload bytes move", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
@@ -319,7 +445,7 @@ def main():
             os.environ["RANK"], os.environ["WORLD_SIZE"] = "0", "1"
         dist.init_process_group("nccl", device_id=dev)
 
-    w = W.config(args.config, scale=args.scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries)
+    cfg, scale, w, chosen_because = choose_workload(args, torch, W, dev)
     w.seed = w.seed + 1000 * rank     # every rank owns its own pool and trace (weak scaling)
     link = hostlink_probe(torch, dev) if rank == 0 and not args.no_hostlink else None
     runner = EpochRunner(w, batch_bytes=args.batch_mb << 20, fill_pattern=True, host_meta=True,
@@ -327,8 +453,7 @@ def main():
     pool = runner.pool
     pool.kv_timing_enable(True)
     from paper_2604_26968_b200 import binding as B
-    B.kv_set_move_variant(args.move_variant)
-    B.kv_set_select_variant(args.select_variant)
+    pool.kv_set_select_variant(args.select_variant)
     pool.kv_set_deferred_packing(not args.no_deferred_packing)
     N, k = w.N, w.k
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -398,6 +523,7 @@ def main():
             torch.cuda.synchronize(dev)
             pool.kv_timing_read()                 # discard warm-up launches
             launches0 = pool.kv_get_stats()["kernel_launches"]
+            sel0 = pool.kv_selection_stats()
             sampler.start()
         ev_entry, ev_hit = gen_events(epoch)
         d_e, d_h, n = runner.stage_events(ev_entry, ev_hit)
@@ -422,6 +548,7 @@ def main():
     if dist_on:
         dist.barrier()
     clocks = sampler.stop()
+    sel1 = pool.kv_selection_stats()
     timing = pool.kv_timing_read()
     status = pool.kv_device_status()
     K = args.steps
@@ -466,7 +593,9 @@ def main():
         tw = torch.tensor([wall], dtype=torch.float64, device=dev)
         if dist_on:
             dist.all_reduce(tw, op=dist.ReduceOp.MAX)
-        e2e = {"value": N * world * e2e_steps / float(tw.item()), "unit": "head-blocks/s (whole epoch, host in/out)",
+        e2e = {"value": N * world * e2e_steps / float(tw.item()), "unit": UNIT,
+               "scope": "whole epoch (score, select, demote, promote) through the C ABI, events copied in "
+                        "from pinned host memory and the victim list read back",
                "h2d_bytes_per_step": h2d_b // e2e_steps, "d2h_bytes_per_step": d2h_b // e2e_steps,
                "steps": e2e_steps, "ms_per_step": 1e3 * float(tw.item()) / e2e_steps}
 
@@ -521,7 +650,10 @@ def main():
     pack_gbs = 2 * timing["pack_bytes"] / max(timing["pack_ms"], 1e-9) / 1e6
     unpack_gbs = 2 * timing["unpack_bytes"] / max(timing["unpack_ms"], 1e-9) / 1e6
     ss_bytes = 39 * N + 5 * (tot["events"] / K) + 4 * k
-    tr = NCU_TRAFFIC_BYTES_PER_PAYLOAD_BYTE[args.move_variant]
+    ss_gbs = ss_bytes / (ss_ms * 1e-3) / 1e9
+    fused = not (args.no_fused or dist_on)
+    ss_traffic = NCU_SCORE_SELECT_TRAFFIC.get(cfg) if (fused and scale == 1.0 and not args.head_weights) else None
+    tr = NCU_PACK_TRAFFIC_BYTES_PER_PAYLOAD_BYTE
     line = {
         "metric": METRIC, "value": N * world / (ss_ms * 1e-3), "unit": UNIT,
         "value_definition": "N / t(scoring + selection), timed with CUDA events inside full steps; "
@@ -531,19 +663,19 @@ def main():
         "whole_step_head_blocks_per_s": N * world / (all_ms * 1e-3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": {"workload": w.name, "pool": args.config, "n_entries": N, "k": k,
+        "config": {"workload": w.name, "pool": cfg, "chosen_because": chosen_because, "n_entries": N, "k": k,
                    "events_per_step": tot["events"] // K, "pool_bytes": sum(p.slab_bytes for p in w.parts),
                    "entry_bytes": [p.entry_bytes for p in w.parts], "batch_bytes": runner.batch_bytes,
                    "deferred_packing": not args.no_deferred_packing,
                    "fused_score_select": not (args.no_fused or dist_on),
                    "head_weights": bool(args.head_weights),
-                   "ring_slots": [p.ring_slots for p in w.parts], "scale": args.scale,
+                   "ring_slots": [p.ring_slots for p in w.parts], "scale": scale,
                    "parallelism": "1 pool per GPU" + (", 256-byte all-reduce of pair counters" if dist_on else ""),
                    "l2": "flushed before every step: 8 x 256 MiB written on the step's stream (and >1 GB of "
                          "fresh blocks admitted between steps)"},
         "phases": {
             "score_select_ms": ss_ms,
-            "score_select_effective_gbs": ss_bytes / (ss_ms * 1e-3) / 1e9,
+            "score_select_effective_gbs": ss_gbs,
             "demote_ms": dem_ms, "demote_gbs": demoted_per_step / (dem_ms * 1e-3) / 1e9,
             "promote_ms": pro_ms, "promote_gbs": promoted_per_step / max(pro_ms * 1e-3, 1e-12) / 1e9,
             "pack_kernel_gbs": pack_gbs, "pack_kernel_frac_of_%s_hbm" % peak_kind: pack_gbs / peak,
@@ -551,10 +683,22 @@ def main():
             "pack_launches": timing["pack_launches"], "unpack_launches": timing["unpack_launches"],
         },
         "hostlink": link,
-        "roofline": {"kernel": PACK_KERNEL_NAME[args.move_variant], "bound": "hbm", "achieved": pack_gbs, "peak": peak,
-                     "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": pack_gbs / peak,
-                     "traffic": (tr * timing["pack_bytes"] / max(timing["pack_launches"], 1)) if tr else None,
-                     "algorithmic_bytes_per_launch": 2 * timing["pack_bytes"] / max(timing["pack_launches"], 1)},
+        "roofline": {"kernel": ("event_reduce_kernel + select_persistent_kernel<true>" if fused else
+                                "event_reduce_kernel + entry_update_kernel + select_persistent_kernel<false>")
+                               + " (the scoring + selection pass that `value` times)",
+                     "bound": "hbm", "achieved": ss_gbs, "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
+                     "frac": ss_gbs / peak, "traffic": ss_traffic,
+                     "algorithmic_bytes_per_launch": ss_bytes,
+                     "algorithmic_bytes": "39 B/entry (30 scoring + 9 selection) + 5 B/event + 4 B/victim",
+                     "launch_us": 1e3 * ss_ms,
+                     "selection_hints": {"selections": sel1["selections"] - sel0["selections"],
+                                         "hits": sel1["hint_hits"] - sel0["hint_hits"],
+                                         "misses": sel1["hint_misses"] - sel0["hint_misses"],
+                                         "thread_blocks_that_reread_their_keys": sel1["reread_ctas"] - sel0["reread_ctas"]}},
+        "roofline_pack": {"kernel": PACK_KERNEL_NAME, "bound": "hbm", "achieved": pack_gbs, "peak": peak,
+                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": pack_gbs / peak,
+                          "traffic": tr * timing["pack_bytes"] / max(timing["pack_launches"], 1),
+                          "algorithmic_bytes_per_launch": 2 * timing["pack_bytes"] / max(timing["pack_launches"], 1)},
         "clocks": clocks,
         "gpu_launches": tot.get("launches", 0),
         "device_status": status,
@@ -574,11 +718,17 @@ def main():
     if not args.no_cpu_baseline:
         n_ep = 6
         t_ss, t_all, done = oracle_epochs(w, n_ep, warm=1)
+        mv = oracle_movement(W, cfg)
         line["cpu_baseline"] = {
             "value": N * done / t_ss, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": "%d epochs of the same pool (N=%d, k=%d) in metadata mode, score+select timed; host has %d cores"
                       % (done, N, k, os.cpu_count() or 0),
-            "ms_per_epoch_score_select": 1e3 * t_ss / done}
+            "ms_per_epoch_score_select": 1e3 * t_ss / done,
+            "whole_epoch_head_blocks_per_s": N * done / t_all,
+            "movement": {"demote_gbs": mv["demote_gbs"], "promote_gbs": mv["promote_gbs"],
+                         "sample": "%d epochs of the same pool scaled by %.4g (%.2f GiB of blocks) in payload mode: "
+                                   "memcpy-based demotion and promotion, 1 thread"
+                                   % (mv["epochs"], mv["scale"], mv["pool_bytes"] / 2**30)}}
     print(json.dumps(line))
     runner.close()
     if dist_on:

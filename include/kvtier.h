@@ -29,7 +29,8 @@
  *     and the other way round); keep each call's copy stream the same over time;
  *   - device and pinned pointers must be 16-byte aligned;
  *   - functions return KV_OK (0) or a negative kv_status; on a negative status
- *     detected by the host nothing has been enqueued and no state has changed;
+ *     detected by the host no state has changed and nothing that changes state has
+ *     been enqueued;
  *   - an entry is one head-granular KV block: physical slot (layer, block, head)
  *     of a partition, local id (layer*blocks_per_layer + block)*heads + head,
  *     global id = partition base + local id (partitions are laid end to end in
@@ -293,13 +294,26 @@ int32_t kv_epoch_score_select(kv_pool* pool, uint32_t epoch, const uint32_t* d_e
  * of a partition takes ring slot (cursor + j) mod ring_slots; a live slot that
  * is overwritten is dropped (d_loc of its tag becomes KV_NONE).  Each victim's
  * slot becomes FREE, its tag KV_NONE, and d_loc[tag] = KV_LOC_HOST | slot.
- * With more than one partition the call waits on the host for a 32-byte
- * readback of the per-partition victim counts (everything enqueued before it on
- * `compute` must finish first); single-partition pools never wait.
+ * With more than one partition the host has to know how many victims fall in
+ * each (ring slots are assigned on the host): kv_demote counts them with a small
+ * read-only kernel and WAITS for the 32-byte answer (everything enqueued before it
+ * on `compute` finishes first; the wait is counted in kv_stats.host_waits).
+ * kv_demote_counted takes the counts from the caller and never waits: every
+ * selection call of a pool with several partitions leaves them in pinned host
+ * memory (kv_victim_counts), valid once the selection's stream has run -- a caller
+ * that synchronises there anyway passes them on.  Single-partition pools never wait.
  * batch_bytes must be in [entry_bytes, staging_bytes - metadata room]; see
  * kv_max_batch_bytes. */
 int32_t kv_demote(kv_pool* pool, const uint32_t* d_victims, uint64_t m, uint64_t batch_bytes,
                   kv_stream_t compute, kv_stream_t copy);
+/* h_counts (host, 4 values): victims per partition, in partition order; their sum must be m. */
+int32_t kv_demote_counted(kv_pool* pool, const uint32_t* d_victims, uint64_t m, const uint64_t* h_counts,
+                          uint64_t batch_bytes, kv_stream_t compute, kv_stream_t copy);
+/* Pinned host memory (4 values) that receives the victims per partition of the pool's
+ * last kv_select_victims / kv_epoch_score_select / kv_select_victim_blocks (entries, not
+ * blocks); written by the device, valid once that call's stream has run.  Only pools
+ * with several partitions fill it. */
+const uint64_t* kv_victim_counts(const kv_pool* pool);
 
 /* Promotes the m host ring slots listed in h_host_slots (host, read during the
  * call; all live and distinct) into partition `partition`: runs of consecutive
@@ -370,7 +384,9 @@ int32_t kv_dedup_digests(const uint8_t* d_digests, uint64_t m, uint32_t* d_canon
  * k_blocks x the largest head count), in ascending id order, ready for kv_demote.
  * *h_n_victims (host) receives the number of entries: known without waiting for
  * a single-partition pool; a pool with several partitions waits on the host for a
- * 32-byte readback (everything enqueued on `stream` before it finishes first).
+ * 32-byte readback (everything enqueued on `stream` before it finishes first) --
+ * unless h_n_victims is NULL: then the call returns at once, and the entries per
+ * partition are in kv_victim_counts once `stream` has run.
  * If k_blocks exceeds the number of candidate blocks (not known to the host) the
  * device status word gets KV_DEV_SELECT_MISMATCH. */
 int32_t kv_select_victim_blocks(kv_pool* pool, uint64_t k_blocks, uint32_t* d_victims,
@@ -414,7 +430,7 @@ int32_t kv_select_victims_static(const float* d_score, const uint8_t* d_state, u
  * all that is left first.  Results are the same as without it.  The price is a
  * contract: d_victims must stay valid, and the caller's own kernels must not
  * write into the freed slots, until a later call on the pool has returned and its
- * work on `compute` has run.  Needs the bulk-copy pack kernels (move variant 1). */
+ * work on `compute` has run. */
 int32_t kv_set_deferred_packing(kv_pool* pool, int32_t on);
 
 /* Enqueues (on the streams the demotion was given) whatever deferred packing still
@@ -441,6 +457,7 @@ typedef struct {
   uint64_t bytes_demoted, bytes_promoted, bytes_dropped;
   uint64_t n_entries, n_free;
   uint64_t kernel_launches; /* kernels launched by the library in this process so far */
+  uint64_t host_waits;      /* times kv_demote, kv_promote or kv_select_victim_blocks blocked the host */
 } kv_stats;
 
 /* Host-side counters, kept eagerly at call time. */
@@ -470,16 +487,22 @@ typedef struct {
 int32_t kv_timing_enable(kv_pool* pool, int32_t on);
 int32_t kv_timing_read(kv_pool* pool, kv_timing* out);
 
-/* Measurement aid: which pack/unpack kernels kv_demote and kv_promote launch from
- * now on (process-wide): 1 = shared-memory-staged bulk asynchronous copies
- * (default), 0 = 16-byte loads and stores through registers. */
-int32_t kv_set_move_variant(int32_t variant);
+/* Measurement aid: how this pool's selections run from now on: 1 = one persistent
+ * cooperative launch (default; falls back to 0 where the device cannot co-schedule it
+ * or the pool has more than 262,144 entries per SM), 0 = one launch per phase of the
+ * radix select. */
+int32_t kv_set_select_variant(kv_pool* pool, int32_t variant);
 
-/* Measurement aid: how kv_select_victims runs from now on (process-wide): 1 = one
- * persistent cooperative launch with the keys held in shared memory (default;
- * falls back to 0 where the device cannot co-schedule it), 0 = one launch per
- * phase of the radix select. */
-int32_t kv_set_select_variant(int32_t variant);
+/* Measurement aid: how the pool's persistent selections went so far.  Each starts from
+ * a hint (the threshold of the selection before it): a hit means one short pass after
+ * the scoring pass finished it, a miss that the keys were read again (two or three
+ * passes); reread_ctas counts thread blocks that read their keys again although the
+ * hint held (more keys near the threshold than they could note).  Blocks the host
+ * until `stream` has drained. */
+typedef struct {
+  uint64_t selections, hint_hits, hint_misses, reread_ctas;
+} kv_select_stats;
+int32_t kv_selection_stats(kv_pool* pool, kv_stream_t stream, kv_select_stats* out);
 
 /* The last CUDA error code seen by a call on this pool (0 = none). */
 int32_t kv_last_cuda_error(const kv_pool* pool);

@@ -61,7 +61,11 @@ class kv_pool_desc(C.Structure):
 class kv_stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in
                 ("epochs", "events", "victims", "promoted", "admitted", "bytes_demoted",
-                 "bytes_promoted", "bytes_dropped", "n_entries", "n_free", "kernel_launches")]
+                 "bytes_promoted", "bytes_dropped", "n_entries", "n_free", "kernel_launches", "host_waits")]
+
+
+class kv_select_stats(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in ("selections", "hint_hits", "hint_misses", "reread_ctas")]
 
 
 class kv_timing(C.Structure):
@@ -83,7 +87,7 @@ EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_
            "kv_epoch_update", "kv_set_policy", "kv_set_lazy_decay", "kv_hash_entries", "kv_dedup_table_slots", "kv_dedup_digests", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
-           "kv_set_move_variant", "kv_set_select_variant", "kv_last_cuda_error", "kv_status_string",
+           "kv_set_select_variant", "kv_selection_stats", "kv_demote_counted", "kv_victim_counts", "kv_last_cuda_error", "kv_status_string",
            "kv_version")
 
 _lib = None
@@ -174,9 +178,13 @@ def load():
     L.kv_timing_read.restype = i32
     L.kv_timing_read.argtypes = [vp, C.POINTER(kv_timing)]
     L.kv_set_select_variant.restype = i32
-    L.kv_set_select_variant.argtypes = [i32]
-    L.kv_set_move_variant.restype = i32
-    L.kv_set_move_variant.argtypes = [i32]
+    L.kv_set_select_variant.argtypes = [vp, i32]
+    L.kv_demote_counted.restype = i32
+    L.kv_demote_counted.argtypes = [vp, vp, u64, vp, u64, vp, vp]
+    L.kv_victim_counts.restype = vp
+    L.kv_victim_counts.argtypes = [vp]
+    L.kv_selection_stats.restype = i32
+    L.kv_selection_stats.argtypes = [vp, vp, vp]
     L.kv_last_cuda_error.restype = i32
     L.kv_last_cuda_error.argtypes = [vp]
     L.kv_status_string.restype = C.c_char_p
@@ -209,14 +217,6 @@ def kv_infer_variant(model: kv_model_desc) -> int:
 
 def kv_entry_bytes(model: kv_model_desc, block_tokens: int) -> int:
     return load().kv_entry_bytes(C.byref(model), block_tokens)
-
-
-def kv_set_select_variant(variant: int) -> int:
-    return load().kv_set_select_variant(int(variant))
-
-
-def kv_set_move_variant(variant: int) -> int:
-    return load().kv_set_move_variant(int(variant))
 
 
 def _stream_ptr(s):
@@ -424,6 +424,16 @@ class Pool:
         return self.lib.kv_demote(self._h, d_victims.data_ptr() if m else None, int(m), int(batch_bytes),
                                   _stream_ptr(self.compute), _stream_ptr(self.copy))
 
+    def kv_demote_counted(self, d_victims, m, counts, batch_bytes):
+        c = (C.c_uint64 * 4)(*([int(x) for x in counts] + [0] * (4 - len(counts))))
+        return self.lib.kv_demote_counted(self._h, d_victims.data_ptr() if m else None, int(m), C.byref(c),
+                                          int(batch_bytes), _stream_ptr(self.compute), _stream_ptr(self.copy))
+
+    def kv_victim_counts(self):
+        """Victims per partition of the last selection (read after synchronising the compute stream)."""
+        addr = self.lib.kv_victim_counts(self._h)
+        return [int(x) for x in (C.c_uint64 * 4).from_address(addr)][:len(self.parts)]
+
     def kv_promote(self, partition, h_slots, batch_bytes):
         h_slots = np.ascontiguousarray(h_slots, dtype=np.uint64)
         return self.lib.kv_promote(self._h, partition, h_slots.ctypes.data_as(C.c_void_p) if h_slots.size else None,
@@ -472,6 +482,16 @@ class Pool:
         if rc != KV_OK:
             raise KVError(rc, "kv_device_status")
         return bits.value
+
+    def kv_set_select_variant(self, variant):
+        return self.lib.kv_set_select_variant(self._h, int(variant))
+
+    def kv_selection_stats(self):
+        s = kv_select_stats()
+        rc = self.lib.kv_selection_stats(self._h, _stream_ptr(self.compute), C.byref(s))
+        if rc != KV_OK:
+            raise KVError(rc, "kv_selection_stats")
+        return {n: int(getattr(s, n)) for n, _ in kv_select_stats._fields_}
 
     def kv_timing_enable(self, on=True):
         return self.lib.kv_timing_enable(self._h, 1 if on else 0)

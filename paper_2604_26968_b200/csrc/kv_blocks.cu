@@ -44,8 +44,13 @@ block_aggregate_kernel(const float* __restrict__ score, const uint8_t* __restric
 // contiguous, so off follows from the per-partition block counts).
 __global__ void __launch_bounds__(kThreads)
 block_expand_kernel(const uint32_t* __restrict__ block_victims, uint64_t k_blocks, const BlockGeom bg,
-                    const unsigned long long* __restrict__ part_counts, uint32_t* __restrict__ victims) {
+                    const unsigned long long* __restrict__ part_counts, uint32_t* __restrict__ victims,
+                    unsigned long long* __restrict__ h_entry_counts) {
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  if (h_entry_counts && blockIdx.x == 0 && threadIdx.x < 4)   // what kv_demote will want to know
+    h_entry_counts[threadIdx.x] = (int)threadIdx.x < bg.n_parts
+                                      ? (bg.n_parts == 1 ? k_blocks : part_counts[threadIdx.x]) * bg.heads[threadIdx.x]
+                                      : 0ull;
   for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k_blocks; j += stride) {
     const uint64_t gb = block_victims[j];
     const int q = block_partition(bg, gb);
@@ -63,13 +68,14 @@ block_expand_kernel(const uint32_t* __restrict__ block_victims, uint64_t k_block
 
 static unsigned grid_for(uint64_t n) {
   uint64_t blocks = (n + kThreads - 1) / kThreads;
-  const uint64_t cap = (uint64_t)kSMs * 8;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   return (unsigned)(blocks ? blocks : 1);
 }
 
 cudaError_t launch_select_blocks(const EntryState& st, const BlockGeom& bg, uint64_t k_blocks,
-                                 uint32_t* d_victims, const Workspace& ws, cudaStream_t s) {
+                                 uint32_t* d_victims, const Workspace& ws, cudaStream_t s,
+                                 unsigned long long* h_entry_counts) {
   const uint64_t n_blocks = bg.block_base[bg.n_parts];
   block_aggregate_kernel<<<grid_for(n_blocks), kThreads, 0, s>>>(st.score, st.state, bg, ws.block_score,
                                                                  ws.block_state);
@@ -80,12 +86,14 @@ cudaError_t launch_select_blocks(const EntryState& st, const BlockGeom& bg, uint
   bs.score = ws.block_score;
   bs.state = ws.block_state;
   bs.n = n_blocks;
-  e = launch_select(bs, k_blocks, ws.block_victims, ws, s);
-  if (e != cudaSuccess) return e;
-  e = launch_partition_counts(ws.block_victims, k_blocks, bg.block_base, bg.n_parts, ws, s);
+  PartCounts pc;   // the selected blocks per partition, a by-product of the selection
+  for (int q = 0; q <= 4; ++q) pc.base[q] = bg.block_base[q < bg.n_parts ? q : bg.n_parts];
+  pc.n_parts = bg.n_parts;
+  pc.d_counts = ws.part_counts;
+  e = launch_select(bs, k_blocks, ws.block_victims, ws, s, 1, &pc);
   if (e != cudaSuccess) return e;
   block_expand_kernel<<<grid_for(k_blocks), kThreads, 0, s>>>(ws.block_victims, k_blocks, bg, ws.part_counts,
-                                                              d_victims);
+                                                              d_victims, h_entry_counts);
   count_launches(1);
   return cudaGetLastError();
 }

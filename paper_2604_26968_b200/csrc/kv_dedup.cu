@@ -225,7 +225,7 @@ __global__ void dedup_resolve_kernel(const uint8_t* __restrict__ digests, uint64
 cudaError_t launch_dedup(const uint8_t* digests, uint64_t m, uint32_t* canon, uint32_t* refcount,
                          uint32_t* table, uint64_t table_slots, uint32_t* n_unique, uint32_t* status,
                          cudaStream_t s) {
-  const uint64_t cap = (uint64_t)kSMs * 8;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
   uint64_t cb = ((table_slots > m ? table_slots : m) + kThreads - 1) / kThreads;
   if (cb == 0) cb = 1;
   dedup_clear_kernel<<<(unsigned)(cb > cap ? cap : cb), kThreads, 0, s>>>(table, table_slots, refcount, m, n_unique);

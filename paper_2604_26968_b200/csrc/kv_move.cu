@@ -1,36 +1,11 @@
-// Data-movement kernels: gather of victims into a staging buffer (demotion),
-// scatter of staged entries into free paged slots (promotion), admission of
-// fresh blocks, and initialisation.
-//
-// Tier 1 of the paper's hierarchy is pinned host memory fed by asynchronous DMA
-// on CUDA streams; the copy engines want large contiguous transfers, so the
-// victims' K/V chunks (two 2-4 KB pieces per head-granular entry, or one larger
-// MLA chunk) are first packed back to back.  The kernels are pure byte movers:
-// every lane moves 16 bytes per access, a warp owns one piece of up to 2 KB and
-// keeps four 16-byte loads in flight per lane before storing, and payload
-// accesses use streaming cache hints so that the per-entry state arrays stay in
-// L2.
+// Admission of fresh blocks (a harness step: pattern fill of every FREE slot) and
+// initialisation of a pool's state.  The gather and scatter kernels of demotion
+// and promotion are in kv_move_tma.cu.
 #include "kvtier_internal.cuh"
 
 namespace kvt {
 
 constexpr uint32_t kPieceBytes = 2048;  // 32 lanes x 4 x 16 bytes
-constexpr uint32_t kMetaBytes = 24;     // sizeof(kv_slot_meta)
-
-__device__ __forceinline__ void copy_piece(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
-                                           uint32_t len, uint32_t lane) {
-  uint4 v[4];
-#pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    const uint32_t off = (u * 32 + lane) * 16;
-    if (off < len) v[u] = __ldcs(reinterpret_cast<const uint4*>(src + off));
-  }
-#pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    const uint32_t off = (u * 32 + lane) * 16;
-    if (off < len) __stcs(reinterpret_cast<uint4*>(dst + off), v[u]);
-  }
-}
 
 // Byte offset of chunk c of local entry `local` inside the partition slab.
 __device__ __forceinline__ uint64_t chunk_offset(const PartGeom& g, uint64_t local, uint32_t c) {
@@ -39,144 +14,15 @@ __device__ __forceinline__ uint64_t chunk_offset(const PartGeom& g, uint64_t loc
   return ((lb * g.n_chunks + c) * g.heads + head) * (uint64_t)g.chunk_bytes;
 }
 
-__global__ void __launch_bounds__(kThreads)
-pack_kernel(const PartGeom g, const EntryState st, uint32_t* __restrict__ loc,
-            const uint32_t* __restrict__ victims, uint64_t count, uint64_t ring_start,
-            uint8_t* __restrict__ staging, uint64_t meta_offset, uint32_t* __restrict__ status) {
-  const uint32_t lane = threadIdx.x & 31u;
-  const uint32_t ppc = (g.chunk_bytes + kPieceBytes - 1) / kPieceBytes;  // pieces per chunk
-  const uint32_t ppe = ppc * g.n_chunks;                                  // pieces per entry
-  const uint64_t total = count * ppe;
-  const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
-  for (uint64_t piece = (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); piece < total;
-       piece += warps) {
-    const uint64_t j = piece / ppe;
-    const uint32_t r = (uint32_t)(piece - j * ppe);
-    const uint32_t c = r / ppc;
-    const uint32_t pp = r - c * ppc;
-    const uint32_t v = victims[j];
-    if ((uint64_t)v < g.base || (uint64_t)v >= g.base + g.n) {
-      if (lane == 0) atomicOr(status, KV_DEV_BAD_INDEX);
-      continue;
-    }
-    const uint64_t local = (uint64_t)v - g.base;
-    const uint32_t in_chunk = pp * kPieceBytes;
-    const uint32_t len = min(kPieceBytes, g.chunk_bytes - in_chunk);
-    copy_piece(g.slab + chunk_offset(g, local, c) + in_chunk,
-               staging + j * (uint64_t)g.entry_bytes + (uint64_t)c * g.chunk_bytes + in_chunk, len, lane);
-    if (r == 0 && lane == 0) {
-      // metadata of victim j: its ring slot, the block table, the slot's new state
-      const uint32_t t = st.tag[v];
-      if (st.state[v] != KV_STATE_RESIDENT || t == KV_NONE) {
-        atomicOr(status, KV_DEV_VICTIM_NOT_RESIDENT);
-        continue;
-      }
-      const uint32_t slot = (uint32_t)((ring_start + j) % g.ring_slots);
-      const uint32_t old = g.r_tag[slot];
-      if (old != KV_NONE) loc[old] = KV_NONE;  // overwritten host entry is dropped
-      const uint32_t pr = st.pair[v], le = st.last_epoch[v];
-      const float em = st.ema[v], de = st.decay[v];
-      g.r_tag[slot] = t;
-      g.r_pair[slot] = (uint8_t)pr;
-      g.r_ema[slot] = em;
-      g.r_decay[slot] = de;
-      g.r_last_epoch[slot] = le;
-      g.r_depoch[slot] = g.epoch_now;
-      loc[t] = KV_LOC_HOST | slot;
-      st.state[v] = KV_STATE_FREE;
-      st.pair[v] = (uint8_t)(pr | kPairFree);
-      st.tag[v] = KV_NONE;
-      st.touch[v] = 0;
-      if (meta_offset != ~0ull) {
-        uint32_t* rec = reinterpret_cast<uint32_t*>(staging + meta_offset + j * kMetaBytes);
-        rec[0] = t;
-        rec[1] = le;
-        rec[2] = __float_as_uint(em);
-        rec[3] = __float_as_uint(de);
-        rec[4] = pr;
-        rec[5] = g.epoch_now;
-      }
-    }
-  }
-}
-
 static unsigned move_grid(uint64_t total_pieces) {
   uint64_t blocks = (total_pieces * 32 + kThreads - 1) / kThreads;
   if (blocks == 0) blocks = 1;
-  const uint64_t cap = (uint64_t)kSMs * 8;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
   return (unsigned)(blocks > cap ? cap : blocks);
 }
 
 static uint64_t pieces_per_entry(const PartGeom& g) {
   return (uint64_t)((g.chunk_bytes + kPieceBytes - 1) / kPieceBytes) * g.n_chunks;
-}
-
-cudaError_t launch_pack(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* victims,
-                        uint64_t count, uint64_t ring_start, uint8_t* staging, uint64_t meta_offset,
-                        const Workspace& ws, cudaStream_t s) {
-  if (count == 0) return cudaSuccess;
-  pack_kernel<<<move_grid(count * pieces_per_entry(g)), kThreads, 0, s>>>(
-      g, st, loc, victims, count, ring_start, staging, meta_offset, ws.status);
-  count_launches(1);
-  return cudaGetLastError();
-}
-
-__global__ void __launch_bounds__(kThreads)
-unpack_kernel(const PartGeom g, const EntryState st, uint32_t* __restrict__ loc,
-              const uint32_t* __restrict__ slots, const uint32_t* __restrict__ free_ids, uint64_t count,
-              const uint8_t* __restrict__ staging, uint32_t* __restrict__ status) {
-  const uint32_t lane = threadIdx.x & 31u;
-  const uint32_t ppc = (g.chunk_bytes + kPieceBytes - 1) / kPieceBytes;
-  const uint32_t ppe = ppc * g.n_chunks;
-  const uint64_t total = count * ppe;
-  const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
-  for (uint64_t piece = (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); piece < total;
-       piece += warps) {
-    const uint64_t j = piece / ppe;
-    const uint32_t r = (uint32_t)(piece - j * ppe);
-    const uint32_t c = r / ppc;
-    const uint32_t pp = r - c * ppc;
-    const uint32_t f = free_ids[j];
-    const uint32_t slot = slots[j];
-    if ((uint64_t)f < g.base || (uint64_t)f >= g.base + g.n || slot >= g.ring_slots) {
-      if (lane == 0) atomicOr(status, KV_DEV_BAD_INDEX);
-      continue;
-    }
-    const uint64_t local = (uint64_t)f - g.base;
-    const uint32_t in_chunk = pp * kPieceBytes;
-    const uint32_t len = min(kPieceBytes, g.chunk_bytes - in_chunk);
-    copy_piece(staging + j * (uint64_t)g.entry_bytes + (uint64_t)c * g.chunk_bytes + in_chunk,
-               g.slab + chunk_offset(g, local, c) + in_chunk, len, lane);
-    if (r == 0 && lane == 0) {
-      const uint32_t t = g.r_tag[slot];
-      if (t == KV_NONE || st.state[f] != KV_STATE_FREE) {
-        atomicOr(status, KV_DEV_BAD_INDEX);
-        continue;
-      }
-      st.pair[f] = g.r_pair[slot];
-      const float de = g.r_decay[slot];
-      float em = g.r_ema[slot];
-      if (g.lazy_decay && g.epoch_now > g.r_depoch[slot]) em = ema_catch_up(em, de, g.epoch_now - g.r_depoch[slot]);
-      st.ema[f] = em;
-      st.decay[f] = de;
-      st.last_epoch[f] = g.r_last_epoch[slot];
-      st.tag[f] = t;
-      st.touch[f] = 0;
-      st.state[f] = KV_STATE_RESIDENT;
-      loc[t] = f;
-      g.r_tag[slot] = KV_NONE;  // the host slot is dead
-    }
-  }
-}
-
-cudaError_t launch_unpack(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
-                          const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
-                          const Workspace& ws, cudaStream_t s) {
-  if (count == 0) return cudaSuccess;
-  unpack_kernel<<<move_grid(count * pieces_per_entry(g)), kThreads, 0, s>>>(
-      g, st, loc, slots, free_ids, count, staging, ws.status);
-  count_launches(1);
-  return cudaGetLastError();
 }
 
 // SplitMix64 output function (Steele, Lea, Flood: "Fast splittable pseudorandom
@@ -301,6 +147,7 @@ __global__ void init_scalars_kernel(uint64_t* hits, uint64_t* misses, float* P, 
     ws.sel->prefix = 0; ws.sel->tau = 0; ws.sel->k_rem = 0; ws.sel->need_eq = 0;
     ws.sel->bar_arrive = 0; ws.sel->bar_done = 0; ws.sel->update_ticket = 0; ws.sel->hint_last = 0;
     ws.sel->hint_valid = 0; ws.sel->hint_tau = 0; ws.sel->hint_n = 0; ws.sel->below = 0;
+    ws.sel->n_select = 0; ws.sel->n_hint_hit = 0; ws.sel->n_hint_miss = 0; ws.sel->n_reread = 0;
   }
 }
 
@@ -309,7 +156,7 @@ cudaError_t launch_init(const EntryState& st, uint64_t* hits, uint64_t* misses, 
                         const Workspace& ws, cudaStream_t s) {
   const uint64_t most = st.n > n_tags ? st.n : n_tags;
   uint64_t blocks = (most + kThreads - 1) / kThreads;
-  const uint64_t cap = (uint64_t)kSMs * 8;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   if (blocks == 0) blocks = 1;
   init_entries_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(st, loc, n_tags);

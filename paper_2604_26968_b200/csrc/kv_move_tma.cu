@@ -295,20 +295,23 @@ move_tma_kernel(const MoveArgs a) {
 }
 
 static unsigned tma_grid(uint64_t count) {
-  const uint64_t cap = (uint64_t)kSMs * kMoveCtasPerSm;
+  const uint64_t cap = (uint64_t)sm_count() * kMoveCtasPerSm;
   uint64_t blocks = count < cap ? count : cap;
   return (unsigned)(blocks ? blocks : 1);
 }
 
 template <bool PACK>
 static cudaError_t launch_move(const MoveArgs& a, cudaStream_t s) {
-  static bool configured = false;
+  // the opt-in for the shared memory belongs to a device: once per device ordinal
+  static std::atomic<bool> configured[64];
   const size_t smem = (size_t)kStages * kStageBytes;
-  if (!configured) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(move_tma_kernel<PACK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
   }
   move_tma_kernel<PACK><<<tma_grid(a.count), kMoveThreads, smem, s>>>(a);
   count_launches(1);

@@ -25,7 +25,7 @@ cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit,
   if (n_events == 0) return cudaSuccess;
   uint64_t blocks = (n_events / 4 + kThreads - 1) / kThreads;
   if (blocks == 0) blocks = 1;
-  const uint64_t cap = (uint64_t)kSMs * 4;  // measured: 4 blocks per SM beat 8 and 2
+  const uint64_t cap = (uint64_t)sm_count() * 4;  // measured: 4 blocks per SM beat 8 and 2
   if (blocks > cap) blocks = cap;
   event_reduce_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(ev_entry, ev_hit, n_events, st.pair, st.touch,
                                                             st.n, ws.delta, ws.status);
@@ -99,7 +99,7 @@ cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* 
                                 const ScoreOptions& opt, const HeadWeights& hw, cudaStream_t s) {
   uint64_t blocks = (st.n / 4 + kThreads - 1) / kThreads;
   if (blocks == 0) blocks = 1;
-  const uint64_t cap = (uint64_t)kSMs * 8;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   const Predictor pd{hits,       misses,    P,          alpha0, beta0, ws.delta, &ws.sel->update_ticket,
                      opt.policy, opt.kappa, opt.window, ws.blend};

@@ -334,22 +334,19 @@ __global__ void select_begin_kernel(SelectScalars* sel, unsigned long long k) {
   sel->need_eq = 0;
 }
 
-// 1 = one persistent cooperative launch (default), 0 = one launch per phase
-int g_select_variant = 1;
-
 static unsigned hist_grid(uint64_t n) {
   uint64_t blocks = (n / 4 + kThreads - 1) / kThreads;
   if (blocks == 0) blocks = 1;
-  const uint64_t cap = (uint64_t)kSMs * 8;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
   return (unsigned)(blocks > cap ? cap : blocks);
 }
 
 cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims, const Workspace& ws,
-                          cudaStream_t s) {
+                          cudaStream_t s, int variant, const PartCounts* pc) {
   if (k == 0 || st.n == 0) return cudaSuccess;
-  if (g_select_variant == 1) {
+  if (variant == 1) {
     bool used = false;
-    const cudaError_t e = launch_select_persistent(st, k, d_victims, ws, s, &used);
+    const cudaError_t e = launch_select_persistent(st, k, d_victims, ws, s, &used, nullptr, pc);
     if (e != cudaSuccess || used) return e;
   }
   const unsigned g = hist_grid(st.n);
@@ -368,6 +365,7 @@ cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims,
                                                     ws.tile_offsets, k, d_victims);
   select_check_kernel<<<1, 1, 0, s>>>(ws.tile_counts, ws.tile_offsets, n_tiles, ws.sel, k, ws.status);
   count_launches(11);
+  if (pc && pc->n_parts > 1) return launch_partition_counts(d_victims, k, *pc, s);
   return cudaGetLastError();
 }
 
@@ -385,31 +383,30 @@ cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uin
   return cudaGetLastError();
 }
 
-// counts[q] = number of victims with bases[q] <= id < bases[q+1]; victims ascending.
+// counts[q] = number of victims with base[q] <= id < base[q+1]; victims ascending.
 __global__ void partition_counts_kernel(const uint32_t* __restrict__ victims, unsigned long long m,
-                                        unsigned long long b0, unsigned long long b1,
-                                        unsigned long long b2, unsigned long long b3,
-                                        unsigned long long b4, int n_parts,
-                                        unsigned long long* __restrict__ counts) {
+                                        const PartCounts pc) {
   __shared__ unsigned long long s_lb[5];
-  const unsigned long long bases[5] = {b0, b1, b2, b3, b4};
   const int q = threadIdx.x;
-  if (q <= n_parts) {
-    unsigned long long lo = 0, hi = m;  // first index with victims[idx] >= bases[q]
+  if (q <= pc.n_parts) {
+    unsigned long long lo = 0, hi = m;  // first index with victims[idx] >= base[q]
     while (lo < hi) {
       const unsigned long long mid = (lo + hi) >> 1;
-      if ((unsigned long long)victims[mid] < bases[q]) lo = mid + 1; else hi = mid;
+      if ((unsigned long long)victims[mid] < pc.base[q]) lo = mid + 1; else hi = mid;
     }
     s_lb[q] = lo;
   }
   __syncthreads();
-  if (q < 4) counts[q] = (q < n_parts) ? s_lb[q + 1] - s_lb[q] : 0ull;
+  if (q < 4) {
+    const unsigned long long c = (q < pc.n_parts) ? s_lb[q + 1] - s_lb[q] : 0ull;
+    pc.d_counts[q] = c;
+    if (pc.h_counts) pc.h_counts[q] = c;
+  }
 }
 
-cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const uint64_t* bases5,
-                                    int n_parts, const Workspace& ws, cudaStream_t s) {
-  partition_counts_kernel<<<1, 32, 0, s>>>(d_victims, m, bases5[0], bases5[1], bases5[2], bases5[3],
-                                           bases5[4], n_parts, ws.part_counts);
+cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const PartCounts& pc,
+                                    cudaStream_t s) {
+  partition_counts_kernel<<<1, 32, 0, s>>>(d_victims, m, pc);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -9,18 +9,18 @@
 //   A  every score becomes an order-preserving key (fused form: the entry pass
 //      itself produces it) and enters the first histogram.  With a hint -- tau of
 //      the previous selection -- the histogram covers a bracket of 2^22 keys
-//      around it, and the pass also leaves in shared memory a bitmap "key below
-//      the bracket" and a list of the keys inside the bracket (index in the
-//      slice, bracket bin, low bits): typically 5-10 % of the slice.
+//      around it; the pass also leaves in shared memory a bitmap "key below the
+//      bracket", and every thread notes the keys it saw inside the bracket
+//      (typically 5-10 % of the slice) in a few private slots: no vote, no atomic.
 //   B  the remaining histograms of the radix select.  When rank k falls inside
 //      the bracket, ONE more histogram (the 2^11 single keys of the bracket bin
-//      that holds rank k) finishes it, and it is built from the list alone: no
-//      second pass over the scores.  Otherwise (no hint, a miss, a list that
-//      overflowed) the keys are re-read from the score array, which then sits
-//      mostly in L2; the last histogram of that path leaves the bitmaps "key
-//      below the final range" and "key inside the final range".
+//      that holds rank k) finishes it, and it is built from the noted keys alone:
+//      no second pass over the scores.  Otherwise (no hint, a miss, a thread that
+//      ran out of slots) the keys are re-read from the score array, which then
+//      sits mostly in L2, and the last histogram of that path leaves the bitmaps
+//      "key below the final range" and "key inside the final range".
 //   C  tau picked: the keys of the final range are sorted into "below tau" and
-//      "equal to tau" -- from the list, or, on the other path, by fetching just
+//      "equal to tau" -- from the notes, or, on the other path, by fetching just
 //      the keys inside the range (not even those when the CTA's own histogram
 //      shows that all of them equal tau: a tie, the usual case when few distinct
 //      scores exist).
@@ -57,9 +57,8 @@ constexpr uint32_t kBracketHalf = 1u << 21;             // ... and the 2,048 bin
 constexpr uint32_t kBracketBits = 22;                   // log2 of the bracket's width in keys
 constexpr uint32_t kPIdxBits = 18;                      // index of an entry inside its slice
 constexpr uint32_t kPMaxSlice = 1u << kPIdxBits;        // entries per CTA the bitmaps are sized for (2 x 32 KB)
-constexpr uint32_t kPListCapMax = 16384;                // bracket keys remembered per CTA (6 bytes each)
+constexpr uint32_t kPSlotsMax = 32;                     // bracket keys a thread can note (its private slots)
 
-static_assert(kPIdxBits + kBracketBits - kBracketShift <= 32, "index and bracket bin share one word");
 
 __device__ __forceinline__ uint32_t p_score_key(float s) {
   uint32_t b = __float_as_uint(s);
@@ -112,7 +111,8 @@ struct PArgs {
   uint32_t* status;
   unsigned long long per; // entries per CTA slice (multiple of 4, at most kPMaxSlice)
   uint32_t words;         // 32-bit words of one bitmap of a slice (a multiple of 4)
-  uint32_t list_cap;      // entries of the bracket list (a multiple of 8)
+  uint32_t slots;         // private slots per thread for keys inside the bracket (at least 10)
+  PartCounts pc;          // partitions of the pool (the victims per partition are a by-product)
   // the scoring pass of the fused form
   EntryState st;
   Predictor pd;
@@ -198,12 +198,12 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   extern __shared__ __align__(16) uint32_t s_dyn[];
   uint32_t* const s_bit_l = s_dyn;                    // bit j: key of local entry j is below tau
   uint32_t* const s_bit_e = s_bit_l + a.words;        // bit j: key of local entry j equals tau
-  uint32_t* const s_list_jb = s_bit_e + a.words;      // bracket list: index in slice | bracket bin << kPIdxBits
-  uint16_t* const s_list_low = reinterpret_cast<uint16_t*>(s_list_jb + a.list_cap);  // ... and key bits below the bin
+  // [slot][thread]: (key - base0) | position in the vector << 22 | chunk << 24; later the
+  // staging buffer of the ordered write
+  uint32_t* const s_note = s_bit_e + a.words;
   __shared__ uint32_t s_hist[kPHistBins];
   __shared__ uint32_t s_warp[32];
   __shared__ uint32_t s_pick[2];
-  __shared__ uint32_t s_list_n;
   __shared__ float sP[16];
   const uint32_t t = threadIdx.x;
   const uint32_t lane = t & 31u;
@@ -281,6 +281,62 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       c -= nb;
     }
   };
+  // The same pass for the re-reads of phase B, where the threads' notes are dead: their
+  // space becomes a ring of stages that asynchronous copies (global -> shared, no registers
+  // in between) keep filled several chunks ahead.  A thread reads back only what it copied
+  // itself, so waiting for its own copy groups is all the synchronisation there is.
+  auto for_chunks_staged = [&](auto body) {
+    constexpr uint32_t kStageWords = kPChunk + kPThreads;   // 4096 scores + 1024 state words
+    const uint32_t n_stages = (a.slots * kPThreads) / kStageWords;   // at least 2 (slots >= 10)
+    const uint32_t depth = n_stages < 8u ? n_stages : 8u;
+    auto issue = [&](uint32_t c, uint32_t stage) {
+      const uint32_t j0 = c * kPChunk + 4u * t;
+      if (j0 + 4 <= len) {
+        uint32_t* dst = s_note + stage * kStageWords;
+        const uint32_t d_sc = (uint32_t)__cvta_generic_to_shared(dst + 4u * t);
+        const uint32_t d_st = (uint32_t)__cvta_generic_to_shared(dst + kPChunk + t);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d_sc), "l"(a.score + s0 + j0) : "memory");
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d_st), "l"(a.state + s0 + j0) : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    // chunks go last to first; chunk number n_chunks-1-i uses stage i % depth
+    for (uint32_t i = 0; i < depth; ++i) {
+      if (i < n_chunks) issue(n_chunks - 1u - i, i);
+      else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (uint32_t i = 0; i < n_chunks; ++i) {
+      // all but the newest depth-1 groups are complete: the oldest one is chunk i's
+      switch (depth) {
+        case 2: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+        case 5: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+        case 6: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+        case 7: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+      }
+      const uint32_t c = n_chunks - 1u - i, stage = i % depth;
+      const uint32_t j0 = c * kPChunk + 4u * t;
+      uint32_t key[4];
+      if (j0 + 4 <= len) {
+        const uint32_t* src = s_note + stage * kStageWords;
+        const float4 sc = *reinterpret_cast<const float4*>(src + 4u * t);
+        const uint32_t st4 = src[kPChunk + t];
+        key[0] = (st4 & 0xFFu) == KV_STATE_RESIDENT ? p_score_key(sc.x) : kExcluded;
+        key[1] = ((st4 >> 8) & 0xFFu) == KV_STATE_RESIDENT ? p_score_key(sc.y) : kExcluded;
+        key[2] = ((st4 >> 16) & 0xFFu) == KV_STATE_RESIDENT ? p_score_key(sc.z) : kExcluded;
+        key[3] = (st4 >> 24) == KV_STATE_RESIDENT ? p_score_key(sc.w) : kExcluded;
+      } else {
+        keys_from_arrays(c, key);   // the ragged end of the slice
+      }
+      // refill the stage with the chunk `depth` further on (an empty group keeps the count)
+      if (i + depth < n_chunks) issue(n_chunks - 1u - (i + depth), stage);
+      else asm volatile("cp.async.commit_group;" ::: "memory");
+      body(c, key);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  };
   // Eight lanes x four bits (a lane holds 4 consecutive entries) -> the bitmap word of
   // the 32 entries starting at j0 of the lane with (lane & 7) == 0, which stores it.
   auto store_word = [&](uint32_t* bits, uint32_t nib, uint32_t j0) {
@@ -316,52 +372,39 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     }
   }
   for (uint32_t w = t; w < 2 * a.words; w += kPThreads) s_bit_l[w] = 0;   // both bitmaps
-  if (t == 0) s_list_n = 0;
 
   // ---- phase A: keys and the first histogram ----
   // Without a hint the first histogram is digit 0 of a plain radix select (bits
   // 31..21 of every key).  With a hint it covers only the bracket [base0, base0 +
   // 2^22) around the hinted tau in 2,048 bins of 2^11 keys; keys below base0 set
-  // their bit in s_bit_l (and are counted), keys inside go on the list: scores
-  // move little from one epoch to the next, so the k-th key is almost always
-  // inside, and then nothing but the list is looked at again.
+  // their bit in s_bit_l (and are counted), keys inside are noted: scores move
+  // little from one epoch to the next, so the k-th key is almost always inside,
+  // and then only the notes are looked at again.
   const bool hint = a.sel->hint_valid != 0 && a.sel->hint_n == a.n;
   const uint32_t hint_tau = a.sel->hint_tau;
   const uint32_t base0 = hint ? (hint_tau > kBracketHalf ? hint_tau - kBracketHalf : 0u) : 0u;
   const uint32_t shift0 = hint ? kBracketShift : 21u;
   WarpHist wh;
+  uint32_t n_noted = 0;   // keys of this thread inside the bracket (noted while slots last)
   auto phase_a = [&](uint32_t c, const uint32_t key[4]) {
     if (!hint) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) wh.add(s_hist, key[q] != kExcluded, key[q] >> 21);
       return;
     }
-    const uint32_t j0 = c * kPChunk + 4u * t;
-    uint32_t nib = 0, d[4], m[4], total = 0;
-    bool in[4];
+    uint32_t nib_l = 0;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      d[q] = key[q] - base0;
-      nib |= (uint32_t)(key[q] < base0) << q;   // (an excluded key is 0xFFFFFFFF: never below)
-      in[q] = key[q] != kExcluded && key[q] >= base0 && (d[q] >> kBracketBits) == 0u;
-      m[q] = __ballot_sync(0xFFFFFFFFu, in[q]);
-      total += (uint32_t)__popc(m[q]);
-    }
-    store_word(s_bit_l, nib, j0);
-    if (total == 0) return;   // (uniform over the warp)
-    uint32_t at = 0;
-    if (lane == 0) at = atomicAdd(&s_list_n, total);
-    at = __shfl_sync(0xFFFFFFFFu, at, 0);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      wh.add_voted(s_hist, m[q], in[q], d[q] >> kBracketShift);
-      const uint32_t pos = at + (uint32_t)__popc(m[q] & ((1u << lane) - 1u));
-      if (in[q] && pos < a.list_cap) {
-        s_list_jb[pos] = (j0 + q) | ((d[q] >> kBracketShift) << kPIdxBits);
-        s_list_low[pos] = (uint16_t)(d[q] & ((1u << kBracketShift) - 1u));
+      const uint32_t d = key[q] - base0;
+      const bool below = key[q] < base0;   // (an excluded key is 0xFFFFFFFF: never below)
+      nib_l |= (uint32_t)below << q;
+      if (!below && (d >> kBracketBits) == 0u && key[q] != kExcluded) {
+        atomicAdd(&s_hist[d >> kBracketShift], 1u);
+        if (n_noted < a.slots) s_note[n_noted * kPThreads + t] = d | ((uint32_t)q << 22) | (c << 24);
+        ++n_noted;
       }
-      at += (uint32_t)__popc(m[q]);
     }
+    store_word(s_bit_l, nib_l, c * kPChunk + 4u * t);
   };
   clear_hist();
   if constexpr (FUSED) {
@@ -409,6 +452,9 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     (void)block_scan_excl(below, s_warp, cta_below0);
     if (t == 0 && cta_below0) atomicAdd(&a.sel->below, (unsigned long long)cta_below0);
   }
+  // a thread that ran out of slots sends the whole CTA the long way (its keys are re-read)
+  const bool notes_complete = __syncthreads_or(n_noted > a.slots) == 0;
+  if (n_noted > a.slots) n_noted = a.slots;
   stamp(1);
   ok = grid_barrier(bar, G);
   stamp(2);
@@ -427,15 +473,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     uint32_t bin, before;
     bool found = true;
     bool clear_below = hint;
-    bool use_list = false;   // rank k is inside the bracket and this CTA's list holds all its bracket keys
-    const uint32_t n_list = s_list_n;
+    bool use_notes = false;   // rank k is inside the hint's bracket and this CTA noted all its bracket keys
     auto hist_pass = [&](uint32_t width_log2, uint32_t new_shift, uint32_t h_new) {
       // histogram of ((key - base) >> new_shift) over the keys in [base, base + 2^width_log2)
       clear_hist();
       const uint32_t top = width_log2 - new_shift;  // log2 of the number of bins
       WarpHist w2;
       if (new_shift != 0) {
-        for_chunks([&](uint32_t, const uint32_t key[4]) {
+        for_chunks_staged([&](uint32_t, const uint32_t key[4]) {
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const uint32_t d = key[q] - base;
@@ -443,27 +488,44 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
                    d >> new_shift);
           }
         });
-      } else if (use_list) {
+      } else if (use_notes) {
         // the last histogram (single keys of the bracket bin that holds rank k) from the
-        // list; listed keys of earlier bins are below the range: their bit joins s_bit_l
+        // notes; noted keys of earlier bins are below the final range: their bit joins s_bit_l
         const uint32_t bin_k = (base - base0) >> kBracketShift;
-        const uint32_t iters = (n_list + kPThreads - 1) / kPThreads;
-        for (uint32_t i = 0; i < iters; ++i) {
-          const uint32_t e = i * kPThreads + t;
-          uint32_t b = 0xFFFFFFFFu, j = 0, low = 0;
-          if (e < n_list) {
-            const uint32_t v = s_list_jb[e];
-            b = v >> kPIdxBits;
-            j = v & (kPMaxSlice - 1u);
-            low = s_list_low[e];
+        uint32_t p_bin = 0, p_cnt = 0;   // the thread's pending count for one key value
+        for (uint32_t i = 0; i < n_noted; ++i) {
+          const uint32_t v = s_note[i * kPThreads + t];
+          const uint32_t d = v & ((1u << kBracketBits) - 1u), b = d >> kBracketShift;
+          if (b < bin_k) {
+            const uint32_t j = (v >> 24) * kPChunk + 4u * t + ((v >> 22) & 3u);
+            atomicOr(&s_bit_l[j >> 5], 1u << (j & 31u));
+          } else if (b == bin_k) {
+            const uint32_t low = d & ((1u << kBracketShift) - 1u);
+            if (low != p_bin) {
+              if (p_cnt) atomicAdd(&s_hist[p_bin], p_cnt);
+              p_bin = low;
+              p_cnt = 0;
+            }
+            ++p_cnt;
           }
-          if (b < bin_k) atomicOr(&s_bit_l[j >> 5], 1u << (j & 31u));
-          w2.add(s_hist, b == bin_k, low);
+        }
+        // pending counts: one atomic per key value and warp
+        for (;;) {
+          const unsigned m = __ballot_sync(0xFFFFFFFFu, p_cnt != 0u);
+          if (m == 0) break;
+          const int leader = __ffs(m) - 1;
+          const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, p_bin, leader);
+          const bool mine = p_cnt != 0u && p_bin == b0;
+          uint32_t sum = mine ? p_cnt : 0u;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+          if ((int)lane == leader) atomicAdd(&s_hist[b0], sum);
+          if (mine) p_cnt = 0;
         }
       } else {
         // the last histogram (single keys) from the arrays; it also leaves the bitmaps "key
         // below the range" in s_bit_l and "key inside the range" in s_bit_e
-        for_chunks([&](uint32_t c, const uint32_t key[4]) {
+        for_chunks_staged([&](uint32_t c, const uint32_t key[4]) {
           uint32_t nl = 0, ne = 0;
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -493,9 +555,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       pick_bin(a.hist, kPHistBins, above ? a.k - below : 1ull, s_warp, s_pick, bin, before);
       if (above && bin != 0xFFFFFFFFu) {
         k_rem = a.k - below;
-        use_list = n_list <= a.list_cap;
+        use_notes = notes_complete;
+        if (t == 0) {
+          if (blockIdx.x == 0) atomicAdd(&a.sel->n_hint_hit, 1u);
+          if (!notes_complete) atomicAdd(&a.sel->n_reread, 1u);
+        }
       } else {
         // rank k is outside the bracket: digit 0 of the plain radix select
+        if (blockIdx.x == 0 && t == 0) atomicAdd(&a.sel->n_hint_miss, 1u);
         base = 0;
         shift = 21;
         hist_pass(32, 21, 1);
@@ -532,12 +599,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     const uint32_t tau = base + tau_low;
     const unsigned long long need_eq = k_rem;
     uint32_t c_l = 0, c_e = 0;
-    if (use_list) {
+    if (use_notes) {
       const uint32_t bin_k = (base - base0) >> kBracketShift;
-      for (uint32_t e = t; e < n_list; e += kPThreads) {
-        const uint32_t v = s_list_jb[e];
-        if ((v >> kPIdxBits) != bin_k) continue;
-        const uint32_t j = v & (kPMaxSlice - 1u), low = s_list_low[e];
+      for (uint32_t i = 0; i < n_noted; ++i) {
+        const uint32_t v = s_note[i * kPThreads + t];
+        const uint32_t d = v & ((1u << kBracketBits) - 1u);
+        if ((d >> kBracketShift) != bin_k) continue;
+        const uint32_t low = d & ((1u << kBracketShift) - 1u);
+        const uint32_t j = (v >> 24) * kPChunk + 4u * t + ((v >> 22) & 3u);
         if (low < tau_low) atomicOr(&s_bit_l[j >> 5], 1u << (j & 31u));
         else if (low == tau_low) atomicOr(&s_bit_e[j >> 5], 1u << (j & 31u));
       }
@@ -577,6 +646,21 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     const uint32_t ex_l = block_scan_excl(c_l, s_warp, tot_l);
     const uint32_t ex_e = block_scan_excl(c_e, s_warp, tot_e);
     if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(tot_l, tot_e);
+    // a partition boundary inside this slice: how many of the slice's marked entries lie before it
+    for (int q = 1; q < a.pc.n_parts; ++q) {   // (the condition is the same for the whole CTA)
+      if (a.pc.base[q] <= s0 || a.pc.base[q] >= s1) continue;
+      const uint32_t jb = (uint32_t)(a.pc.base[q] - s0);   // first local entry of partition q
+      uint32_t bl = 0, be = 0;
+      for (uint32_t w = t; w <= (jb >> 5) && w < a.words; w += kPThreads) {
+        const uint32_t m = w < (jb >> 5) ? 0xFFFFFFFFu : ((1u << (jb & 31u)) - 1u);
+        bl += (uint32_t)__popc(s_bit_l[w] & m);
+        be += (uint32_t)__popc(s_bit_e[w] & m);
+      }
+      uint32_t sl, se;
+      (void)block_scan_excl(bl, s_warp, sl);
+      (void)block_scan_excl(be, s_warp, se);
+      if (t == 0) a.sel->bsplit[q - 1] = make_uint2(sl, se);
+    }
     stamp(5);
     ok = grid_barrier(bar, ++nbar * G);
     stamp(6);
@@ -599,27 +683,64 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     if (found) {
       // Position of a victim.  With L entries below tau and E entries equal to tau before it
       // in id order, an entry below tau goes to L + min(E, need_eq) and an entry equal to tau,
-      // taken while E < need_eq, to L + E.
-      unsigned long long n_l = less_before + ex_l, n_e = eq_before + ex_e;
-      for (uint32_t w = w0; w < w1; ++w) {
-        const uint32_t bl = s_bit_l[w], be = s_bit_e[w];
-        uint32_t bits = bl | be;
-        while (bits) {
-          const uint32_t b = (uint32_t)__ffs(bits) - 1u;
-          bits &= bits - 1u;
-          const unsigned long long id = s0 + 32ull * w + b;
-          if ((bl >> b) & 1u) {
-            const unsigned long long pos = n_l + (n_e < need_eq ? n_e : need_eq);
-            if (pos < a.k) a.victims[pos] = (uint32_t)id;
-            ++n_l;
-          } else {
-            if (n_e < need_eq) {
-              const unsigned long long pos = n_l + n_e;
-              if (pos < a.k) a.victims[pos] = (uint32_t)id;
+      // taken while E < need_eq, to L + E.  The CTA's victims form one contiguous piece of the
+      // output, starting at p0.  Every thread walks the set bits of its own words and puts the
+      // ids in order in shared memory (the notes' space, free by now), from where they leave
+      // as full-line stores, a stage-full per round.
+      const unsigned long long eq_taken_before = eq_before < need_eq ? eq_before : need_eq;
+      const unsigned long long p0 = less_before + eq_taken_before;
+      const unsigned long long eq_room64 = need_eq - eq_taken_before;
+      const uint32_t eq_room = eq_room64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)eq_room64;
+      const uint32_t cta_total = tot_l + (tot_e < eq_room ? tot_e : eq_room);
+      uint32_t* const s_stage = s_note;
+      const uint32_t stage_cap = a.slots * kPThreads;
+      // the thread's own victims are the consecutive positions [p_first, p_first + p_count)
+      const uint32_t e0 = ex_e < eq_room ? ex_e : eq_room;
+      const uint32_t e1 = ex_e + c_e < eq_room ? ex_e + c_e : eq_room;
+      const uint32_t p_first = ex_l + e0, p_count = c_l + (e1 - e0);
+      const uint32_t id_base = (uint32_t)s0;   // (ids fit 32 bits)
+      __syncthreads();   // every thread is done with the notes
+      for (uint32_t r0 = 0; r0 < cta_total; r0 += stage_cap) {
+        if (p_count != 0 && p_first < r0 + stage_cap && p_first + p_count > r0) {
+          uint32_t n_l = ex_l, n_e = ex_e;   // counts inside the CTA before the current word
+          for (uint32_t w = w0; w < w1; ++w) {
+            const uint32_t bl = s_bit_l[w], be = s_bit_e[w];
+            const uint32_t id0 = id_base + 32u * w;
+            if (be == 0u) {
+              // no entry at tau in this word: its victims take consecutive positions
+              uint32_t pos = n_l + (n_e < eq_room ? n_e : eq_room) - r0;   // (wraps below r0: skipped)
+              uint32_t bits = bl;
+              while (bits) {
+                const uint32_t b = (uint32_t)__ffs(bits) - 1u;
+                bits &= bits - 1u;
+                if (pos < stage_cap) s_stage[pos] = id0 + b;
+                ++pos;
+              }
+              n_l += (uint32_t)__popc(bl);
+              continue;
             }
-            ++n_e;
+            uint32_t bits = bl | be;
+            while (bits) {
+              const uint32_t b = (uint32_t)__ffs(bits) - 1u;
+              bits &= bits - 1u;
+              uint32_t pos = 0xFFFFFFFFu;
+              if ((bl >> b) & 1u) {
+                pos = n_l + (n_e < eq_room ? n_e : eq_room);
+                ++n_l;
+              } else {
+                if (n_e < eq_room) pos = n_l + n_e;
+                ++n_e;
+              }
+              if (pos >= r0 && pos - r0 < stage_cap) s_stage[pos - r0] = id0 + b;
+            }
           }
         }
+        __syncthreads();
+        stamp(4);
+        const uint32_t n_out = cta_total - r0 < stage_cap ? cta_total - r0 : stage_cap;
+        for (uint32_t i = t; i < n_out; i += kPThreads)
+          if (p0 + r0 + i < a.k) a.victims[p0 + r0 + i] = s_stage[i];
+        __syncthreads();
       }
     }
     if (blockIdx.x == G - 1 && t == 0) {
@@ -628,8 +749,30 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       for (uint32_t g = 0; g < G; ++g) { const uint2 cc = __ldcg(&a.cta_counts[g]); tl += cc.x; te += cc.y; }
       const unsigned long long got = tl + (te < need_eq ? te : need_eq);
       if (!found || got != a.k) atomicOr(a.status, KV_DEV_SELECT_MISMATCH);
+      if (a.pc.n_parts > 1 && a.pc.d_counts) {
+        // victims before each partition boundary = entries below tau before it + the taken
+        // ones among the entries equal to tau before it
+        unsigned long long before[5] = {0, 0, 0, 0, 0};
+        for (int q = 1; q <= a.pc.n_parts; ++q) {
+          if (q == a.pc.n_parts || a.pc.base[q] >= a.n) { before[q] = got; continue; }
+          const uint32_t cb = (uint32_t)(a.pc.base[q] / a.per);          // the CTA whose slice holds the boundary
+          unsigned long long l = 0, e = 0;
+          for (uint32_t g = 0; g < cb && g < G; ++g) { const uint2 cc = __ldcg(&a.cta_counts[g]); l += cc.x; e += cc.y; }
+          if (a.pc.base[q] > (unsigned long long)cb * a.per) {            // strictly inside that slice
+            const uint2 sp = __ldcg(&a.sel->bsplit[q - 1]);
+            l += sp.x; e += sp.y;
+          }
+          before[q] = l + (e < need_eq ? e : need_eq);
+        }
+        for (int q = 0; q < 4; ++q) {
+          const unsigned long long c = q < a.pc.n_parts ? before[q + 1] - before[q] : 0ull;
+          a.pc.d_counts[q] = c;
+          if (a.pc.h_counts) a.pc.h_counts[q] = c;
+        }
+      }
       a.sel->tau = tau;
       a.sel->need_eq = need_eq;
+      a.sel->n_select += 1;
       // hint for the next selection over the same keys: this tau moved on by as much as it
       // moved since the selection before (while a pool warms up its scores grow epoch after
       // epoch, and the trend is a better centre for the bracket than the last value)
@@ -675,9 +818,10 @@ constexpr int kPMaxDevices = 64;
 std::mutex g_persist_mutex;
 PersistDevice g_persist[kPMaxDevices];
 
-// Dynamic shared memory of a launch: two bitmaps and the bracket list.
-inline size_t persist_smem(uint32_t words, uint32_t list_cap) {
-  return (size_t)words * 8u + (size_t)list_cap * 6u;
+// Dynamic shared memory of a launch: two bitmaps and the threads' private slots (which the
+// ordered write reuses as its staging buffer).
+inline size_t persist_smem(uint32_t words, uint32_t slots) {
+  return (size_t)words * 8u + (size_t)slots * kPThreads * 4u;
 }
 }  // namespace
 
@@ -685,7 +829,8 @@ inline size_t persist_smem(uint32_t words, uint32_t list_cap) {
 // if the device can hold one CTA per SM of it co-resident and the slices fit the
 // bitmaps; *used = false (and nothing launched) otherwise.
 cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
-                                     const Workspace& ws, cudaStream_t s, bool* used, const FusedScore* fs) {
+                                     const Workspace& ws, cudaStream_t s, bool* used, const FusedScore* fs,
+                                     const PartCounts* pc) {
   *used = false;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return cudaGetLastError();
@@ -703,8 +848,8 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
       cudaError_t e = cudaFuncGetAttributes(&fa, select_persistent_kernel<false>);
       if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, select_persistent_kernel<true>);
       const size_t fixed = fa.sharedSizeBytes > fb.sharedSizeBytes ? fa.sharedSizeBytes : fb.sharedSizeBytes;
-      // the most a launch asks for: the largest bitmaps and the longest list
-      const size_t want = persist_smem(kPMaxSlice / 32, kPListCapMax);
+      // the most a launch asks for: the largest bitmaps and the most slots
+      const size_t want = persist_smem(kPMaxSlice / 32, kPSlotsMax);
       if ((size_t)optin < fixed + want) e = cudaErrorInvalidValue;
       d.smem_max = want;
       if (e == cudaSuccess)
@@ -744,16 +889,18 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   a.per = ((st.n + G - 1) / G + 3) / 4 * 4;
   if (a.per > kPMaxSlice) return cudaSuccess;  // slices beyond the bitmaps: the multi-launch selection runs
   a.words = (uint32_t)((a.per + 31) / 32 + 3) / 4 * 4;
-  // The list holds the keys inside the hint's bracket, typically 5-10 % of a slice; a CTA whose
-  // list overflows re-reads its keys instead.  What this kernel does not take of the shared
-  // memory stays with the L1, whose lines hold the loads in flight of the streaming entry pass.
-  uint64_t list_cap = (a.per / 4 + 7) / 8 * 8;
-  if (const char* e = std::getenv("KVTIER_SELECT_LIST")) list_cap = (uint64_t)std::atoi(e) / 8 * 8;
-  if (list_cap < 8) list_cap = 8;
-  if (list_cap > kPListCapMax) list_cap = kPListCapMax;
-  a.list_cap = (uint32_t)list_cap;
-  const size_t smem = persist_smem(a.words, a.list_cap);
+  // The hint's bracket typically holds 5-10 % of a slice's keys, but slices differ (blocks of one
+  // history sit together), and a thread that runs out of slots sends its CTA the long way.  What this kernel does not take
+  // of the shared memory stays with the L1, whose lines hold the loads in flight of the streaming
+  // entry pass.
+  uint64_t slots = (a.per + kPThreads - 1) / kPThreads;   // as many as the thread sees keys, up to the maximum
+  if (const char* e = std::getenv("KVTIER_SELECT_SLOTS")) slots = (uint64_t)std::atoi(e);
+  if (slots < 10) slots = 10;   // (two stages of the re-reading passes fit)
+  if (slots > kPSlotsMax) slots = kPSlotsMax;
+  a.slots = (uint32_t)slots;
+  const size_t smem = persist_smem(a.words, a.slots);
   if (smem > pd.smem_max) return cudaSuccess;
+  a.pc = pc ? *pc : PartCounts{};
   a.st = st;
   a.pd = Predictor{};
   a.hw = HeadWeights{};

@@ -14,8 +14,6 @@ using namespace kvt;
 namespace kvt {
 std::atomic<uint64_t> g_kernel_launches{0};
 }
-// which pack/unpack kernels run: 1 = bulk-copy engine (default), 0 = register path
-static int g_move_variant = 1;
 
 namespace {
 
@@ -100,6 +98,9 @@ struct kv_pool {
   int demote_turn = 0, promote_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
   ScoreOptions score_opt;   // eviction policy and confidence blend
+  int select_variant = 1;   // 1 = persistent cooperative selection, 0 = one launch per phase
+  PartCounts pc;            // partition bases and where selections leave the victims per partition
+  uint32_t* h_sel_stats = nullptr;
   HeadWeights head{};       // head-granular importance matrices and weights
   uint32_t n_head_imp = 0, n_head_w = 0;
   // a demotion whose later chunks are not enqueued yet (deferred packing)
@@ -129,7 +130,7 @@ struct Layout {
   uint64_t delta, hist, sel, status, blend, block_score, block_state, block_victims, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
   uint64_t ring[4][6];
   uint64_t dev_total;
-  uint64_t h_list[2], h_counts, h_status, host_total;
+  uint64_t h_list[2], h_counts, h_status, h_sel_stats, host_total;
   uint32_t n_tiles;
 };
 
@@ -220,6 +221,7 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
   L->h_list[1] = htake(d->max_promote * 4);
   L->h_counts = htake(4 * 8);
   L->h_status = htake(4);
+  L->h_sel_stats = htake(16);
   L->host_total = h;
 }
 
@@ -235,6 +237,22 @@ int32_t cuda_fail(kv_pool* p, cudaError_t e) {
     cudaError_t e__ = (call);                        \
     if (e__ != cudaSuccess) return cuda_fail(pool, e__); \
   } while (0)
+
+// On a pool of several partitions every selection leaves the victims per partition in the
+// pinned host workspace (kv_victim_counts): the kernels write them there themselves where
+// the device can address that memory, else a 32-byte copy follows them.
+int32_t counts_to_host(kv_pool* p, cudaStream_t s) {
+  if (p->n_parts == 1 || p->pc.h_counts) return KV_OK;
+  const cudaError_t e = cudaMemcpyAsync(p->h_counts, p->ws.part_counts, 4 * sizeof(uint64_t), cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) { p->last_cuda_error = (int)e; return KV_ERR_CUDA; }
+  return KV_OK;
+}
+
+// A scoring pass has been enqueued.
+void scoring_pass_enqueued(kv_pool* p, uint32_t epoch) {
+  p->stats.epochs += 1;
+  for (int q = 0; q < p->n_parts; ++q) p->geom[q].epoch_now = epoch;
+}
 
 void timing_settle(kv_pool* p, kv_pool::Timed& t) {
   if (!t.pending) return;
@@ -294,12 +312,8 @@ int32_t enqueue_pack_chunk(kv_pool* p, int q, uint64_t c0, uint64_t cnt) {
   const uint32_t* victims = pd.victims + pd.off[q] + c0;
   {
     TimedScope ts(p, 0, cnt * eb, compute);
-    if (g_move_variant)
-      KV_CUDA(p, launch_pack_tma(g, p->st, p->desc.d_loc, victims, cnt, slot0, p->staging[b], meta_off, p->ws,
-                                 compute, pd.meta_done ? 2u : 0u));
-    else
-      KV_CUDA(p, launch_pack(g, p->st, p->desc.d_loc, victims, cnt, slot0, p->staging[b], meta_off, p->ws,
-                             compute));
+    KV_CUDA(p, launch_pack_tma(g, p->st, p->desc.d_loc, victims, cnt, slot0, p->staging[b], meta_off, p->ws,
+                               compute, pd.meta_done ? 2u : 0u));
   }
   KV_CUDA(p, cudaEventRecord(p->ev_ready[b], compute));
   KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_ready[b], 0));
@@ -462,8 +476,20 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
   p->h_list[1] = reinterpret_cast<uint32_t*>(hw + L.h_list[1]);
   p->h_counts = reinterpret_cast<uint64_t*>(hw + L.h_counts);
   p->h_status = reinterpret_cast<uint32_t*>(hw + L.h_status);
+  for (int q = 0; q <= 4; ++q) p->pc.base[q] = g.bases[q];
+  p->pc.n_parts = g.n_parts;
+  p->pc.d_counts = p->ws.part_counts;
+  {
+    // kernels write the counts straight into the pinned host workspace where the device can address it
+    void* dp = nullptr;
+    if (cudaHostGetDevicePointer(&dp, p->h_counts, 0) == cudaSuccess) p->pc.h_counts = static_cast<unsigned long long*>(dp);
+    else (void)cudaGetLastError();
+    for (int q = 0; q < 4; ++q) p->h_counts[q] = 0;
+  }
+  p->h_sel_stats = reinterpret_cast<uint32_t*>(hw + L.h_sel_stats);
   p->st = EntryState{desc->d_ema, desc->d_decay, desc->d_touch, desc->d_last_epoch, desc->d_pair,
                      desc->d_state, desc->d_tag, desc->d_score, g.N};
+
   for (int q = 0; q < g.n_parts; ++q) {
     PartGeom& pg = p->geom[q];
     pg.slab = static_cast<uint8_t*>(desc->part[q].d_slab);
@@ -607,8 +633,7 @@ int32_t kv_epoch_update(kv_pool* p, uint32_t epoch, kv_stream_t stream) {
   KV_DRAIN_ALL(p);
   KV_CUDA(p, launch_entry_update(p->st, p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
                                  p->desc.beta0, p->ws, epoch, p->score_opt, p->head, S(stream)));
-  p->stats.epochs += 1;
-  for (int q = 0; q < p->n_parts; ++q) p->geom[q].epoch_now = epoch;
+  scoring_pass_enqueued(p, epoch);
   return KV_OK;
 }
 
@@ -650,8 +675,8 @@ int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream
   if (k > p->stats.n_entries - p->stats.n_free) return KV_ERR_K_TOO_LARGE;
   if (k == 0) return KV_OK;
   if (!d_victims || !aligned16(d_victims)) return KV_ERR_INVALID_ARG;
-  KV_CUDA(p, launch_select(p->st, k, d_victims, p->ws, S(stream)));
-  return KV_OK;
+  KV_CUDA(p, launch_select(p->st, k, d_victims, p->ws, S(stream), p->select_variant, &p->pc));
+  return counts_to_host(p, S(stream));
 }
 
 int32_t kv_epoch_score_select(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_entry,
@@ -666,15 +691,14 @@ int32_t kv_epoch_score_select(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_e
   KV_CUDA(p, launch_event_reduce(d_ev_entry, d_ev_hit, n_events, p->st, p->ws, S(stream)));
   p->stats.events += n_events;
   bool used = false;
-  if (k > 0 && g_select_variant != 0) {
+  if (k > 0 && p->select_variant != 0) {
     const FusedScore fs{p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
                         p->desc.beta0,  epoch,            p->score_opt,  p->head};
-    KV_CUDA(p, launch_select_persistent(p->st, k, d_victims, p->ws, S(stream), &used, &fs));
+    KV_CUDA(p, launch_select_persistent(p->st, k, d_victims, p->ws, S(stream), &used, &fs, &p->pc));
   }
   if (used) {
-    p->stats.epochs += 1;
-    for (int q = 0; q < p->n_parts; ++q) p->geom[q].epoch_now = epoch;
-    return KV_OK;
+    scoring_pass_enqueued(p, epoch);
+    return counts_to_host(p, S(stream));
   }
   const int32_t rc = kv_epoch_update(p, epoch, stream);
   if (rc != KV_OK || k == 0) return rc;
@@ -689,21 +713,31 @@ int32_t kv_select_victim_blocks(kv_pool* p, uint64_t k_blocks, uint32_t* d_victi
   if (k_blocks > p->bgeom.block_base[p->n_parts]) return KV_ERR_K_TOO_LARGE;
   if (k_blocks == 0) return KV_OK;
   if (!d_victims || !aligned16(d_victims)) return KV_ERR_INVALID_ARG;
-  KV_CUDA(p, launch_select_blocks(p->st, p->bgeom, k_blocks, d_victims, p->ws, S(stream)));
-  uint64_t m = 0;
+  KV_CUDA(p, launch_select_blocks(p->st, p->bgeom, k_blocks, d_victims, p->ws, S(stream), p->pc.h_counts));
   if (p->n_parts == 1) {
-    m = k_blocks * p->bgeom.heads[0];
-  } else {
-    // which partitions the chosen blocks fall in is only known on the device
+    if (h_n_victims) *h_n_victims = k_blocks * p->bgeom.heads[0];
+    return KV_OK;
+  }
+  // which partitions the chosen blocks fall in is only known on the device
+  if (!p->pc.h_counts) {
+    // (the expansion kernel could not write the entry counts to the host itself)
     KV_CUDA(p, cudaMemcpyAsync(p->h_counts, p->ws.part_counts, 4 * sizeof(uint64_t), cudaMemcpyDeviceToHost,
                                S(stream)));
-    KV_CUDA(p, cudaEventRecord(p->ev_counts, S(stream)));
-    KV_CUDA(p, cudaEventSynchronize(p->ev_counts));
-    for (int q = 0; q < p->n_parts; ++q) m += p->h_counts[q] * p->bgeom.heads[q];
   }
-  if (h_n_victims) *h_n_victims = m;
+  if (!h_n_victims) return KV_OK;   // the caller reads kv_victim_counts once the stream has run
+  KV_CUDA(p, cudaEventRecord(p->ev_counts, S(stream)));
+  p->stats.host_waits += 1;
+  KV_CUDA(p, cudaEventSynchronize(p->ev_counts));
+  uint64_t m = 0;
+  for (int q = 0; q < p->n_parts; ++q) {
+    if (!p->pc.h_counts) p->h_counts[q] *= p->bgeom.heads[q];   // block counts came over: make them entries
+    m += p->h_counts[q];
+  }
+  *h_n_victims = m;
   return KV_OK;
 }
+
+const uint64_t* kv_victim_counts(const kv_pool* p) { return p ? p->h_counts : nullptr; }
 
 uint64_t kv_max_batch_bytes(const kv_pool* p, int32_t q) {
   if (!p || q < 0 || q >= p->n_parts) return 0;
@@ -714,6 +748,33 @@ uint64_t kv_max_batch_bytes(const kv_pool* p, int32_t q) {
 int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t batch_bytes,
                   kv_stream_t compute_, kv_stream_t copy_) {
   if (!p) return KV_ERR_INVALID_ARG;
+  if (p->n_parts == 1 || m == 0) {
+    const uint64_t one[4] = {m, 0, 0, 0};
+    return kv_demote_counted(p, d_victims, m, one, batch_bytes, compute_, copy_);
+  }
+  KV_DRAIN_ALL(p);
+  if (!d_victims || !aligned16(d_victims) || m > p->stats.n_entries - p->stats.n_free)
+    return KV_ERR_INVALID_ARG;
+  // Several partitions and no counts from the caller: count on the device (a read-only kernel)
+  // and wait for the answer.
+  cudaStream_t compute = S(compute_);
+  PartCounts pc = p->pc;
+  pc.h_counts = nullptr;
+  KV_CUDA(p, launch_partition_counts(d_victims, m, pc, compute));
+  KV_CUDA(p, cudaMemcpyAsync(p->h_counts, p->ws.part_counts, 4 * sizeof(uint64_t), cudaMemcpyDeviceToHost,
+                             compute));
+  KV_CUDA(p, cudaEventRecord(p->ev_counts, compute));
+  p->stats.host_waits += 1;
+  KV_CUDA(p, cudaEventSynchronize(p->ev_counts));
+  uint64_t counts[4] = {0, 0, 0, 0}, sum = 0;
+  for (int q = 0; q < p->n_parts; ++q) { counts[q] = p->h_counts[q]; sum += counts[q]; }
+  if (sum != m) return KV_ERR_INTERNAL;  // ids outside every partition
+  return kv_demote_counted(p, d_victims, m, counts, batch_bytes, compute_, copy_);
+}
+
+int32_t kv_demote_counted(kv_pool* p, const uint32_t* d_victims, uint64_t m, const uint64_t* counts,
+                          uint64_t batch_bytes, kv_stream_t compute_, kv_stream_t copy_) {
+  if (!p || (m > 0 && !counts)) return KV_ERR_INVALID_ARG;
   KV_DRAIN_ALL(p);
   if (m == 0) {
     for (int q = 0; q < 4; ++q) p->last_counts[q] = 0;
@@ -722,19 +783,9 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
   if (!d_victims || !aligned16(d_victims) || m > p->stats.n_entries - p->stats.n_free)
     return KV_ERR_INVALID_ARG;
   cudaStream_t compute = S(compute_), copy = S(copy_);
-  uint64_t kq[4] = {0, 0, 0, 0};
-  if (p->n_parts == 1) {
-    kq[0] = m;
-  } else {
-    KV_CUDA(p, launch_partition_counts(d_victims, m, p->bases, p->n_parts, p->ws, compute));
-    KV_CUDA(p, cudaMemcpyAsync(p->h_counts, p->ws.part_counts, 4 * sizeof(uint64_t),
-                               cudaMemcpyDeviceToHost, compute));
-    KV_CUDA(p, cudaEventRecord(p->ev_counts, compute));
-    KV_CUDA(p, cudaEventSynchronize(p->ev_counts));
-    uint64_t sum = 0;
-    for (int q = 0; q < p->n_parts; ++q) { kq[q] = p->h_counts[q]; sum += kq[q]; }
-    if (sum != m) return KV_ERR_INTERNAL;  // ids outside every partition
-  }
+  uint64_t kq[4] = {0, 0, 0, 0}, sum = 0;
+  for (int q = 0; q < p->n_parts; ++q) { kq[q] = counts[q]; sum += kq[q]; }
+  if (sum != m) return KV_ERR_INVALID_ARG;
   uint64_t per[4] = {0, 0, 0, 0};
   for (int q = 0; q < p->n_parts; ++q) {
     if (kq[q] == 0) continue;
@@ -750,7 +801,7 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
   pd.victims = d_victims;
   pd.compute = compute;
   pd.copy = copy;
-  pd.meta_done = p->deferred_packing && g_move_variant == 1;
+  pd.meta_done = p->deferred_packing;
   uint64_t off = 0;
   for (int q = 0; q < 4; ++q) {
     pd.off[q] = off;
@@ -819,7 +870,13 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
   const int li = p->list_turn;
   p->list_turn ^= 1;
   auto restore = [&]() { for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 1; };
-  cudaError_t e = cudaEventSynchronize(p->ev_list_copied[li]);  // the pinned list buffer is ours again
+  // the pinned list buffer of two calls ago must have been copied: normally long done
+  cudaError_t e = cudaEventQuery(p->ev_list_copied[li]);
+  if (e == cudaErrorNotReady) {
+    (void)cudaGetLastError();
+    p->stats.host_waits += 1;
+    e = cudaEventSynchronize(p->ev_list_copied[li]);
+  }
   if (e != cudaSuccess) { restore(); return cuda_fail(p, e); }
   // The H2D copies below may run on another stream than the D2H copies that filled the slots, so the
   // copy stream has to wait for the demotion(s) whose slot ranges the list touches.  d2h[q][0] is the
@@ -880,9 +937,8 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
     KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_ready[b], 0));
     {
       TimedScope ts(p, 1, cnt * eb, compute);
-      KV_CUDA(p, (g_move_variant ? launch_unpack_tma : launch_unpack)(
-                     g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, p->ws.free_list + c0, cnt,
-                     p->staging[b], p->ws, compute));
+      KV_CUDA(p, launch_unpack_tma(g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, p->ws.free_list + c0, cnt,
+                                   p->staging[b], p->ws, compute));
     }
     KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], compute));
   }
@@ -1021,15 +1077,22 @@ int32_t kv_set_deferred_packing(kv_pool* p, int32_t on) {
   return KV_OK;
 }
 
-int32_t kv_set_move_variant(int32_t variant) {
-  if (variant != 0 && variant != 1) return KV_ERR_INVALID_ARG;
-  g_move_variant = variant;
+int32_t kv_set_select_variant(kv_pool* p, int32_t variant) {
+  if (!p || (variant != 0 && variant != 1)) return KV_ERR_INVALID_ARG;
+  p->select_variant = variant;
   return KV_OK;
 }
 
-int32_t kv_set_select_variant(int32_t variant) {
-  if (variant != 0 && variant != 1) return KV_ERR_INVALID_ARG;
-  kvt::g_select_variant = variant;
+int32_t kv_selection_stats(kv_pool* p, kv_stream_t stream, kv_select_stats* out) {
+  if (!p || !out) return KV_ERR_INVALID_ARG;
+  KV_DRAIN_ALL(p);
+  KV_CUDA(p, cudaMemcpyAsync(p->h_sel_stats, &p->ws.sel->n_select, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost,
+                             S(stream)));
+  KV_CUDA(p, cudaStreamSynchronize(S(stream)));
+  out->selections = p->h_sel_stats[0];
+  out->hint_hits = p->h_sel_stats[1];
+  out->hint_misses = p->h_sel_stats[2];
+  out->reread_ctas = p->h_sel_stats[3];
   return KV_OK;
 }
 

@@ -9,7 +9,6 @@
 
 namespace kvt {
 
-constexpr int kSMs = 148;            // B200: 2 dies x 74 SMs
 constexpr int kThreads = 256;
 constexpr uint32_t kRadixBits1 = 11, kRadixBits2 = 11, kRadixBits3 = 10;
 constexpr uint32_t kHistBins = 2048;  // bins of the widest digit
@@ -21,6 +20,18 @@ constexpr uint32_t kPairFree = 0x80u;
 // Kernels launched by this library in this process (all pools).
 extern std::atomic<uint64_t> g_kernel_launches;
 inline void count_launches(uint64_t n) { g_kernel_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// Streaming multiprocessors of the current device (148 on a B200); grids are sized in
+// multiples of it.  Asked of the runtime at every launch: the answer belongs to the
+// device that is current, not to the process.
+inline int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    return 1;
+  }
+  return n;
+}
 
 // Geometry of one partition, as the kernels need it.
 struct PartGeom {
@@ -57,6 +68,7 @@ __device__ __forceinline__ float ema_catch_up(float ema, float decay, uint32_t m
 }
 
 // Per-entry state arrays.
+//
 struct EntryState {
   float* ema;
   float* decay;
@@ -84,6 +96,14 @@ struct SelectScalars {
   unsigned long long hint_n;   // ... and the number of keys it ran over
   unsigned long long below;    // keys below the bracket (accumulated per launch, cleared inside it)
   unsigned long long phase_ns[8];  // %globaltimer at the phase boundaries of the last persistent selection (CTA 0)
+  // how the persistent selections went so far (kv_selection_stats)
+  unsigned int n_select;       // selections run
+  unsigned int n_hint_hit;     // ... whose hint's bracket held rank k
+  unsigned int n_hint_miss;    // ... whose hint's bracket did not
+  unsigned int n_reread;       // CTAs (over all selections) that had to re-read their keys although the hint held
+  // persistent selection on a pool of several partitions: (below tau, equal to tau) counts of
+  // the entries before partition boundary q + 1 inside the slice of the CTA that holds it
+  uint2 bsplit[3];
 };
 
 // Sliding window of per-epoch (pair, hit) counts for the confidence-weighted
@@ -166,9 +186,19 @@ cudaError_t launch_head_init(const HeadWeights& hw, uint32_t n_imp, uint32_t n_w
 cudaError_t launch_blend_reset(const Workspace& ws, cudaStream_t s);
 
 // ---- kv_select.cu ----
+// Where the victims of a selection fall: partition bases (global entry ids; [n_parts] = N),
+// and where the per-partition victim counts go (device, and host memory the device can
+// write, or nullptr).
+struct PartCounts {
+  unsigned long long base[5] = {0, 0, 0, 0, 0};
+  int n_parts = 1;
+  unsigned long long* d_counts = nullptr;   // [4]
+  unsigned long long* h_counts = nullptr;   // [4] device-visible address of pinned host memory
+};
+// variant 1 = one persistent cooperative launch (falls back to 0 where the device cannot run
+// it or the slices are too long), 0 = one launch per phase of the radix select
 cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims, const Workspace& ws,
-                          cudaStream_t s);
-extern int g_select_variant;  // which selection launch_select uses (see kv_select.cu)
+                          cudaStream_t s, int variant = 1, const PartCounts* pc = nullptr);
 // kv_select_persist.cu: the same selection as one cooperative launch; *used tells
 // whether it was launched (false: the device cannot co-schedule it, nothing was enqueued)
 // With fs the launch also does the entry pass first (posterior, EMA, score; the
@@ -184,16 +214,19 @@ struct FusedScore {
 };
 cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t* d_victims,
                                      const Workspace& ws, cudaStream_t s, bool* used,
-                                     const FusedScore* fs = nullptr);
+                                     const FusedScore* fs = nullptr, const PartCounts* pc = nullptr);
 // kv_blocks.cu: k_blocks lowest blocks by weighted aggregate score; writes all their entries
-// (ascending) to d_victims and the per-partition block counts to ws.part_counts
+// (ascending) to d_victims, the per-partition block counts to ws.part_counts and the
+// per-partition ENTRY counts to h_entry_counts (host memory the device can write; may be nullptr)
 cudaError_t launch_select_blocks(const EntryState& st, const BlockGeom& bg, uint64_t k_blocks,
-                                 uint32_t* d_victims, const Workspace& ws, cudaStream_t s);
+                                 uint32_t* d_victims, const Workspace& ws, cudaStream_t s,
+                                 unsigned long long* h_entry_counts);
 // ascending ids of FREE entries in [lo, hi), at most `limit` of them, into ws.free_list
 cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uint64_t limit,
                              const Workspace& ws, cudaStream_t s);
-cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const uint64_t* bases5,
-                                    int n_parts, const Workspace& ws, cudaStream_t s);
+// victims per partition of an ascending list into pc.d_counts (and pc.h_counts)
+cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const PartCounts& pc,
+                                    cudaStream_t s);
 
 // ---- kv_dedup.cu ----
 // SHA-256 of the images of entries ids[0..m) (ids == nullptr: entries 0..m-1), 32 bytes each
@@ -208,21 +241,15 @@ cudaError_t launch_dedup(const uint8_t* digests, uint64_t m, uint32_t* canon, ui
 cudaError_t launch_init(const EntryState& st, uint64_t* hits, uint64_t* misses, float* P, float p0,
                         uint32_t* loc, uint64_t n_tags, const PartGeom* parts, int n_parts,
                         const Workspace& ws, cudaStream_t s);
-// packs victims[first .. first+count) of one partition into staging (images back to back)
-// followed, at meta_offset, by kv_slot_meta records; also moves the metadata.
-cudaError_t launch_pack(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* victims,
-                        uint64_t count, uint64_t ring_start, uint8_t* staging, uint64_t meta_offset,
-                        const Workspace& ws, cudaStream_t s);
-// scatters staging images [0, count) into free_list[first_free ..] slots of the partition
-cudaError_t launch_unpack(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
-                          const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
-                          const Workspace& ws, cudaStream_t s);
-// ---- kv_move_tma.cu: the same two operations on the bulk asynchronous copy engine ----
+// ---- kv_move_tma.cu: gather (demotion) and scatter (promotion) on the bulk asynchronous copy engine ----
+// pack: victims[0 .. count) of one partition into staging (images back to back) followed, at
+// meta_offset, by kv_slot_meta records; also moves the metadata.
 // mode: 0 = metadata and payload, 1 = metadata only (staging unused), 2 = payload only
 // (the metadata moved earlier; host-mirror records are rebuilt from the ring mirror)
 cudaError_t launch_pack_tma(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* victims,
                             uint64_t count, uint64_t ring_start, uint8_t* staging, uint64_t meta_offset,
                             const Workspace& ws, cudaStream_t s, uint32_t mode = 0);
+// unpack: staging images [0, count) into the listed free slots of the partition
 cudaError_t launch_unpack_tma(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
                               const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
                               const Workspace& ws, cudaStream_t s);
