@@ -83,6 +83,12 @@ def parse():
                          "deduplication of the digests; reported under phases, not part of a step")
     ap.add_argument("--tiny-entries", action="store_true",
                     help="32-64 byte blocks (same entry count and traces): for profiling scoring/selection")
+    ap.add_argument("--promote-run", type=int, default=None,
+                    help="promote lists made of runs of at most this many consecutive ring slots at seeded starts "
+                         "(instead of the pool's own list style)")
+    ap.add_argument("--gather-kb", type=int, default=None,
+                    help="promote lists whose runs average less than this many KiB go through the gather kernel "
+                         "(0 = always one transfer per run; default: the library's 256)")
     ap.add_argument("--select-variant", type=int, default=1, choices=[0, 1],
                     help="selection: 1 = one persistent cooperative launch, 0 = one launch per phase")
     return ap.parse_args()
@@ -447,6 +453,9 @@ def main():
 
     cfg, scale, w, chosen_because = choose_workload(args, torch, W, dev)
     w.seed = w.seed + 1000 * rank     # every rank owns its own pool and trace (weak scaling)
+    if args.promote_run is not None:
+        w.promote_style, w.max_run = "runs", args.promote_run
+    w.epochs = args.warmup + args.steps + 12   # block handles for every epoch this run admits (timed, e2e, breakdown)
     link = hostlink_probe(torch, dev) if rank == 0 and not args.no_hostlink else None
     runner = EpochRunner(w, batch_bytes=args.batch_mb << 20, fill_pattern=True, host_meta=True,
                          device=str(dev))
@@ -455,6 +464,8 @@ def main():
     from paper_2604_26968_b200 import binding as B
     pool.kv_set_select_variant(args.select_variant)
     pool.kv_set_deferred_packing(not args.no_deferred_packing)
+    if args.gather_kb is not None:
+        pool.kv_set_gather_threshold(args.gather_kb << 10)
     N, k = w.N, w.k
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     counts = pool.kv_epoch_counts() if dist_on else None
@@ -486,7 +497,7 @@ def main():
         else:
             runner.check(pool.kv_epoch_score_select(e, d_e, d_h, n, k, runner.victims), "kv_epoch_score_select")
         ev[1].record(pool.compute)
-        runner.check(pool.kv_demote(runner.victims, k, runner.batch_bytes), "kv_demote")
+        runner.check(runner.demote(), "kv_demote")
         lists = runner.promote_lists(e)
         ev[4].record(pool.copy_h2d)
         for q, lst in enumerate(lists):
@@ -538,7 +549,7 @@ def main():
             tot["ss"] += ev[0].elapsed_time(ev[1])
             tot["dem"] += ev[1].elapsed_time(ev[2])
             tot["pro"] += ev[4].elapsed_time(ev[5])
-            tot["all"] += max(ev[0].elapsed_time(ev[2]), ev[0].elapsed_time(ev[3]))
+            tot["all"] += max(ev[0].elapsed_time(ev[2]), ev[0].elapsed_time(ev[3]), ev[0].elapsed_time(ev[5]))
             tot["events"] += n
             tot["promoted_bytes"] += sum(len(l) * p.entry_bytes for l, p in zip(lists, w.parts))
             tot["launches"] = tot.get("launches", 0) + launches_step
@@ -616,7 +627,7 @@ def main():
             evb[2].record(pool.compute)
             runner.check(pool.kv_select_victims(k, runner.victims), "kv_select_victims")
             evb[3].record(pool.compute)
-            runner.check(pool.kv_demote(runner.victims, k, runner.batch_bytes), "kv_demote")
+            runner.check(runner.demote(), "kv_demote")
             for q, lst in enumerate(runner.promote_lists(epoch)):
                 runner.check(pool.kv_promote(q, lst, runner.batch_bytes), "kv_promote")
             runner.check(pool.kv_flush(), "kv_flush")
@@ -648,7 +659,7 @@ def main():
     demoted_per_step = eb_bytes
     promoted_per_step = tot["promoted_bytes"] / K
     pack_gbs = 2 * timing["pack_bytes"] / max(timing["pack_ms"], 1e-9) / 1e6
-    unpack_gbs = 2 * timing["unpack_bytes"] / max(timing["unpack_ms"], 1e-9) / 1e6
+    unpack_gbs = (2 * timing["unpack_bytes"] / max(timing["unpack_ms"], 1e-9) / 1e6) if timing["unpack_launches"] else None
     ss_bytes = 39 * N + 5 * (tot["events"] / K) + 4 * k
     ss_gbs = ss_bytes / (ss_ms * 1e-3) / 1e9
     fused = not (args.no_fused or dist_on)
@@ -667,6 +678,7 @@ def main():
                    "events_per_step": tot["events"] // K, "pool_bytes": sum(p.slab_bytes for p in w.parts),
                    "entry_bytes": [p.entry_bytes for p in w.parts], "batch_bytes": runner.batch_bytes,
                    "deferred_packing": not args.no_deferred_packing,
+                   "promote_lists": w.promote_style + ("" if w.promote_style != "runs" else " of <= %d slots" % w.max_run),
                    "fused_score_select": not (args.no_fused or dist_on),
                    "head_weights": bool(args.head_weights),
                    "ring_slots": [p.ring_slots for p in w.parts], "scale": scale,
@@ -679,8 +691,12 @@ def main():
             "demote_ms": dem_ms, "demote_gbs": demoted_per_step / (dem_ms * 1e-3) / 1e9,
             "promote_ms": pro_ms, "promote_gbs": promoted_per_step / max(pro_ms * 1e-3, 1e-12) / 1e9,
             "pack_kernel_gbs": pack_gbs, "pack_kernel_frac_of_%s_hbm" % peak_kind: pack_gbs / peak,
-            "unpack_kernel_gbs": unpack_gbs, "unpack_kernel_frac_of_%s_hbm" % peak_kind: unpack_gbs / peak,
+            "unpack_kernel_gbs": unpack_gbs,
+            "unpack_kernel_frac_of_%s_hbm" % peak_kind: (unpack_gbs / peak) if unpack_gbs else None,
             "pack_launches": timing["pack_launches"], "unpack_launches": timing["unpack_launches"],
+            "gather_launches": timing["gather_launches"],
+            "gather_kernel_gbs_over_the_host_link": (timing["gather_bytes"] / max(timing["gather_ms"], 1e-9) / 1e6
+                                                     if timing["gather_launches"] else None),
         },
         "hostlink": link,
         "roofline": {"kernel": ("event_reduce_kernel + select_persistent_kernel<true>" if fused else
@@ -717,7 +733,9 @@ def main():
         line["e2e"] = e2e
     if not args.no_cpu_baseline:
         n_ep = 6
-        t_ss, t_all, done = oracle_epochs(w, n_ep, warm=1)
+        # (a workload of its own: the trace generators keep session state from epoch to epoch)
+        w_cpu = W.config(cfg, scale=scale, ring_slots=args.ring_slots, tiny_entries=args.tiny_entries)
+        t_ss, t_all, done = oracle_epochs(w_cpu, n_ep, warm=1)
         mv = oracle_movement(W, cfg)
         line["cpu_baseline"] = {
             "value": N * done / t_ss, "unit": UNIT, "cores": 1, "kind": "oracle",

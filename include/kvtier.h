@@ -324,6 +324,17 @@ const uint64_t* kv_victim_counts(const kv_pool* pool);
 int32_t kv_promote(kv_pool* pool, int32_t partition, const uint64_t* h_host_slots, uint64_t m,
                    uint64_t batch_bytes, kv_stream_t compute, kv_stream_t copy);
 
+/* How kv_promote moves the bytes.  Runs of consecutive ring slots in the list become
+ * one DMA transfer each into a staging buffer, which the unpack kernel scatters; that
+ * is right for long runs.  A list ordered by token position (RoPE-aware prefetching
+ * section: blocks covering the next positions of a sequence, every layer of a block
+ * in turn) names slots that lie far apart -- only a block's heads are neighbours in a
+ * ring filled in (layer, block, head) order -- and breaks into runs of a few slots.
+ * For a list whose runs average less than run_bytes the entries are instead fetched
+ * by a kernel on the copy stream, through the device's view of the pinned ring, and
+ * written straight into their slots.  Default 256 KiB; 0 = always per-run transfers. */
+int32_t kv_set_gather_threshold(kv_pool* pool, uint64_t run_bytes);
+
 /* Lazy decay of promoted entries (off by default).  The head-granular eviction
  * section updates importance on every step for blocks in HBM; the paper does not
  * say what a block's importance is when it returns from a lower tier.  Off, the
@@ -458,6 +469,7 @@ typedef struct {
   uint64_t n_entries, n_free;
   uint64_t kernel_launches; /* kernels launched by the library in this process so far */
   uint64_t host_waits;      /* times kv_demote, kv_promote or kv_select_victim_blocks blocked the host */
+  uint64_t gathered;        /* entries promoted by the gather kernel instead of per-run transfers */
 } kv_stats;
 
 /* Host-side counters, kept eagerly at call time. */
@@ -483,6 +495,8 @@ typedef struct {
   double pack_ms, unpack_ms;            /* summed kernel durations */
   uint64_t pack_launches, unpack_launches;
   uint64_t pack_bytes, unpack_bytes;    /* payload bytes moved (read + written counted once each) */
+  double gather_ms;                     /* the same for the gather kernel of kv_promote, which reads */
+  uint64_t gather_launches, gather_bytes; /* the host ring itself: its time is the host link's */
 } kv_timing;
 int32_t kv_timing_enable(kv_pool* pool, int32_t on);
 int32_t kv_timing_read(kv_pool* pool, kv_timing* out);

@@ -61,7 +61,7 @@ class kv_pool_desc(C.Structure):
 class kv_stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in
                 ("epochs", "events", "victims", "promoted", "admitted", "bytes_demoted",
-                 "bytes_promoted", "bytes_dropped", "n_entries", "n_free", "kernel_launches", "host_waits")]
+                 "bytes_promoted", "bytes_dropped", "n_entries", "n_free", "kernel_launches", "host_waits", "gathered")]
 
 
 class kv_select_stats(C.Structure):
@@ -71,7 +71,8 @@ class kv_select_stats(C.Structure):
 class kv_timing(C.Structure):
     _fields_ = [("pack_ms", C.c_double), ("unpack_ms", C.c_double),
                 ("pack_launches", C.c_uint64), ("unpack_launches", C.c_uint64),
-                ("pack_bytes", C.c_uint64), ("unpack_bytes", C.c_uint64)]
+                ("pack_bytes", C.c_uint64), ("unpack_bytes", C.c_uint64),
+                ("gather_ms", C.c_double), ("gather_launches", C.c_uint64), ("gather_bytes", C.c_uint64)]
 
 
 class kv_slot_meta(C.Structure):
@@ -87,7 +88,7 @@ EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_
            "kv_epoch_update", "kv_set_policy", "kv_set_lazy_decay", "kv_hash_entries", "kv_dedup_table_slots", "kv_dedup_digests", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
-           "kv_set_select_variant", "kv_selection_stats", "kv_demote_counted", "kv_victim_counts", "kv_last_cuda_error", "kv_status_string",
+           "kv_set_select_variant", "kv_selection_stats", "kv_demote_counted", "kv_victim_counts", "kv_set_gather_threshold", "kv_last_cuda_error", "kv_status_string",
            "kv_version")
 
 _lib = None
@@ -183,6 +184,8 @@ def load():
     L.kv_demote_counted.argtypes = [vp, vp, u64, vp, u64, vp, vp]
     L.kv_victim_counts.restype = vp
     L.kv_victim_counts.argtypes = [vp]
+    L.kv_set_gather_threshold.restype = i32
+    L.kv_set_gather_threshold.argtypes = [vp, u64]
     L.kv_selection_stats.restype = i32
     L.kv_selection_stats.argtypes = [vp, vp, vp]
     L.kv_last_cuda_error.restype = i32
@@ -413,11 +416,13 @@ class Pool:
         return self.lib.kv_select_victims(self._h, int(k), d_victims.data_ptr() if k else None,
                                           _stream_ptr(self.compute))
 
-    def kv_select_victim_blocks(self, k_blocks, d_victims):
-        """Returns (status, number of entries written)."""
+    def kv_select_victim_blocks(self, k_blocks, d_victims, wait=True):
+        """Returns (status, number of entries written).  wait=False passes no place for the
+        number: the call then never blocks, and the entries per partition are in
+        kv_victim_counts() once the compute stream has run (the number returned is 0)."""
         n = C.c_uint64(0)
         rc = self.lib.kv_select_victim_blocks(self._h, int(k_blocks), d_victims.data_ptr() if k_blocks else None,
-                                              C.byref(n), _stream_ptr(self.compute))
+                                              C.byref(n) if wait else None, _stream_ptr(self.compute))
         return rc, n.value
 
     def kv_demote(self, d_victims, m, batch_bytes):
@@ -445,6 +450,9 @@ class Pool:
         rc = self.lib.kv_admit(self._h, epoch, decay, d_new_pairs.data_ptr(), d_new_pairs.numel(),
                                1 if fill_pattern else 0, C.byref(n), _stream_ptr(self.compute))
         return rc, n.value
+
+    def kv_set_gather_threshold(self, run_bytes):
+        return self.lib.kv_set_gather_threshold(self._h, int(run_bytes))
 
     def kv_set_deferred_packing(self, on=True):
         return self.lib.kv_set_deferred_packing(self._h, 1 if on else 0)

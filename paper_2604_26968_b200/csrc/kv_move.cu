@@ -147,6 +147,7 @@ __global__ void init_scalars_kernel(uint64_t* hits, uint64_t* misses, float* P, 
     ws.sel->prefix = 0; ws.sel->tau = 0; ws.sel->k_rem = 0; ws.sel->need_eq = 0;
     ws.sel->bar_arrive = 0; ws.sel->bar_done = 0; ws.sel->update_ticket = 0; ws.sel->hint_last = 0;
     ws.sel->hint_valid = 0; ws.sel->hint_tau = 0; ws.sel->hint_n = 0; ws.sel->below = 0;
+    ws.sel->hint_shift = 11; ws.sel->hint_resid = 0;
     ws.sel->n_select = 0; ws.sel->n_hint_hit = 0; ws.sel->n_hint_miss = 0; ws.sel->n_reread = 0;
   }
 }

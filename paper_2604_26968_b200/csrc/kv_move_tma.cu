@@ -14,6 +14,8 @@
 //
 // Every wait is bounded: a lane that gives up sets KV_DEV_WAIT_EXPIRED in the
 // device status word, drains its own stores and leaves.
+#include <cstdlib>
+
 #include "kvtier_internal.cuh"
 
 namespace kvt {
@@ -292,6 +294,71 @@ move_tma_kernel(const MoveArgs a) {
     }
     bulk_wait_all();
   }
+}
+
+// ---- promotion of scattered host entries --------------------------------------------
+// A prefetch list ordered by token position names, for every block, its layers one after
+// the other; in the host ring only a block's heads are neighbours, its layers lie a whole
+// demotion's share apart.  Such a list breaks into runs of a few slots, and one DMA
+// transfer per run spends its time on set-up.  This kernel fetches the listed entries
+// itself, through the address at which the device sees the pinned ring, and writes them
+// straight into their paged slots: no staging buffer, no per-run transfer.  A warp moves
+// one piece of up to 2 KB at a time with four 16-byte loads in flight per lane; with two
+// blocks of eight warps per SM several MB are in flight, which a host link with a round
+// trip of a few microseconds needs.
+constexpr uint32_t kGatherPiece = 2048;   // 32 lanes x 4 x 16 bytes
+constexpr uint32_t kGatherThreads = 256;
+
+__global__ void __launch_bounds__(kGatherThreads)
+gather_promote_kernel(const MoveArgs a, const uint8_t* __restrict__ ring) {
+  const PartGeom& g = a.g;
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t ppc = (g.chunk_bytes + kGatherPiece - 1) / kGatherPiece;  // pieces per chunk
+  const uint32_t ppe = ppc * g.n_chunks;                                    // pieces per entry
+  const uint64_t total = a.count * ppe;
+  const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  for (uint64_t piece = (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); piece < total; piece += warps) {
+    const uint64_t j = piece / ppe;
+    const uint32_t r = (uint32_t)(piece - j * ppe);
+    const uint32_t c = r / ppc;
+    const uint32_t in_chunk = (r - c * ppc) * kGatherPiece;
+    const uint32_t f = a.ids[j];
+    const uint32_t slot = a.slots[j];
+    if ((uint64_t)f < g.base || (uint64_t)f >= g.base + g.n || slot >= g.ring_slots) {
+      if (lane == 0 && r == 0) atomicOr(a.status, KV_DEV_BAD_INDEX);
+      continue;
+    }
+    const uint32_t len = min(kGatherPiece, g.chunk_bytes - in_chunk);
+    const uint8_t* src = ring + (uint64_t)slot * g.entry_bytes + (uint64_t)c * g.chunk_bytes + in_chunk;
+    uint8_t* dst = g.slab + slab_chunk_offset(g, (uint64_t)f - g.base, c) + in_chunk;
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t off = (u * 32 + lane) * 16;
+      if (off < len) v[u] = __ldcs(reinterpret_cast<const uint4*>(src + off));
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t off = (u * 32 + lane) * 16;
+      if (off < len) __stcs(reinterpret_cast<uint4*>(dst + off), v[u]);
+    }
+    if (r == 0 && lane == 0) promote_meta(a, f, slot);
+  }
+}
+
+cudaError_t launch_gather_promote(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
+                                  const uint32_t* free_ids, uint64_t count, const uint8_t* ring_dev,
+                                  const Workspace& ws, cudaStream_t s) {
+  if (count == 0) return cudaSuccess;
+  MoveArgs a{g, st, loc, free_ids, slots, count, 0, nullptr, ~0ull, ws.status, kMoveAll};
+  const uint64_t pieces = count * ((g.chunk_bytes + kGatherPiece - 1) / kGatherPiece) * g.n_chunks;
+  uint64_t blocks = (pieces * 32 + kGatherThreads - 1) / kGatherThreads;
+  uint64_t cap = 32;
+  if (const char* e = std::getenv("KVTIER_GATHER_BLOCKS")) cap = (uint64_t)std::atoi(e);
+  if (blocks > cap) blocks = cap;
+  gather_promote_kernel<<<(unsigned)(blocks ? blocks : 1), kGatherThreads, 0, s>>>(a, ring_dev);
+  count_launches(1);
+  return cudaGetLastError();
 }
 
 static unsigned tma_grid(uint64_t count) {

@@ -370,7 +370,7 @@ cudaError_t launch_select(const EntryState& st, uint64_t k, uint32_t* d_victims,
 }
 
 cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uint64_t limit,
-                             const Workspace& ws, cudaStream_t s) {
+                             const Workspace& ws, cudaStream_t s, uint64_t out_offset) {
   if (hi <= lo || limit == 0) return cudaSuccess;
   const uint64_t tile0 = lo / kTileEntries;
   const uint32_t n_tiles = (uint32_t)((hi + kTileEntries - 1) / kTileEntries - tile0);
@@ -378,7 +378,7 @@ cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uin
                                                     ws.tile_counts);
   tile_scan_kernel<<<1, 1024, 0, s>>>(ws.tile_counts, ws.tile_offsets, n_tiles);
   tile_write_kernel<1><<<n_tiles, kThreads, 0, s>>>(st.score, st.state, st.n, lo, hi, tile0, ws.sel,
-                                                    ws.tile_offsets, limit, ws.free_list);
+                                                    ws.tile_offsets, limit, ws.free_list + out_offset);
   count_launches(3);
   return cudaGetLastError();
 }

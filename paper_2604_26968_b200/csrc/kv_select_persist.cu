@@ -52,9 +52,9 @@ constexpr uint32_t kPChunk = kPThreads * 4;             // 4096 entries: one 16-
 constexpr uint32_t kPHistBins = 2048;
 constexpr uint32_t kExcluded = 0xFFFFFFFFu;             // key of a non-candidate (FREE) entry
 constexpr uint32_t kBarrierSpins = 1u << 22;
-constexpr uint32_t kBracketShift = 11;                  // a bracket bin is 2^11 keys wide ...
-constexpr uint32_t kBracketHalf = 1u << 21;             // ... and the 2,048 bins reach 2^21 keys to either side of the hint
-constexpr uint32_t kBracketBits = 22;                   // log2 of the bracket's width in keys
+constexpr uint32_t kBracketShiftMax = 11;               // a bracket bin is at most 2^11 keys wide: the 2,048 bins then
+                                                        // reach 2^21 keys to either side of the hint ...
+constexpr uint32_t kBracketShiftMin = 7;                // ... and at least 2^7 (2^17 keys to either side)
 constexpr uint32_t kPIdxBits = 18;                      // index of an entry inside its slice
 constexpr uint32_t kPMaxSlice = 1u << kPIdxBits;        // entries per CTA the bitmaps are sized for (2 x 32 KB)
 constexpr uint32_t kPSlotsMax = 32;                     // bracket keys a thread can note (its private slots)
@@ -113,6 +113,7 @@ struct PArgs {
   uint32_t words;         // 32-bit words of one bitmap of a slice (a multiple of 4)
   uint32_t slots;         // private slots per thread for keys inside the bracket (at least 10)
   PartCounts pc;          // partitions of the pool (the victims per partition are a by-product)
+  uint32_t* spill;        // [n] global scratch for the notes a thread's slots cannot hold (nullptr: none)
   // the scoring pass of the fused form
   EntryState st;
   Predictor pd;
@@ -382,10 +383,19 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   // and then only the notes are looked at again.
   const bool hint = a.sel->hint_valid != 0 && a.sel->hint_n == a.n;
   const uint32_t hint_tau = a.sel->hint_tau;
-  const uint32_t base0 = hint ? (hint_tau > kBracketHalf ? hint_tau - kBracketHalf : 0u) : 0u;
-  const uint32_t shift0 = hint ? kBracketShift : 21u;
+  // The bracket's width follows how well the hints have been doing: 2,048 bins of 2^bshift keys.
+  uint32_t bshift = a.sel->hint_shift;
+  bshift = bshift < kBracketShiftMin ? kBracketShiftMin : (bshift > kBracketShiftMax ? kBracketShiftMax : bshift);
+  const uint32_t bbits = bshift + 11u;                  // log2 of the bracket's width in keys
+  const uint32_t bhalf = 1u << (bbits - 1u);
+  const uint32_t base0 = hint ? (hint_tau > bhalf ? hint_tau - bhalf : 0u) : 0u;
+  const uint32_t shift0 = hint ? bshift : 21u;
+  bool hint_hit = false;
   WarpHist wh;
-  uint32_t n_noted = 0;   // keys of this thread inside the bracket (noted while slots last)
+  uint32_t n_noted = 0;   // keys of this thread inside the bracket
+  // notes beyond the thread's slots: the CTA's stretch of the global scratch, laid out like the slots
+  uint32_t* const spill = a.spill ? a.spill + s0 : nullptr;
+  auto note_at = [&](uint32_t i) { return i < a.slots ? s_note[i * kPThreads + t] : __ldcg(&spill[(i - a.slots) * kPThreads + t]); };
   auto phase_a = [&](uint32_t c, const uint32_t key[4]) {
     if (!hint) {
 #pragma unroll
@@ -398,9 +408,11 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       const uint32_t d = key[q] - base0;
       const bool below = key[q] < base0;   // (an excluded key is 0xFFFFFFFF: never below)
       nib_l |= (uint32_t)below << q;
-      if (!below && (d >> kBracketBits) == 0u && key[q] != kExcluded) {
-        atomicAdd(&s_hist[d >> kBracketShift], 1u);
-        if (n_noted < a.slots) s_note[n_noted * kPThreads + t] = d | ((uint32_t)q << 22) | (c << 24);
+      if (!below && (d >> bbits) == 0u && key[q] != kExcluded) {
+        atomicAdd(&s_hist[d >> bshift], 1u);
+        const uint32_t note = d | ((uint32_t)q << 22) | (c << 24);
+        if (n_noted < a.slots) s_note[n_noted * kPThreads + t] = note;
+        else if (spill) spill[(n_noted - a.slots) * kPThreads + t] = note;   // (a dense slice: the rest goes to L2)
         ++n_noted;
       }
     }
@@ -452,9 +464,10 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     (void)block_scan_excl(below, s_warp, cta_below0);
     if (t == 0 && cta_below0) atomicAdd(&a.sel->below, (unsigned long long)cta_below0);
   }
-  // a thread that ran out of slots sends the whole CTA the long way (its keys are re-read)
-  const bool notes_complete = __syncthreads_or(n_noted > a.slots) == 0;
-  if (n_noted > a.slots) n_noted = a.slots;
+  // without the global scratch a thread that ran out of slots sends the whole CTA the long way
+  // (its keys are re-read)
+  const bool notes_complete = spill != nullptr || __syncthreads_or(n_noted > a.slots) == 0;
+  if (!spill && n_noted > a.slots) n_noted = a.slots;
   stamp(1);
   ok = grid_barrier(bar, G);
   stamp(2);
@@ -491,16 +504,16 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       } else if (use_notes) {
         // the last histogram (single keys of the bracket bin that holds rank k) from the
         // notes; noted keys of earlier bins are below the final range: their bit joins s_bit_l
-        const uint32_t bin_k = (base - base0) >> kBracketShift;
+        const uint32_t bin_k = (base - base0) >> bshift;
         uint32_t p_bin = 0, p_cnt = 0;   // the thread's pending count for one key value
         for (uint32_t i = 0; i < n_noted; ++i) {
-          const uint32_t v = s_note[i * kPThreads + t];
-          const uint32_t d = v & ((1u << kBracketBits) - 1u), b = d >> kBracketShift;
+          const uint32_t v = note_at(i);
+          const uint32_t d = v & ((1u << 22) - 1u), b = d >> bshift;
           if (b < bin_k) {
             const uint32_t j = (v >> 24) * kPChunk + 4u * t + ((v >> 22) & 3u);
             atomicOr(&s_bit_l[j >> 5], 1u << (j & 31u));
           } else if (b == bin_k) {
-            const uint32_t low = d & ((1u << kBracketShift) - 1u);
+            const uint32_t low = d & ((1u << bshift) - 1u);
             if (low != p_bin) {
               if (p_cnt) atomicAdd(&s_hist[p_bin], p_cnt);
               p_bin = low;
@@ -555,6 +568,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       pick_bin(a.hist, kPHistBins, above ? a.k - below : 1ull, s_warp, s_pick, bin, before);
       if (above && bin != 0xFFFFFFFFu) {
         k_rem = a.k - below;
+        hint_hit = true;
         use_notes = notes_complete;
         if (t == 0) {
           if (blockIdx.x == 0) atomicAdd(&a.sel->n_hint_hit, 1u);
@@ -600,12 +614,12 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     const unsigned long long need_eq = k_rem;
     uint32_t c_l = 0, c_e = 0;
     if (use_notes) {
-      const uint32_t bin_k = (base - base0) >> kBracketShift;
+      const uint32_t bin_k = (base - base0) >> bshift;
       for (uint32_t i = 0; i < n_noted; ++i) {
-        const uint32_t v = s_note[i * kPThreads + t];
-        const uint32_t d = v & ((1u << kBracketBits) - 1u);
-        if ((d >> kBracketShift) != bin_k) continue;
-        const uint32_t low = d & ((1u << kBracketShift) - 1u);
+        const uint32_t v = note_at(i);
+        const uint32_t d = v & ((1u << 22) - 1u);
+        if ((d >> bshift) != bin_k) continue;
+        const uint32_t low = d & ((1u << bshift) - 1u);
         const uint32_t j = (v >> 24) * kPChunk + 4u * t + ((v >> 22) & 3u);
         if (low < tau_low) atomicOr(&s_bit_l[j >> 5], 1u << (j & 31u));
         else if (low == tau_low) atomicOr(&s_bit_e[j >> 5], 1u << (j & 31u));
@@ -781,6 +795,21 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       long long guess = (long long)tau + step;
       if (guess < 0) guess = 0;
       if (guess > 0xFFFFFFFEll) guess = 0xFFFFFFFEll;
+      // ... and the bracket is as wide as the hints have been off lately: eight times a slowly
+      // decaying maximum of |tau - hinted tau|, full width again after a miss (a narrow
+      // bracket means fewer keys to note; a miss costs two more passes over the keys)
+      uint32_t resid = a.sel->hint_resid, new_shift = kBracketShiftMax;
+      if (hint_hit) {
+        const uint32_t off = tau > hint_tau ? tau - hint_tau : hint_tau - tau;
+        resid -= resid >> 2;
+        if (off > resid) resid = off;
+        new_shift = kBracketShiftMin;
+        while (new_shift < kBracketShiftMax && (1ull << (new_shift + 10u)) < 8ull * resid) ++new_shift;
+      } else {
+        resid = 1u << 18;
+      }
+      a.sel->hint_resid = resid;
+      a.sel->hint_shift = new_shift;
       a.sel->hint_last = tau;
       a.sel->hint_tau = (uint32_t)guess;
       a.sel->hint_n = a.n;
@@ -901,6 +930,7 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   const size_t smem = persist_smem(a.words, a.slots);
   if (smem > pd.smem_max) return cudaSuccess;
   a.pc = pc ? *pc : PartCounts{};
+  a.spill = ws.free_list;   // (scratch of promotions and admissions: idle while a selection runs)
   a.st = st;
   a.pd = Predictor{};
   a.hw = HeadWeights{};

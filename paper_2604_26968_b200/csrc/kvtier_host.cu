@@ -18,6 +18,9 @@ std::atomic<uint64_t> g_kernel_launches{0};
 namespace {
 
 constexpr uint64_t kAlign = 256;
+// promote lists in flight: pinned host buffers (and their device copies) used in turn, so that
+// kv_promote only ever has to wait for the copy of the list given kListBufs calls earlier
+constexpr int kListBufs = 8;
 inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -66,6 +69,7 @@ struct PartHost {
   std::vector<uint8_t> live;
   uint8_t* h_ring = nullptr;
   uint8_t* h_meta = nullptr;
+  const uint8_t* ring_dev = nullptr;   // where the device sees h_ring (nullptr: it cannot)
 };
 
 }  // namespace
@@ -81,13 +85,13 @@ struct kv_pool {
   uint8_t* staging[4] = {nullptr, nullptr, nullptr, nullptr};  // [0,1] demotion, [2,3] promotion
   uint64_t staging_bytes = 0;
   uint64_t max_promote = 0;
-  uint32_t* h_list[2] = {nullptr, nullptr};
+  uint32_t* h_list[kListBufs] = {};
   uint64_t* h_counts = nullptr;
   uint32_t* h_status = nullptr;
   uint64_t next_tag = 0;
   kv_stats stats;
   uint64_t last_counts[4] = {0, 0, 0, 0};
-  cudaEvent_t ev_staging_free[4], ev_ready[4], ev_list_copied[2], ev_list_free[2], ev_counts;
+  cudaEvent_t ev_staging_free[4], ev_ready[4], ev_list_copied[kListBufs], ev_list_free[kListBufs], ev_counts;
   // copies in flight: the last two demotions per partition (ring slot range + completion event of
   // their D2H copies) and the last promotion's H2D copies
   struct D2H { cudaEvent_t ev; uint64_t start = 0, count = 0; bool valid = false; };
@@ -98,6 +102,11 @@ struct kv_pool {
   int demote_turn = 0, promote_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
   ScoreOptions score_opt;   // eviction policy and confidence blend
+  uint64_t gather_run_bytes = 256u << 10;   // promote lists whose runs average less go through the gather kernel
+  // promotions run their kernels on the copy stream they are given; the compute stream joins
+  // them (waits for ev_promoted) before the next kernel that reads what they wrote
+  cudaEvent_t ev_promote_ready, ev_promoted[4];
+  bool promote_open[4] = {false, false, false, false};
   int select_variant = 1;   // 1 = persistent cooperative selection, 0 = one launch per phase
   PartCounts pc;            // partition bases and where selections leave the victims per partition
   uint32_t* h_sel_stats = nullptr;
@@ -127,10 +136,10 @@ namespace {
 
 struct Layout {
   uint64_t head_imp, head_mult, head_w;
-  uint64_t delta, hist, sel, status, blend, block_score, block_state, block_victims, part_counts, tile_counts, tile_offsets, free_list, slot_list[2];
+  uint64_t delta, hist, sel, status, blend, block_score, block_state, block_victims, part_counts, tile_counts, tile_offsets, free_list, slot_list[kListBufs];
   uint64_t ring[4][6];
   uint64_t dev_total;
-  uint64_t h_list[2], h_counts, h_status, h_sel_stats, host_total;
+  uint64_t h_list[kListBufs], h_counts, h_status, h_sel_stats, host_total;
   uint32_t n_tiles;
 };
 
@@ -206,8 +215,7 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
   L->tile_counts = take((uint64_t)L->n_tiles * 8);
   L->tile_offsets = take((uint64_t)L->n_tiles * 8);
   L->free_list = take(g.N * 4);
-  L->slot_list[0] = take(d->max_promote * 4);
-  L->slot_list[1] = take(d->max_promote * 4);
+  for (int b = 0; b < kListBufs; ++b) L->slot_list[b] = take(d->max_promote * 4);
   for (int q = 0; q < g.n_parts; ++q) {
     const uint64_t R = d->part[q].ring_slots;
     for (int a = 0; a < 4; ++a) L->ring[q][a] = take(R * 4);
@@ -217,8 +225,7 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
   L->dev_total = o;
   uint64_t h = 0;
   auto htake = [&h](uint64_t bytes) { uint64_t at = h; h = align_up(h + bytes, kAlign); return at; };
-  L->h_list[0] = htake(d->max_promote * 4);
-  L->h_list[1] = htake(d->max_promote * 4);
+  for (int b = 0; b < kListBufs; ++b) L->h_list[b] = htake(d->max_promote * 4);
   L->h_counts = htake(4 * 8);
   L->h_status = htake(4);
   L->h_sel_stats = htake(16);
@@ -254,12 +261,26 @@ void scoring_pass_enqueued(kv_pool* p, uint32_t epoch) {
   for (int q = 0; q < p->n_parts; ++q) p->geom[q].epoch_now = epoch;
 }
 
+// every event object the pool owns (the timing events apart)
+std::vector<cudaEvent_t*> all_events(kv_pool* p) {
+  std::vector<cudaEvent_t*> evs;
+  for (int b = 0; b < 4; ++b) { evs.push_back(&p->ev_staging_free[b]); evs.push_back(&p->ev_ready[b]); }
+  for (int q = 0; q < 4; ++q) { evs.push_back(&p->d2h[q][0].ev); evs.push_back(&p->d2h[q][1].ev); }
+  evs.push_back(&p->ev_h2d_done);
+  for (int b = 0; b < kListBufs; ++b) { evs.push_back(&p->ev_list_copied[b]); evs.push_back(&p->ev_list_free[b]); }
+  evs.push_back(&p->ev_counts);
+  evs.push_back(&p->ev_promote_ready);
+  for (int q = 0; q < 4; ++q) evs.push_back(&p->ev_promoted[q]);
+  return evs;
+}
+
 void timing_settle(kv_pool* p, kv_pool::Timed& t) {
   if (!t.pending) return;
   float ms = 0.f;
   if (cudaEventSynchronize(t.b) == cudaSuccess && cudaEventElapsedTime(&ms, t.a, t.b) == cudaSuccess) {
     if (t.kind == 0) { p->totals.pack_ms += ms; p->totals.pack_launches += 1; p->totals.pack_bytes += t.bytes; }
-    else { p->totals.unpack_ms += ms; p->totals.unpack_launches += 1; p->totals.unpack_bytes += t.bytes; }
+    else if (t.kind == 1) { p->totals.unpack_ms += ms; p->totals.unpack_launches += 1; p->totals.unpack_bytes += t.bytes; }
+    else { p->totals.gather_ms += ms; p->totals.gather_launches += 1; p->totals.gather_bytes += t.bytes; }
   }
   t.pending = false;
 }
@@ -334,16 +355,18 @@ int32_t enqueue_pack_chunk(kv_pool* p, int q, uint64_t c0, uint64_t cnt) {
   return KV_OK;
 }
 
-// Enqueues pending chunks of the last demotion, in order, until partition q_upto
-// has `need` of its victims packed (q_upto < 0: everything), or `max_chunks` were
-// enqueued.
-int32_t drain_pending(kv_pool* p, int q_upto, uint64_t need, uint64_t max_chunks) {
+// Enqueues pending chunks of the last demotion: of partition q_only until `need` of its
+// victims are packed (the other partitions' chunks stay where they are: every partition has
+// its own ring, so their order among each other is free), or, with q_only < 0, of every
+// partition in order; never more than `max_chunks`.
+int32_t drain_pending(kv_pool* p, int q_only, uint64_t need, uint64_t max_chunks) {
   kv_pool::Pending& pd = p->pending;
   if (!pd.active) return KV_OK;
   uint64_t done = 0;
   for (int q = 0; q < p->n_parts; ++q) {
+    if (q_only >= 0 && q != q_only) continue;
     while (pd.next[q] < pd.kq[q]) {
-      if (q_upto >= 0 && (q > q_upto || (q == q_upto && pd.next[q] >= need))) return KV_OK;
+      if (q_only >= 0 && pd.next[q] >= need) break;
       if (done >= max_chunks) return KV_OK;
       const uint64_t c0 = pd.next[q];
       const uint64_t cnt = (pd.kq[q] - c0 < pd.per[q]) ? pd.kq[q] - c0 : pd.per[q];
@@ -363,7 +386,9 @@ int32_t drain_pending(kv_pool* p, int q_upto, uint64_t need, uint64_t max_chunks
       }
     }
   }
-  pd.active = false;
+  bool left = false;
+  for (int q = 0; q < p->n_parts; ++q) left = left || pd.next[q] < pd.kq[q];
+  pd.active = left;
   return KV_OK;
 }
 
@@ -371,6 +396,26 @@ int32_t drain_pending(kv_pool* p, int q_upto, uint64_t need, uint64_t max_chunks
   do {                                                                      \
     const int32_t rc__ = drain_pending(pool, -1, 0, ~0ull);                  \
     if (rc__ != KV_OK) return rc__;                                         \
+  } while (0)
+
+// Makes `s` wait for the promotions whose kernels may still be running on their copy streams
+// (all of them, or partition q's only).
+int32_t join_promotions(kv_pool* p, cudaStream_t s, int q_only = -1) {
+  for (int q = 0; q < p->n_parts; ++q) {
+    if (!p->promote_open[q] || (q_only >= 0 && q != q_only)) continue;
+    KV_CUDA(p, cudaStreamWaitEvent(s, p->ev_promoted[q], 0));
+    p->promote_open[q] = false;
+  }
+  return KV_OK;
+}
+
+// Every call that reads or changes entry state first enqueues what deferred packing holds back
+// and lets its stream wait for the promotions in flight.
+#define KV_SETTLE(pool, stream)                                             \
+  do {                                                                      \
+    KV_DRAIN_ALL(pool);                                                     \
+    const int32_t rc2__ = join_promotions(pool, S(stream));                 \
+    if (rc2__ != KV_OK) return rc2__;                                       \
   } while (0)
 
 }  // namespace
@@ -468,12 +513,10 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
   p->ws.tile_counts = reinterpret_cast<uint2*>(w + L.tile_counts);
   p->ws.tile_offsets = reinterpret_cast<uint2*>(w + L.tile_offsets);
   p->ws.free_list = reinterpret_cast<uint32_t*>(w + L.free_list);
-  p->ws.slot_list[0] = reinterpret_cast<uint32_t*>(w + L.slot_list[0]);
-  p->ws.slot_list[1] = reinterpret_cast<uint32_t*>(w + L.slot_list[1]);
+  for (int b = 0; b < kListBufs; ++b) p->ws.slot_list[b] = reinterpret_cast<uint32_t*>(w + L.slot_list[b]);
   p->ws.n_tiles = L.n_tiles;
   uint8_t* hw = static_cast<uint8_t*>(desc->h_workspace);
-  p->h_list[0] = reinterpret_cast<uint32_t*>(hw + L.h_list[0]);
-  p->h_list[1] = reinterpret_cast<uint32_t*>(hw + L.h_list[1]);
+  for (int b = 0; b < kListBufs; ++b) p->h_list[b] = reinterpret_cast<uint32_t*>(hw + L.h_list[b]);
   p->h_counts = reinterpret_cast<uint64_t*>(hw + L.h_counts);
   p->h_status = reinterpret_cast<uint32_t*>(hw + L.h_status);
   for (int q = 0; q <= 4; ++q) p->pc.base[q] = g.bases[q];
@@ -514,6 +557,11 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
     ph.live.assign((size_t)desc->part[q].ring_slots, 0);
     ph.h_ring = static_cast<uint8_t*>(desc->part[q].h_ring);
     ph.h_meta = static_cast<uint8_t*>(desc->part[q].h_meta);
+    {
+      void* dp = nullptr;
+      if (ph.h_ring && cudaHostGetDevicePointer(&dp, ph.h_ring, 0) == cudaSuccess) ph.ring_dev = static_cast<const uint8_t*>(dp);
+      else (void)cudaGetLastError();
+    }
   }
   {
     HeadWeights& hd = p->head;
@@ -565,13 +613,7 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
   p->stats.n_entries = g.N;
   p->stats.n_free = g.N;
 
-  cudaEvent_t* evs[] = {&p->ev_staging_free[0], &p->ev_staging_free[1], &p->ev_ready[0], &p->ev_ready[1],
-                        &p->ev_staging_free[2], &p->ev_staging_free[3], &p->ev_ready[2], &p->ev_ready[3],
-                        &p->d2h[0][0].ev, &p->d2h[0][1].ev, &p->d2h[1][0].ev, &p->d2h[1][1].ev,
-                        &p->d2h[2][0].ev, &p->d2h[2][1].ev, &p->d2h[3][0].ev, &p->d2h[3][1].ev,
-                        &p->ev_h2d_done,
-                        &p->ev_list_copied[0], &p->ev_list_copied[1], &p->ev_list_free[0],
-                        &p->ev_list_free[1], &p->ev_counts};
+  std::vector<cudaEvent_t*> evs = all_events(p);
   int made = 0;
   cudaError_t e = cudaSuccess;
   for (cudaEvent_t* ev : evs) {
@@ -587,7 +629,7 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
     if (e == cudaSuccess) e = launch_head_init(p->head, p->n_head_imp, p->n_head_w, S(stream));
   }
   if (e != cudaSuccess) {
-    for (int i = 0; i < made; ++i) cudaEventDestroy(*evs[i]);
+    for (int i = 0; i < made; ++i) cudaEventDestroy(*evs[(size_t)i]);
     delete p;
     return KV_ERR_CUDA;
   }
@@ -599,14 +641,8 @@ int32_t kv_pool_destroy(kv_pool* p) {
   if (!p) return KV_ERR_INVALID_ARG;
   (void)drain_pending(p, -1, 0, ~0ull);
   if (p->events_made) {
-    cudaEvent_t evs[] = {p->ev_staging_free[0], p->ev_staging_free[1], p->ev_ready[0], p->ev_ready[1],
-                         p->ev_staging_free[2], p->ev_staging_free[3], p->ev_ready[2], p->ev_ready[3],
-                         p->d2h[0][0].ev, p->d2h[0][1].ev, p->d2h[1][0].ev, p->d2h[1][1].ev,
-                         p->d2h[2][0].ev, p->d2h[2][1].ev, p->d2h[3][0].ev, p->d2h[3][1].ev,
-                         p->ev_h2d_done,
-                         p->ev_list_copied[0], p->ev_list_copied[1], p->ev_list_free[0],
-                         p->ev_list_free[1], p->ev_counts};
-    for (cudaEvent_t ev : evs) cudaEventDestroy(ev);
+    std::vector<cudaEvent_t*> evs = all_events(p);
+    for (cudaEvent_t* ev : evs) cudaEventDestroy(*ev);
   }
   for (auto& t : p->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
   delete p;
@@ -616,7 +652,7 @@ int32_t kv_pool_destroy(kv_pool* p) {
 int32_t kv_epoch_events(kv_pool* p, const uint32_t* d_ev_entry, const uint8_t* d_ev_hit,
                         uint64_t n_events, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   if (n_events > 0 && (!d_ev_entry || !d_ev_hit || !aligned16(d_ev_entry) || !aligned16(d_ev_hit)))
     return KV_ERR_INVALID_ARG;
   KV_CUDA(p, launch_event_reduce(d_ev_entry, d_ev_hit, n_events, p->st, p->ws, S(stream)));
@@ -630,7 +666,7 @@ uint64_t* kv_epoch_counts(kv_pool* p) {
 
 int32_t kv_epoch_update(kv_pool* p, uint32_t epoch, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   KV_CUDA(p, launch_entry_update(p->st, p->desc.d_hits, p->desc.d_misses, p->desc.d_P, p->desc.alpha0,
                                  p->desc.beta0, p->ws, epoch, p->score_opt, p->head, S(stream)));
   scoring_pass_enqueued(p, epoch);
@@ -647,7 +683,7 @@ int32_t kv_epoch_score(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_entry, c
 int32_t kv_head_importance_update(kv_pool* p, int32_t q, const float* d_x, float decay, kv_stream_t stream) {
   if (!p || q < 0 || q >= p->n_parts || !d_x || !aligned16(d_x)) return KV_ERR_INVALID_ARG;
   if (!(decay >= 0.0f) || !(decay <= 1.0f)) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   KV_CUDA(p, launch_head_update(p->head, q, 0, d_x, decay, p->ws, S(stream)));
   p->head.on |= 1u << q;
   return KV_OK;
@@ -655,7 +691,7 @@ int32_t kv_head_importance_update(kv_pool* p, int32_t q, const float* d_x, float
 
 int32_t kv_set_head_multipliers(kv_pool* p, int32_t q, const float* d_mult, kv_stream_t stream) {
   if (!p || q < 0 || q >= p->n_parts || (d_mult && !aligned16(d_mult))) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   KV_CUDA(p, launch_head_update(p->head, q, 1, d_mult, 0.0f, p->ws, S(stream)));
   p->head.on |= 1u << q;
   return KV_OK;
@@ -671,7 +707,7 @@ const float* kv_head_weights(kv_pool* p, int32_t q) {
 
 int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   if (k > p->stats.n_entries - p->stats.n_free) return KV_ERR_K_TOO_LARGE;
   if (k == 0) return KV_OK;
   if (!d_victims || !aligned16(d_victims)) return KV_ERR_INVALID_ARG;
@@ -683,7 +719,7 @@ int32_t kv_epoch_score_select(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_e
                               const uint8_t* d_ev_hit, uint64_t n_events, uint64_t k, uint32_t* d_victims,
                               kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   if (n_events > 0 && (!d_ev_entry || !d_ev_hit || !aligned16(d_ev_entry) || !aligned16(d_ev_hit)))
     return KV_ERR_INVALID_ARG;
   if (k > p->stats.n_entries - p->stats.n_free) return KV_ERR_K_TOO_LARGE;
@@ -708,7 +744,7 @@ int32_t kv_epoch_score_select(kv_pool* p, uint32_t epoch, const uint32_t* d_ev_e
 int32_t kv_select_victim_blocks(kv_pool* p, uint64_t k_blocks, uint32_t* d_victims, uint64_t* h_n_victims,
                                 kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   if (h_n_victims) *h_n_victims = 0;
   if (k_blocks > p->bgeom.block_base[p->n_parts]) return KV_ERR_K_TOO_LARGE;
   if (k_blocks == 0) return KV_OK;
@@ -752,7 +788,7 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
     const uint64_t one[4] = {m, 0, 0, 0};
     return kv_demote_counted(p, d_victims, m, one, batch_bytes, compute_, copy_);
   }
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, compute_);
   if (!d_victims || !aligned16(d_victims) || m > p->stats.n_entries - p->stats.n_free)
     return KV_ERR_INVALID_ARG;
   // Several partitions and no counts from the caller: count on the device (a read-only kernel)
@@ -775,7 +811,7 @@ int32_t kv_demote(kv_pool* p, const uint32_t* d_victims, uint64_t m, uint64_t ba
 int32_t kv_demote_counted(kv_pool* p, const uint32_t* d_victims, uint64_t m, const uint64_t* counts,
                           uint64_t batch_bytes, kv_stream_t compute_, kv_stream_t copy_) {
   if (!p || (m > 0 && !counts)) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, compute_);
   if (m == 0) {
     for (int q = 0; q < 4; ++q) p->last_counts[q] = 0;
     return KV_OK;
@@ -866,11 +902,16 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
     return ok ? KV_ERR_NO_FREE_SLOT : KV_ERR_BAD_HOST_SLOT;
   }
   cudaStream_t compute = S(compute_), copy = S(copy_);
+  {
+    // an earlier promotion into this partition may still be scattering: the free list must see its result
+    const int32_t rcj = join_promotions(p, compute, q);
+    if (rcj != KV_OK) { for (uint64_t j2 = 0; j2 < m; ++j2) h.live[h_slots[j2]] = 1; return rcj; }
+  }
   const uint64_t per = batch_bytes / eb;
   const int li = p->list_turn;
-  p->list_turn ^= 1;
+  p->list_turn = (p->list_turn + 1) % kListBufs;
   auto restore = [&]() { for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 1; };
-  // the pinned list buffer of two calls ago must have been copied: normally long done
+  // the list given kListBufs calls ago must have left this pinned buffer: normally long done
   cudaError_t e = cudaEventQuery(p->ev_list_copied[li]);
   if (e == cudaErrorNotReady) {
     (void)cudaGetLastError();
@@ -907,44 +948,71 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(p->ws.slot_list[li], p->h_list[li], m * 4, cudaMemcpyHostToDevice, copy);
   if (e == cudaSuccess) e = cudaEventRecord(p->ev_list_copied[li], copy);
-  if (e == cudaSuccess) e = launch_free_list(p->st, g.base, g.base + g.n, m, p->ws, compute);
+  // this partition's free slots, ascending, in the partition's own stretch of the list scratch
+  if (e == cudaSuccess) e = launch_free_list(p->st, g.base, g.base + g.n, m, p->ws, compute, g.base);
   if (e != cudaSuccess) { restore(); return cuda_fail(p, e); }
-  for (uint64_t c0 = 0; c0 < m; c0 += per) {
+  const uint32_t* free_ids = p->ws.free_list + g.base;
+  // With P entries promoted into the partition since the pending demotion began, chunk [c0, c0+cnt)
+  // fills FREE slots number P+c0 .. P+c0+cnt-1 of the free set as it was right after that demotion.
+  // Any of those that the demotion freed is among its first P+c0+cnt victims of the partition (victims
+  // and free slots are both in ascending id order), so that much of its payload must have been
+  // packed: enqueue it, and let the copy stream wait for it (and for the free list).
+  auto ready_for = [&](uint64_t upto) -> int32_t {
+    if (p->pending.active) {
+      const int32_t rc = drain_pending(p, q, p->pending.promoted[q] + upto, ~0ull);
+      if (rc != KV_OK) return rc;
+    }
+    KV_CUDA(p, cudaEventRecord(p->ev_promote_ready, compute));
+    KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_promote_ready, 0));
+    return KV_OK;
+  };
+  // A list of short runs (a position-ordered prefetch: a block's layers lie far apart in the
+  // ring) would cost one DMA set-up per run; the gather kernel fetches such entries itself.
+  uint64_t n_runs = 0;
+  for (uint64_t j = 0; j < m; ++j) n_runs += (j == 0 || h_slots[j] != h_slots[j - 1] + 1);
+  const bool gather = h.ring_dev && m * eb < n_runs * p->gather_run_bytes;
+  // The transfers AND the scatter kernels go to the copy stream: the compute stream never waits
+  // for the host link, and pack kernels of a demotion keep flowing between them.  Transfers run
+  // one chunk ahead of the kernels (two staging buffers).
+  auto h2d_chunk = [&](uint64_t c0) -> int32_t {
     const uint64_t cnt = (m - c0 < per) ? m - c0 : per;
-    const int b = 2 + p->promote_turn;
-    p->promote_turn ^= 1;
-    KV_CUDA(p, cudaStreamWaitEvent(copy, p->ev_staging_free[b], 0));
-    // runs of consecutive ring slots become single copies
+    uint8_t* stage = p->staging[2 + ((c0 / per) & 1u)];
     uint64_t j = 0;
-    while (j < cnt) {
+    while (j < cnt) {   // runs of consecutive ring slots become single copies
       const uint64_t s0 = h_slots[c0 + j];
       uint64_t len = 1;
       while (j + len < cnt && h_slots[c0 + j + len] == s0 + len) ++len;
-      KV_CUDA(p, cudaMemcpyAsync(p->staging[b] + j * eb, h.h_ring + s0 * eb, len * eb,
-                                 cudaMemcpyHostToDevice, copy));
+      KV_CUDA(p, cudaMemcpyAsync(stage + j * eb, h.h_ring + s0 * eb, len * eb, cudaMemcpyHostToDevice, copy));
       j += len;
     }
-    KV_CUDA(p, cudaEventRecord(p->ev_ready[b], copy));
-    // With P entries promoted into the partition since the pending demotion began, this chunk
-    // fills FREE slots number P+c0 .. P+c0+cnt-1 of the free set as it was right after that
-    // demotion.  Any of those that the demotion freed is among its first P+c0+cnt victims of the
-    // partition (victims and free slots are both in ascending id order), so that much of its
-    // payload must have been packed: enqueue it first.
-    if (p->pending.active) {
-      const int32_t rc = drain_pending(p, q, p->pending.promoted[q] + c0 + cnt, ~0ull);
+    return KV_OK;
+  };
+  if (!gather) {
+    const int32_t rc = h2d_chunk(0);
+    if (rc != KV_OK) return rc;
+  }
+  for (uint64_t c0 = 0; c0 < m; c0 += per) {
+    const uint64_t cnt = (m - c0 < per) ? m - c0 : per;
+    if (!gather && c0 + per < m) {
+      const int32_t rc = h2d_chunk(c0 + per);
       if (rc != KV_OK) return rc;
     }
-    KV_CUDA(p, cudaStreamWaitEvent(compute, p->ev_ready[b], 0));
-    {
-      TimedScope ts(p, 1, cnt * eb, compute);
-      KV_CUDA(p, launch_unpack_tma(g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, p->ws.free_list + c0, cnt,
-                                   p->staging[b], p->ws, compute));
-    }
-    KV_CUDA(p, cudaEventRecord(p->ev_staging_free[b], compute));
+    const int32_t rc = ready_for(c0 + cnt);
+    if (rc != KV_OK) return rc;
+    TimedScope ts(p, gather ? 2 : 1, cnt * eb, copy);
+    if (gather)
+      KV_CUDA(p, launch_gather_promote(g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, free_ids + c0, cnt,
+                                       h.ring_dev, p->ws, copy));
+    else
+      KV_CUDA(p, launch_unpack_tma(g, p->st, p->desc.d_loc, p->ws.slot_list[li] + c0, free_ids + c0, cnt,
+                                   p->staging[2 + ((c0 / per) & 1u)], p->ws, copy));
   }
-  KV_CUDA(p, cudaEventRecord(p->ev_list_free[li], compute));
+  KV_CUDA(p, cudaEventRecord(p->ev_list_free[li], copy));
   KV_CUDA(p, cudaEventRecord(p->ev_h2d_done, copy));
+  KV_CUDA(p, cudaEventRecord(p->ev_promoted[q], copy));
+  p->promote_open[q] = true;
   p->h2d_valid = true;
+  if (gather) p->stats.gathered += m;
   if (p->pending.active) p->pending.promoted[q] += m;
   for (uint64_t j = 0; j < m; ++j) h.live[h_slots[j]] = 0;
   h.n_live -= m;
@@ -958,7 +1026,7 @@ int32_t kv_promote(kv_pool* p, int32_t q, const uint64_t* h_slots, uint64_t m, u
 int32_t kv_admit(kv_pool* p, uint32_t epoch, float decay, const uint8_t* d_new_pairs, uint64_t n_new_pairs,
                  int32_t fill_pattern, uint64_t* n_admitted, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   const uint64_t n_free = p->stats.n_free;
   if (n_admitted) *n_admitted = 0;
   if (n_free == 0) return KV_OK;
@@ -1004,7 +1072,7 @@ int32_t kv_last_demote_counts(const kv_pool* p, uint64_t* counts4) {
 
 int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) {
   if (!p || !status_bits) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   KV_CUDA(p, cudaMemcpyAsync(p->h_status, p->ws.status, 4, cudaMemcpyDeviceToHost, S(stream)));
   KV_CUDA(p, cudaMemsetAsync(p->ws.status, 0, 4, S(stream)));
   KV_CUDA(p, cudaStreamSynchronize(S(stream)));
@@ -1014,7 +1082,7 @@ int32_t kv_device_status(kv_pool* p, kv_stream_t stream, uint32_t* status_bits) 
 
 int32_t kv_hash_entries(kv_pool* p, const uint32_t* d_ids, uint64_t m, uint8_t* d_digests, kv_stream_t stream) {
   if (!p) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   if (m == 0) return KV_OK;
   if (!d_digests || !aligned16(d_digests) || (d_ids && !aligned16(d_ids))) return KV_ERR_INVALID_ARG;
   if (!d_ids && m > p->stats.n_entries) return KV_ERR_INVALID_ARG;
@@ -1070,6 +1138,12 @@ int32_t kv_flush(kv_pool* p) {
   return KV_OK;
 }
 
+int32_t kv_set_gather_threshold(kv_pool* p, uint64_t run_bytes) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  p->gather_run_bytes = run_bytes;
+  return KV_OK;
+}
+
 int32_t kv_set_deferred_packing(kv_pool* p, int32_t on) {
   if (!p) return KV_ERR_INVALID_ARG;
   KV_DRAIN_ALL(p);
@@ -1085,7 +1159,7 @@ int32_t kv_set_select_variant(kv_pool* p, int32_t variant) {
 
 int32_t kv_selection_stats(kv_pool* p, kv_stream_t stream, kv_select_stats* out) {
   if (!p || !out) return KV_ERR_INVALID_ARG;
-  KV_DRAIN_ALL(p);
+  KV_SETTLE(p, stream);
   KV_CUDA(p, cudaMemcpyAsync(p->h_sel_stats, &p->ws.sel->n_select, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost,
                              S(stream)));
   KV_CUDA(p, cudaStreamSynchronize(S(stream)));

@@ -104,6 +104,10 @@ struct SelectScalars {
   // persistent selection on a pool of several partitions: (below tau, equal to tau) counts of
   // the entries before partition boundary q + 1 inside the slice of the CTA that holds it
   uint2 bsplit[3];
+  // width of the next selection's bracket: its 2,048 bins are 2^hint_shift keys wide (7..11);
+  // hint_resid is a slowly decaying maximum of how far tau landed from where the hint put it
+  uint32_t hint_shift;
+  uint32_t hint_resid;
 };
 
 // Sliding window of per-epoch (pair, hit) counts for the confidence-weighted
@@ -163,7 +167,7 @@ struct Workspace {
   uint2* tile_counts;          // [n_tiles] (less, equal) or (free, 0)
   uint2* tile_offsets;         // [n_tiles] exclusive prefix of tile_counts
   uint32_t* free_list;         // [max(N, ..)] ascending ids of FREE entries
-  uint32_t* slot_list[2];      // [max_promote] promote lists (ring slots)
+  uint32_t* slot_list[8];      // [max_promote] promote lists (ring slots), used in turn
   unsigned long long* part_counts;  // [4] victims per partition
   uint32_t n_tiles;
 };
@@ -221,9 +225,9 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
 cudaError_t launch_select_blocks(const EntryState& st, const BlockGeom& bg, uint64_t k_blocks,
                                  uint32_t* d_victims, const Workspace& ws, cudaStream_t s,
                                  unsigned long long* h_entry_counts);
-// ascending ids of FREE entries in [lo, hi), at most `limit` of them, into ws.free_list
+// ascending ids of FREE entries in [lo, hi), at most `limit` of them, into ws.free_list + out_offset
 cudaError_t launch_free_list(const EntryState& st, uint64_t lo, uint64_t hi, uint64_t limit,
-                             const Workspace& ws, cudaStream_t s);
+                             const Workspace& ws, cudaStream_t s, uint64_t out_offset = 0);
 // victims per partition of an ascending list into pc.d_counts (and pc.h_counts)
 cudaError_t launch_partition_counts(const uint32_t* d_victims, uint64_t m, const PartCounts& pc,
                                     cudaStream_t s);
@@ -253,6 +257,11 @@ cudaError_t launch_pack_tma(const PartGeom& g, const EntryState& st, uint32_t* l
 cudaError_t launch_unpack_tma(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
                               const uint32_t* free_ids, uint64_t count, const uint8_t* staging,
                               const Workspace& ws, cudaStream_t s);
+// the same scatter with the entries fetched by the kernel itself from the pinned ring (ring_dev:
+// the address at which the device sees it): for lists of short runs
+cudaError_t launch_gather_promote(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* slots,
+                                  const uint32_t* free_ids, uint64_t count, const uint8_t* ring_dev,
+                                  const Workspace& ws, cudaStream_t s);
 // admits free_list[first .. first+count) of one partition
 cudaError_t launch_admit(const PartGeom& g, const EntryState& st, uint32_t* loc, const uint32_t* free_ids,
                          uint64_t first, uint64_t count, uint64_t first_tag, const uint8_t* new_pairs,

@@ -23,13 +23,19 @@ class EpochRunner:
             staging_bytes = self.batch_bytes + (self.batch_bytes // min(p.entry_bytes for p in workload.parts) + 2) * 24 + 64
         staging_bytes = max(int(staging_bytes), max_eb + 256)
         self.pool = B.Pool(workload.parts, workload.n_tags, workload.alpha0, workload.beta0,
-                           staging_bytes=staging_bytes, max_promote=max(workload.N, 4),
+                           staging_bytes=staging_bytes, max_promote=self.max_promote(workload),
                            host_meta=host_meta, device=device)
         self.fill_pattern = fill_pattern
         self.k = workload.k
         self.victims = torch.empty(max(self.k, 4), dtype=torch.int32, device=self.pool.device)
         self.fresh = None      # entries admitted by the last admit() (input of the next epoch's trace)
         self.check(self.admit(0, key=INITIAL_EPOCH_KEY), "initial kv_admit")
+
+    @staticmethod
+    def max_promote(w):
+        """Longest promote list a harness call gives the pool: the workload's promotion share of
+        its largest partition (never less than 4,096, for tests that promote by hand)."""
+        return max(4096, int(w.promote_frac * max(p.n_entries for p in w.parts)) + 16)
 
     def next_events(self, epoch):
         """Draws the epoch's trace from the pool's current pair ids and last admissions."""
@@ -65,6 +71,18 @@ class EpochRunner:
         self._keep = d_pairs   # the kernel reads it asynchronously
         return rc
 
+    def demote(self, k=None):
+        """Demotes the victims of the last selection.  A pool of several partitions needs the
+        victims per partition on the host: the selection left them in pinned memory, so the
+        caller waits for its own stream here and passes them on (the library itself never
+        blocks on this path)."""
+        k = self.k if k is None else k
+        p = self.pool
+        if len(self.w.parts) == 1 or k == 0:
+            return p.kv_demote(self.victims, k, self.batch_bytes)
+        p.compute.synchronize()
+        return p.kv_demote_counted(self.victims, k, p.kv_victim_counts(), self.batch_bytes)
+
     def promote_lists(self, epoch):
         """Per-partition promote lists for the state the ring is in right now."""
         counts = self.pool.kv_last_demote_counts()
@@ -84,7 +102,7 @@ class EpochRunner:
         else:
             self.check(p.kv_epoch_score(epoch, d_ev_entry, d_ev_hit, n_events), "kv_epoch_score")
             self.check(p.kv_select_victims(self.k, self.victims), "kv_select_victims")
-        self.check(p.kv_demote(self.victims, self.k, self.batch_bytes), "kv_demote")
+        self.check(self.demote(), "kv_demote")
         if promote_lists is None:
             promote_lists = self.promote_lists(epoch)
         for q, lst in enumerate(promote_lists):

@@ -94,7 +94,7 @@ class Workload:
     beta0: float = 1.0
     epochs: int = 50
     pair_weights: Optional[np.ndarray] = None   # None = uniform over the 16 pairs
-    promote_style: str = "runs"                 # "recent" or "runs"
+    promote_style: str = "runs"                 # "recent", "runs" or "position"
     max_run: int = 2048
     _static: dict = field(default_factory=dict, repr=False)
 
@@ -195,6 +195,8 @@ class Workload:
             if int(live.sum()) - int(live[idx].sum()) >= m:
                 live = live.copy()
                 live[idx] = 0
+        if self.promote_style == "position":
+            return self._position_list(epoch, q, m, cursor, live, just_written)
         if self.promote_style == "recent":
             # the m most recently written live slots, oldest first
             order = (cursor - 1 - np.arange(R)) % R
@@ -223,6 +225,51 @@ class Workload:
             rest = np.flatnonzero((live != 0) & ~taken)[: m - n]
             out.append(rest)
         return np.concatenate(out)[:m].astype(np.uint64)
+
+
+def _position_list(self, epoch, q, m, cursor, live, just_written):
+    """Position-ordered prefetch (long-context pool): round-robin over 64 sequences, for each
+    the next window of 128 blocks, ordered by (position, layer, head).  A demotion fills
+    the ring in (layer, block, head) order, so the part of the ring older than this
+    epoch's demotion is read as n_layers stripes of equal length in which a block's heads
+    are neighbours and its layers lie one stripe apart: the list comes out as runs of
+    `heads` slots, a stripe apart -- the fragmented case of kv_promote."""
+    p = self.parts[q]
+    L, H, R = p.n_layers, p.heads, live.size
+    seg_len = R - min(just_written, R)
+    per_layer = seg_len // L // H * H
+    n_blocks = per_layer // H
+    if n_blocks == 0:
+        return np.flatnonzero(live)[:m].astype(np.uint64)
+    n_seq, win = 64, 128
+    bps = max(1, n_blocks // n_seq)                     # blocks of one sequence's stripe
+    n_win = -(-bps // win)
+    lh = (np.arange(L, dtype=np.int64)[:, None] * per_layer + np.arange(H, dtype=np.int64)[None, :]).reshape(-1)
+    out, n = [], 0
+    for wi in range(n_win):
+        w0 = ((epoch + wi) % n_win) * win
+        blocks = (np.arange(n_seq, dtype=np.int64)[:, None] * bps
+                  + (w0 + np.arange(win, dtype=np.int64))[None, :] % bps).reshape(-1)
+        blocks = blocks[blocks < n_blocks]
+        slots = (cursor + blocks[:, None] * H + lh[None, :]).reshape(-1) % R
+        slots = slots[live[slots] != 0]
+        out.append(slots)
+        n += slots.size
+        if n >= m:
+            break
+    lst = np.concatenate(out) if out else np.zeros(0, np.int64)
+    _, first = np.unique(lst, return_index=True)          # (windows of short stripes can overlap)
+    lst = lst[np.sort(first)][:m]
+    if lst.size < m:      # a ring still filling up: the rest from whatever else is live, oldest first
+        taken = np.zeros(R, dtype=bool)
+        taken[lst] = True
+        order = (cursor + np.arange(R, dtype=np.int64)) % R
+        rest = order[(live[order] != 0) & ~taken[order]][: m - lst.size]
+        lst = np.concatenate([lst, rest])
+    return lst.astype(np.uint64)
+
+
+Workload._position_list = _position_list
 
 
 # ---- trace styles (each returns local entry ids of one partition) ----------
@@ -397,17 +444,17 @@ def config(i: int, scale: float = 1.0, ring_slots: Optional[int] = None,
         w = Workload("llama3-8b-chat", [gqa(32, 32, 8, 128, 16, nb(12288), ring(1 << 20), "chat")],
                      0.10, 0.03, seed=1)
     elif i == 3:
-        w = Workload("llama3-70b-longctx", [gqa(80, 64, 8, 128, 16, nb(18432), ring(1 << 21), "long")],
-                     0.15, 0.10, seed=2, epochs=10, max_run=81920)
+        w = Workload("llama3-70b-longctx", [gqa(80, 64, 8, 128, 16, nb(18432), ring(1 << 22), "long")],
+                     0.15, 0.10, seed=2, epochs=10, max_run=81920, promote_style="position")
     elif i == 4:
         w = Workload("deepseek-v3-agentic", [mla(61, 512, 64, 64, nb(14912), ring(1 << 17), "agentic")],
                      0.10, 0.05, seed=3, epochs=40)
     elif i == 5:
         blocks = nb(10720)
-        parts = [mha(32, 32, 128, 16, blocks, ring(3 << 19), "mixed"),
-                 gqa(80, 64, 8, 128, 16, blocks, ring(1 << 20), "mixed"),
-                 mqa(32, 32, 128, 16, blocks, ring(1 << 17), "mixed"),
-                 mla(61, 512, 64, 16, blocks, ring(1 << 17), "mixed")]
+        parts = [mha(32, 32, 128, 16, blocks, ring(3 << 20), "mixed"),
+                 gqa(80, 64, 8, 128, 16, blocks, ring(1 << 21), "mixed"),
+                 mqa(32, 32, 128, 16, blocks, ring(1 << 18), "mixed"),
+                 mla(61, 512, 64, 16, blocks, ring(1 << 18), "mixed")]
         w = Workload("mixed-fleet", parts, 0.10, 0.03, seed=4, epochs=8)
         w.pair_weights = np.random.default_rng([4, 77]).dirichlet(np.full(16, 0.5))
     else:

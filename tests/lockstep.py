@@ -37,7 +37,7 @@ def oracle_admit(w, pool, epoch, key=None):
 class Lockstep:
     def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True,
                  policy=0, blend=None, deferred=False, fused=False, heads=None, lazy=False,
-                 split_promote=1):
+                 split_promote=1, counted=False, select_variant=1):
         self.w = w
         self.payload = payload
         self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
@@ -46,11 +46,13 @@ class Lockstep:
         self.deferred = deferred
         self.fused = fused   # score and select through the single fused call
         self.split_promote = split_promote   # each partition's promote list goes in this many calls
+        self.counted = counted   # pools of several partitions: demote with the counts the selection left
         # heads = (decay, every): importance matrices of all partitions updated before every
         # epoch's scoring, multipliers set on epochs divisible by `every` and reset on the next
         self.heads = heads
         if deferred:
             assert self.gpu.pool.kv_set_deferred_packing(True) == 0
+        assert self.gpu.pool.kv_set_select_variant(select_variant) == 0
         # room for any k a test may ask for
         self.gpu.victims = self.gpu.torch.empty(max(w.N, 4), dtype=self.gpu.torch.int32,
                                                 device=self.gpu.pool.device)
@@ -183,14 +185,28 @@ class Lockstep:
         else:
             rc, v = o.select_victim_blocks(k_blocks)
             assert rc == O.OK
-            rc, k = g.pool.kv_select_victim_blocks(k_blocks, g.victims)
-            g.check(rc, "kv_select_victim_blocks")
+            if self.counted:      # no place for the count: the call must not block
+                rc, _ = g.pool.kv_select_victim_blocks(k_blocks, g.victims, wait=False)
+                g.check(rc, "kv_select_victim_blocks")
+                g.pool.sync()
+                per_part = g.pool.kv_victim_counts() if len(w.parts) > 1 else [len(v)]
+                k = sum(per_part)
+            else:
+                rc, k = g.pool.kv_select_victim_blocks(k_blocks, g.victims)
+                g.check(rc, "kv_select_victim_blocks")
             assert k == len(v), (k, len(v))
         g.pool.sync()
         got = g.victims[:k].cpu().numpy().view(np.uint32)
         assert np.array_equal(got, v), "epoch %d victims" % e
         assert o.demote(v) == O.OK
-        g.check(g.pool.kv_demote(g.victims, k, g.batch_bytes), "kv_demote")
+        if self.counted and len(w.parts) > 1:
+            # the counts the selection left in pinned memory (the stream has been synchronised above)
+            counts = g.pool.kv_victim_counts()
+            inf = [o.info(q) for q in range(len(w.parts))]
+            assert counts == [int(((v >= i["base"]) & (v < i["base"] + i["n"])).sum()) for i in inf], counts
+            g.check(g.pool.kv_demote_counted(g.victims, k, counts, g.batch_bytes), "kv_demote_counted")
+        else:
+            g.check(g.pool.kv_demote(g.victims, k, g.batch_bytes), "kv_demote")
         if not self.deferred:   # (a status read would enqueue the deferred chunks and undo the interleaving)
             self.compare_state("epoch %d demote" % e, scores=False)
             self.compare_ring("epoch %d demote" % e)
