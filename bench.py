@@ -48,7 +48,7 @@ PACK_KERNEL_NAME = "move_tma_kernel<true> (pack)"
 # select_persistent_kernel<true>) from ncu, bytes per launch pair, keyed by pool number: captured
 # at the pool's full entry count with --tiny-entries (these kernels never touch block payload).
 # None = no capture of the kernels as they stand.
-NCU_SCORE_SELECT_TRAFFIC = {}
+NCU_SCORE_SELECT_TRAFFIC = {5: 547.2e6, 3: 423.7e6}
 
 
 def parse():
@@ -84,7 +84,7 @@ def parse():
     ap.add_argument("--tiny-entries", action="store_true",
                     help="32-64 byte blocks (same entry count and traces): for profiling scoring/selection")
     ap.add_argument("--promote-run", type=int, default=None,
-                    help="promote lists made of runs of at most this many consecutive ring slots at seeded starts "
+                    help="promote lists made of runs of exactly this many consecutive ring slots at seeded places "
                          "(instead of the pool's own list style)")
     ap.add_argument("--gather-kb", type=int, default=None,
                     help="promote lists whose runs average less than this many KiB go through the gather kernel "
@@ -454,7 +454,7 @@ def main():
     cfg, scale, w, chosen_because = choose_workload(args, torch, W, dev)
     w.seed = w.seed + 1000 * rank     # every rank owns its own pool and trace (weak scaling)
     if args.promote_run is not None:
-        w.promote_style, w.max_run = "runs", args.promote_run
+        w.promote_style, w.max_run = "aligned-runs", args.promote_run
     w.epochs = args.warmup + args.steps + 12   # block handles for every epoch this run admits (timed, e2e, breakdown)
     link = hostlink_probe(torch, dev) if rank == 0 and not args.no_hostlink else None
     runner = EpochRunner(w, batch_bytes=args.batch_mb << 20, fill_pattern=True, host_meta=True,
@@ -678,7 +678,7 @@ def main():
                    "events_per_step": tot["events"] // K, "pool_bytes": sum(p.slab_bytes for p in w.parts),
                    "entry_bytes": [p.entry_bytes for p in w.parts], "batch_bytes": runner.batch_bytes,
                    "deferred_packing": not args.no_deferred_packing,
-                   "promote_lists": w.promote_style + ("" if w.promote_style != "runs" else " of <= %d slots" % w.max_run),
+                   "promote_lists": w.promote_style + ("" if "runs" not in w.promote_style else " of %d slots" % w.max_run),
                    "fused_score_select": not (args.no_fused or dist_on),
                    "head_weights": bool(args.head_weights),
                    "ring_slots": [p.ring_slots for p in w.parts], "scale": scale,

@@ -284,9 +284,17 @@ class Pool:
         self.slabs, self.rings, self.metas = [], [], []
         d = kv_pool_desc()
         d.n_partitions = len(self.parts)
+        self.entry_bytes = []
         for q, p in enumerate(self.parts):
-            slab = torch.empty(p.slab_bytes, dtype=torch.uint8, device=dev)
-            ring = torch.empty(max(p.ring_slots * p.entry_bytes, 16), dtype=torch.uint8, pin_memory=True)
+            # sizes come from the library's own sizing calls (Eq. "unified"), not from the workload
+            m = model_desc(p)
+            eb = kv_entry_bytes(m, p.block_tokens)
+            per_block = kv_size_bytes(m, p.block_tokens, per_layer=True)
+            if eb <= 0 or per_block <= 0:
+                raise KVError(min(eb, per_block), "kv_entry_bytes / kv_size_bytes")
+            self.entry_bytes.append(eb)
+            slab = torch.empty(p.n_layers * p.blocks_per_layer * per_block, dtype=torch.uint8, device=dev)
+            ring = torch.empty(max(p.ring_slots * eb, 16), dtype=torch.uint8, pin_memory=True)
             meta = (torch.zeros(max(p.ring_slots * 24, 16), dtype=torch.uint8, pin_memory=True)
                     if host_meta else None)
             self.slabs.append(slab)

@@ -14,8 +14,6 @@
 //
 // Every wait is bounded: a lane that gives up sets KV_DEV_WAIT_EXPIRED in the
 // device status word, drains its own stores and leaves.
-#include <cstdlib>
-
 #include "kvtier_internal.cuh"
 
 namespace kvt {
@@ -303,9 +301,7 @@ move_tma_kernel(const MoveArgs a) {
 // transfer per run spends its time on set-up.  This kernel fetches the listed entries
 // itself, through the address at which the device sees the pinned ring, and writes them
 // straight into their paged slots: no staging buffer, no per-run transfer.  A warp moves
-// one piece of up to 2 KB at a time with four 16-byte loads in flight per lane; with two
-// blocks of eight warps per SM several MB are in flight, which a host link with a round
-// trip of a few microseconds needs.
+// one piece of up to 2 KB at a time with four 16-byte loads in flight per lane.
 constexpr uint32_t kGatherPiece = 2048;   // 32 lanes x 4 x 16 bytes
 constexpr uint32_t kGatherThreads = 256;
 
@@ -353,8 +349,10 @@ cudaError_t launch_gather_promote(const PartGeom& g, const EntryState& st, uint3
   MoveArgs a{g, st, loc, free_ids, slots, count, 0, nullptr, ~0ull, ws.status, kMoveAll};
   const uint64_t pieces = count * ((g.chunk_bytes + kGatherPiece - 1) / kGatherPiece) * g.n_chunks;
   uint64_t blocks = (pieces * 32 + kGatherThreads - 1) / kGatherThreads;
-  uint64_t cap = 32;
-  if (const char* e = std::getenv("KVTIER_GATHER_BLOCKS")) cap = (uint64_t)std::atoi(e);
+  // 32 blocks keep 512 KB of reads in flight, several round trips' worth of the host link; more
+  // blocks crowd out the D2H transfers of a demotion running at the same time without moving more
+  // (measured: both directions together carry ~63 GB/s whatever the split)
+  const uint64_t cap = 32;
   if (blocks > cap) blocks = cap;
   gather_promote_kernel<<<(unsigned)(blocks ? blocks : 1), kGatherThreads, 0, s>>>(a, ring_dev);
   count_launches(1);

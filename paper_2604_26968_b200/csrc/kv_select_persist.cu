@@ -39,7 +39,6 @@
 // disappears.  The event reduction stays a launch of its own ahead of it: its
 // scattered gathers and atomics ran 2.5x slower inside this kernel when that was
 // tried, and a grid barrier costs about what the launch boundary does.
-#include <cstdlib>
 #include <mutex>
 #include <type_traits>
 
@@ -923,7 +922,6 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   // of the shared memory stays with the L1, whose lines hold the loads in flight of the streaming
   // entry pass.
   uint64_t slots = (a.per + kPThreads - 1) / kPThreads;   // as many as the thread sees keys, up to the maximum
-  if (const char* e = std::getenv("KVTIER_SELECT_SLOTS")) slots = (uint64_t)std::atoi(e);
   if (slots < 10) slots = 10;   // (two stages of the re-reading passes fit)
   if (slots > kPSlotsMax) slots = kPSlotsMax;
   a.slots = (uint32_t)slots;

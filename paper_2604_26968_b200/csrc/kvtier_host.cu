@@ -102,7 +102,7 @@ struct kv_pool {
   int demote_turn = 0, promote_turn = 0, list_turn = 0;
   int last_cuda_error = 0;
   ScoreOptions score_opt;   // eviction policy and confidence blend
-  uint64_t gather_run_bytes = 256u << 10;   // promote lists whose runs average less go through the gather kernel
+  uint64_t gather_run_bytes = 1u << 20;    // promote lists whose runs average less go through the gather kernel
   // promotions run their kernels on the copy stream they are given; the compute stream joins
   // them (waits for ev_promoted) before the next kernel that reads what they wrote
   cudaEvent_t ev_promote_ready, ev_promoted[4];

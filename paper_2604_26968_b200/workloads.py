@@ -94,7 +94,7 @@ class Workload:
     beta0: float = 1.0
     epochs: int = 50
     pair_weights: Optional[np.ndarray] = None   # None = uniform over the 16 pairs
-    promote_style: str = "runs"                 # "recent", "runs" or "position"
+    promote_style: str = "runs"                 # "recent", "runs", "position" or "aligned-runs"
     max_run: int = 2048
     _static: dict = field(default_factory=dict, repr=False)
 
@@ -202,6 +202,8 @@ class Workload:
             order = (cursor - 1 - np.arange(R)) % R
             picked = order[live[order] != 0][:m]
             return picked[::-1].astype(np.uint64)
+        if self.promote_style == "aligned-runs":
+            return self._aligned_runs(epoch, q, m, live)
         r = self.rng(epoch, 3 + q)
         taken = np.zeros(R, dtype=bool)
         out = []
@@ -269,7 +271,23 @@ def _position_list(self, epoch, q, m, cursor, live, just_written):
     return lst.astype(np.uint64)
 
 
+def _aligned_runs(self, epoch, q, m, live):
+    """Runs of exactly max_run consecutive live slots at seeded places: the ring is cut into
+    rows of max_run slots, every second row is a candidate (so that two chosen runs never
+    touch), and a seeded shuffle of the fully live candidates gives the list.  For timing
+    kv_promote against the run length; built without a Python loop per run."""
+    run, R = int(self.max_run), live.size
+    rows = R // run
+    full = (live[:rows * run].reshape(rows, run) != 0).all(axis=1)
+    cand = np.flatnonzero(full[::2]) * 2
+    self.rng(epoch, 3 + q).shuffle(cand)
+    cand = cand[: -(-m // run)]
+    lst = (cand[:, None].astype(np.int64) * run + np.arange(run, dtype=np.int64)[None, :]).reshape(-1)[:m]
+    return lst.astype(np.uint64)
+
+
 Workload._position_list = _position_list
+Workload._aligned_runs = _aligned_runs
 
 
 # ---- trace styles (each returns local entry ids of one partition) ----------
