@@ -15,6 +15,8 @@
 //     Bayesian-reuse section exactly (Eq. "reuse").
 //   * the EMA recurrence, the product score, the per-(layer, head) importance
 //     weighting (recurrence, group maximum, multipliers: okv_head_importance_update),
+//     the per-layer prefetch window and the position-ordered prefetch list
+//     (okv_prefetch_window_update, okv_prefetch_list),
 //     the ring organisation of the host
 //     tier, the free-slot rule of promotion and the lazy decay of promoted
 //     entries (okv_set_lazy_decay) are NOT printed in the paper (it withholds
@@ -33,6 +35,7 @@
 // Build: see oracle/build.py (g++ -std=c++17 -shared -fPIC).
 
 #include <algorithm>
+#include <cmath>
 #include <cstdint>
 #include <cstring>
 #include <limits>
@@ -162,6 +165,10 @@ struct Part {
   std::vector<float> h_imp;     // [L][QH] importance matrix
   std::vector<float> h_mult;    // [L][H] task-transition multipliers
   std::vector<float> h_w;       // [L][H] weight of a KV head: group maximum x multiplier
+  // per-layer prefetch window (see okv_prefetch_window_update)
+  std::vector<float> pf_span;     // [L] EMA of the observed attention span, in tokens
+  std::vector<uint32_t> pf_win;   // [L] window in blocks
+  uint32_t pf_max;                // most blocks a window may have
 };
 
 struct Stats {
@@ -221,6 +228,17 @@ void copy_image_to_entry(Part& pt, int64_t local, const uint8_t* image) {
   for (int c = 0; c < pt.n_chunks; ++c)
     std::memcpy(pt.slab.data() + chunk_offset(pt, local, c), image + c * pt.chunk_bytes,
                 (size_t)pt.chunk_bytes);
+}
+
+// w[l] = min(w_max, max(1, ceil(S[l] / block_tokens))): one IEEE division, the ceiling exact.
+void recompute_windows(Part& pt) {
+  for (int64_t l = 0; l < pt.L; ++l) {
+    const float q = pt.pf_span[(size_t)l] / (float)pt.d.block_tokens;
+    double c = std::ceil((double)q);
+    if (c < 1.0) c = 1.0;
+    if (c > (double)pt.pf_max) c = (double)pt.pf_max;
+    pt.pf_win[(size_t)l] = (uint32_t)c;
+  }
 }
 
 // Weight of KV head (l, h): the maximum importance over the query heads that
@@ -321,6 +339,10 @@ void* okv_create(int32_t n_parts, const PartDesc* parts, float alpha0, float bet
     pt.head_weights = false;
     pt.h_imp.assign((size_t)(pt.L * pt.QH), 1.0f);
     pt.h_mult.assign((size_t)(pt.L * pt.H), 1.0f);
+    pt.pf_max = 65535;
+    pt.pf_span.assign((size_t)pt.L, 2048.0f);
+    pt.pf_win.assign((size_t)pt.L, 0);
+    recompute_windows(pt);
     pt.h_w.assign((size_t)(pt.L * pt.H), 1.0f);
     base += pt.n;
   }
@@ -509,6 +531,93 @@ int32_t okv_set_head_multipliers(void* h, int32_t q, const float* mult) {
   for (int64_t i = 0; i < n; ++i) pt.h_mult[(size_t)i] = mult ? mult[i] : 1.0f;
   pt.head_weights = true;
   recompute_head_weights(pt);
+  return OK;
+}
+
+// Per-layer prefetch window (RoPE-aware prefetching section: when a sequence is at
+// position n, blocks covering positions [n, n+w] are promoted ahead of use, and the
+// window w adapts per layer -- narrow for local-attention layers, wide for
+// global-attention layers).  The paper prints neither how w adapts nor its unit
+// [reading]:
+//   S[l] <- d*S[l] + (1-d)*x[l]      x[l] = attention span observed in layer l this
+//                                    step, in tokens (binary32, each operation
+//                                    rounded once); S starts at 2,048 tokens;
+//   w[l] = min(w_max, max(1, ceil(S[l] / block_tokens)))   blocks.
+// x: L observations (>= 0, finite).
+int32_t okv_prefetch_window_update(void* h, int32_t q, const float* x, float d) {
+  Pool* p = static_cast<Pool*>(h);
+  if (q < 0 || q >= p->n_parts || !x || !(d >= 0.0f) || !(d <= 1.0f)) return ERR_INVALID_ARG;
+  Part& pt = p->part[q];
+  for (int64_t l = 0; l < pt.L; ++l)
+    if (!(x[l] >= 0.0f) || !(x[l] <= std::numeric_limits<float>::max())) return ERR_INVALID_ARG;
+  for (int64_t l = 0; l < pt.L; ++l) {
+    float t1 = d * pt.pf_span[(size_t)l];
+    float t2 = 1.0f - d;
+    float t3 = t2 * x[l];
+    pt.pf_span[(size_t)l] = t1 + t3;
+  }
+  recompute_windows(pt);
+  return OK;
+}
+
+// Sets every layer's span to `tokens` (>= 0, finite) and the cap to max_blocks (>= 1).
+int32_t okv_set_prefetch_window(void* h, int32_t q, float tokens, uint32_t max_blocks) {
+  Pool* p = static_cast<Pool*>(h);
+  if (q < 0 || q >= p->n_parts || !(tokens >= 0.0f) || !(tokens <= std::numeric_limits<float>::max()) ||
+      max_blocks < 1)
+    return ERR_INVALID_ARG;
+  Part& pt = p->part[q];
+  pt.pf_max = max_blocks;
+  for (int64_t l = 0; l < pt.L; ++l) pt.pf_span[(size_t)l] = tokens;
+  recompute_windows(pt);
+  return OK;
+}
+
+// which: 0 spans (float [L]), 1 windows (uint32 [L])
+void* okv_prefetch_array(void* h, int32_t q, int32_t which) {
+  Pool* p = static_cast<Pool*>(h);
+  if (q < 0 || q >= p->n_parts) return nullptr;
+  Part& pt = p->part[q];
+  return which == 0 ? (void*)pt.pf_span.data() : which == 1 ? (void*)pt.pf_win.data() : nullptr;
+}
+
+// The prefetch list of one sequence (same section): table[(pb*L + l)*H + h] is the
+// block handle (tag) of the sequence's block at position-block pb, layer l, KV head h,
+// for pb in [0, n_pos).  With the sequence at position-block pos0, layer l wants the
+// w[l] blocks at distance 0 .. w[l]-1 from pos0: pb = pos0 + dist when dir > 0 (the
+// positions [n, n+w] the prefetcher requests), pb = pos0 - dist when dir < 0 (the
+// positions [n-w, n] the section names as the likeliest to be read next) [reading: the
+// section gives both ranges; the caller picks].  Those blocks that sit in the host tier
+// are listed by their ring slot, ordered by (distance, layer, head).  Handles that are
+// not cached (dropped, never admitted, >= n_tags) or already in HBM are skipped.
+// Writes at most max_out slots; *count receives how many qualified (more than max_out:
+// the list was cut).
+int32_t okv_prefetch_list(void* h, int32_t q, const uint32_t* table, uint64_t n_pos, uint64_t pos0,
+                          int32_t dir, uint64_t* out, uint64_t max_out, uint64_t* count) {
+  Pool* p = static_cast<Pool*>(h);
+  if (q < 0 || q >= p->n_parts || !count || dir == 0 || (n_pos > 0 && !table)) return ERR_INVALID_ARG;
+  if (n_pos > 0 && pos0 >= n_pos) return ERR_INVALID_ARG;
+  Part& pt = p->part[q];
+  uint64_t n = 0;
+  for (uint64_t dist = 0; n_pos > 0; ++dist) {
+    if (dir > 0 ? dist >= n_pos - pos0 : dist > pos0) break;  // left the table
+    const uint64_t pb = dir > 0 ? pos0 + dist : pos0 - dist;
+    bool any = false;   // some layer still wants this distance
+    for (int64_t l = 0; l < pt.L; ++l) {
+      if (dist >= pt.pf_win[(size_t)l]) continue;
+      any = true;
+      for (int64_t hd = 0; hd < pt.H; ++hd) {
+        const uint32_t t = table[(pb * (uint64_t)pt.L + (uint64_t)l) * (uint64_t)pt.H + (uint64_t)hd];
+        if (t >= p->loc.size()) continue;
+        const uint32_t where = p->loc[t];
+        if (where == NONE || !(where & HOST_BIT)) continue;
+        if (n < max_out && out) out[n] = where & ~HOST_BIT;
+        ++n;
+      }
+    }
+    if (!any) break;
+  }
+  *count = n;
   return OK;
 }
 

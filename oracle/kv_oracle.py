@@ -84,6 +84,15 @@ def lib():
         L.okv_set_head_multipliers.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
         L.okv_head_array.restype = C.c_void_p
         L.okv_head_array.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+        L.okv_prefetch_window_update.restype = C.c_int32
+        L.okv_prefetch_window_update.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_float]
+        L.okv_set_prefetch_window.restype = C.c_int32
+        L.okv_set_prefetch_window.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_uint32]
+        L.okv_prefetch_array.restype = C.c_void_p
+        L.okv_prefetch_array.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+        L.okv_prefetch_list.restype = C.c_int32
+        L.okv_prefetch_list.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_uint64, C.c_uint64, C.c_int32,
+                                        C.c_void_p, C.c_uint64, C.c_void_p]
         L.okv_epoch_score.restype = C.c_int32
         L.okv_epoch_score.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64]
         L.okv_select_victims.restype = C.c_int32
@@ -236,6 +245,42 @@ class OraclePool:
         """'importance' [L*QH], 'multipliers' [L*H] or 'weights' [L*H] of partition q."""
         which = {"importance": 0, "multipliers": 1, "weights": 2}[name]
         return _view(lib().okv_head_array(self._h, q, which), np.float32, self._head_shape(q, min(which, 1)))
+
+    def prefetch_window_update(self, q, span, decay):
+        """EMA step of partition q's per-layer attention span (tokens); recomputes the windows."""
+        if not 0 <= q < self.n_parts:
+            return ERR_INVALID_ARG
+        span = np.ascontiguousarray(span, dtype=np.float32)
+        assert span.size == self._parts[q]["model"].n_layers
+        return lib().okv_prefetch_window_update(self._h, q, _ptr(span), float(decay))
+
+    def set_prefetch_window(self, q, tokens, max_blocks):
+        if not 0 <= q < self.n_parts:
+            return ERR_INVALID_ARG
+        return lib().okv_set_prefetch_window(self._h, q, float(tokens), int(max_blocks))
+
+    def prefetch_array(self, q, name):
+        """'span' (float32 [L], tokens) or 'window' (uint32 [L], blocks) of partition q."""
+        which = {"span": 0, "window": 1}[name]
+        n_layers = self._parts[q]["model"].n_layers
+        return _view(lib().okv_prefetch_array(self._h, q, which), (np.float32, np.uint32)[which], n_layers)
+
+    def prefetch_list(self, q, table, pos0, direction=1, max_out=None):
+        """Ring slots of the host-tier blocks inside the per-layer windows of a sequence at
+        position-block pos0; table is [n_pos][L][H] block handles.  Returns (rc, slots, count)."""
+        if not 0 <= q < self.n_parts:
+            return ERR_INVALID_ARG, None, 0
+        table = np.ascontiguousarray(table, dtype=np.uint32)
+        m = self._parts[q]["model"]
+        per = m.n_layers * self.info(q)["H"]
+        assert table.size % per == 0
+        n_pos = table.size // per
+        cap = table.size if max_out is None else int(max_out)
+        out = np.zeros(max(cap, 1), dtype=np.uint64)
+        n = C.c_uint64(0)
+        rc = lib().okv_prefetch_list(self._h, q, _ptr(table) if table.size else None, n_pos, int(pos0),
+                                     int(direction), _ptr(out), cap, C.byref(n))
+        return rc, out[:min(cap, n.value)].copy(), int(n.value)
 
     def info(self, q):
         L = lib()
