@@ -12,6 +12,8 @@
  *                      asynchronous DMA on CUDA streams)
  *   kv_promote         RoPE-aware prefetching section (asynchronous promotion
  *                      requests from lower tiers)
+ *   kv_prefetch_list   same section (the blocks covering the next positions of a
+ *                      sequence, inside a window that adapts per layer)
  * The paper withholds the EMA recurrence, the way the reuse probability and the
  * importance are combined, and the organisation of the host tier; the
  * definitions used here are stated at each function.
@@ -78,6 +80,7 @@ typedef enum { KV_AUTO = -1, KV_MHA = 0, KV_GQA = 1, KV_MQA = 2, KV_MLA = 3 } kv
 #define KV_DEV_BAD_INDEX 16u         /* an index was out of range and the access was skipped */
 #define KV_DEV_WAIT_EXPIRED 32u      /* a bounded wait inside a kernel gave up */
 #define KV_DEV_BAD_HEAD_VALUE 64u    /* a head observation or multiplier was negative or not finite */
+#define KV_DEV_BAD_SPAN_VALUE 128u   /* an attention-span observation was negative or not finite */
 
 typedef struct {
   int32_t variant;    /* kv_variant_t; KV_AUTO infers it from the fields below */
@@ -323,6 +326,49 @@ const uint64_t* kv_victim_counts(const kv_pool* pool);
  * passes it missed if kv_set_lazy_decay is on); the host slot dies. */
 int32_t kv_promote(kv_pool* pool, int32_t partition, const uint64_t* h_host_slots, uint64_t m,
                    uint64_t batch_bytes, kv_stream_t compute, kv_stream_t copy);
+
+/* Per-layer prefetch window and the prefetch list of a sequence (RoPE-aware
+ * prefetching section).  The section states that with a sequence at position n the
+ * prefetcher requests promotion of the blocks covering positions [n, n+w] (it also
+ * names [n-w, n] as the range likeliest to be read next), and that the window w
+ * adapts to the observed attention patterns: narrow for local-attention (early)
+ * layers, wide for global-attention (later) layers.  It prints no formula; the form
+ * used here, per partition q (one model):
+ *   S[l] <- decay*S[l] + (1-decay)*x[l]    x[l] = attention span observed in layer l,
+ *                                  in tokens (binary32, each operation rounded once;
+ *                                  S starts at 2,048 tokens)
+ *   w[l] = min(w_max, max(1, ceil(S[l] / block_tokens)))   blocks (w_max starts at 65,535)
+ *   kv_prefetch_window_update  d_span: device f32 [n_layers], observations >= 0 and
+ *                              finite; 0 <= decay <= 1.  If any observation is
+ *                              negative, NaN or infinite the partition keeps all its
+ *                              spans and KV_DEV_BAD_SPAN_VALUE is set.
+ *   kv_set_prefetch_window     every span of the partition = tokens (>= 0, finite),
+ *                              w_max = max_blocks (>= 1).
+ *   kv_prefetch_span / kv_prefetch_window: device addresses of S (f32 [n_layers]) and
+ *                              w (u32 [n_layers]) of partition q.
+ * kv_prefetch_list: d_table (device, u32 [n_pos][n_layers][KV heads]; one column for
+ * MLA) holds the block handles (tags) of one sequence, position-block by
+ * position-block.  With the sequence at position-block pos0 (< n_pos), layer l wants
+ * the w[l] blocks at distance 0 .. w[l]-1 from pos0, toward higher positions when
+ * direction > 0 and toward lower ones when direction < 0, as far as the table reaches.
+ * Of those, the blocks that sit in the host tier (d_loc[tag] has KV_LOC_HOST) are
+ * written to d_out_slots (device-accessible u64 [max_out]) as ring slots, ordered by
+ * (distance, layer, head): a list kv_promote accepts once it has been brought to the
+ * host.  Handles >= n_tags, dropped or never admitted, and blocks already in HBM are
+ * skipped.  *d_out_count (device-accessible u64) receives how many qualified; if that
+ * exceeds max_out only the first max_out were written.  n_pos == 0 gives count 0.
+ * Two small launches on `stream`, which first joins the pool's promotions in flight
+ * (they write d_loc); call it on the pool's compute stream.  Calls of one pool share a
+ * scratch array: do not run two of them concurrently on different streams. */
+int32_t kv_prefetch_window_update(kv_pool* pool, int32_t q, const float* d_span, float decay,
+                                  kv_stream_t stream);
+int32_t kv_set_prefetch_window(kv_pool* pool, int32_t q, float tokens, uint32_t max_blocks,
+                               kv_stream_t stream);
+const float* kv_prefetch_span(kv_pool* pool, int32_t q);
+const uint32_t* kv_prefetch_window(kv_pool* pool, int32_t q);
+int32_t kv_prefetch_list(kv_pool* pool, int32_t q, const uint32_t* d_table, uint64_t n_pos,
+                         uint64_t pos0, int32_t direction, uint64_t* d_out_slots, uint64_t max_out,
+                         uint64_t* d_out_count, kv_stream_t stream);
 
 /* How kv_promote moves the bytes.  Runs of consecutive ring slots in the list become
  * one DMA transfer each into a staging buffer, which the unpack kernel scatters; that

@@ -28,6 +28,7 @@ KV_POLICY_BAYESIAN, KV_POLICY_EMA, KV_POLICY_LRU = 0, 1, 2
 KV_NONE = 0xFFFFFFFF
 KV_DEV_BAD_INDEX = 16
 KV_DEV_BAD_HEAD_VALUE = 64
+KV_DEV_BAD_SPAN_VALUE = 128
 KV_LOC_HOST = 0x80000000
 
 
@@ -85,7 +86,7 @@ SLOT_META_DTYPE = np.dtype([("tag", "<u4"), ("last_epoch", "<u4"), ("ema", "<f4"
 
 EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_bytes",
            "kv_pool_create", "kv_pool_destroy", "kv_epoch_score", "kv_epoch_score_select", "kv_epoch_events", "kv_epoch_counts",
-           "kv_epoch_update", "kv_set_policy", "kv_set_lazy_decay", "kv_hash_entries", "kv_dedup_table_slots", "kv_dedup_digests", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
+           "kv_epoch_update", "kv_set_policy", "kv_set_lazy_decay", "kv_hash_entries", "kv_dedup_table_slots", "kv_dedup_digests", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_prefetch_window_update", "kv_set_prefetch_window", "kv_prefetch_span", "kv_prefetch_window", "kv_prefetch_list", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
            "kv_set_select_variant", "kv_selection_stats", "kv_demote_counted", "kv_victim_counts", "kv_set_gather_threshold", "kv_last_cuda_error", "kv_status_string",
@@ -148,6 +149,16 @@ def load():
     L.kv_head_importance.argtypes = [vp, i32]
     L.kv_head_weights.restype = vp
     L.kv_head_weights.argtypes = [vp, i32]
+    L.kv_prefetch_window_update.restype = i32
+    L.kv_prefetch_window_update.argtypes = [vp, i32, vp, C.c_float, vp]
+    L.kv_set_prefetch_window.restype = i32
+    L.kv_set_prefetch_window.argtypes = [vp, i32, C.c_float, C.c_uint32, vp]
+    L.kv_prefetch_span.restype = vp
+    L.kv_prefetch_span.argtypes = [vp, i32]
+    L.kv_prefetch_window.restype = vp
+    L.kv_prefetch_window.argtypes = [vp, i32]
+    L.kv_prefetch_list.restype = i32
+    L.kv_prefetch_list.argtypes = [vp, i32, vp, C.c_uint64, C.c_uint64, i32, vp, C.c_uint64, vp, vp]
     L.kv_select_victims.restype = i32
     L.kv_select_victims.argtypes = [vp, u64, vp, vp]
     L.kv_select_victim_blocks.restype = i32
@@ -419,6 +430,30 @@ class Pool:
         """Partition q's [layers][KV heads] score weights."""
         p = self.parts[q]
         return self._head_view(self.lib.kv_head_weights(self._h, int(q)), p.n_layers * p.heads)
+
+    def kv_prefetch_window_update(self, q, d_span, decay):
+        return self.lib.kv_prefetch_window_update(self._h, int(q), d_span.data_ptr() if d_span is not None else None,
+                                                  float(decay), _stream_ptr(self.compute))
+
+    def kv_set_prefetch_window(self, q, tokens, max_blocks):
+        return self.lib.kv_set_prefetch_window(self._h, int(q), float(tokens), int(max_blocks),
+                                               _stream_ptr(self.compute))
+
+    def kv_prefetch_span(self, q):
+        """Partition q's per-layer attention-span EMA in tokens (float32 tensor aliasing device memory)."""
+        return self._head_view(self.lib.kv_prefetch_span(self._h, int(q)), self.parts[q].n_layers)
+
+    def kv_prefetch_window(self, q):
+        """Partition q's per-layer prefetch window in blocks (int32 view of the device's uint32 values)."""
+        off = self.lib.kv_prefetch_window(self._h, int(q)) - self.workspace.data_ptr()
+        return self.workspace[off:off + 4 * self.parts[q].n_layers].view(self.torch.int32)
+
+    def kv_prefetch_list(self, q, d_table, n_pos, pos0, direction, d_out_slots, max_out, d_out_count):
+        return self.lib.kv_prefetch_list(self._h, int(q), d_table.data_ptr() if d_table is not None else None,
+                                         int(n_pos), int(pos0), int(direction),
+                                         d_out_slots.data_ptr() if d_out_slots is not None else None, int(max_out),
+                                         d_out_count.data_ptr() if d_out_count is not None else None,
+                                         _stream_ptr(self.compute))
 
     def kv_select_victims(self, k, d_victims):
         return self.lib.kv_select_victims(self._h, int(k), d_victims.data_ptr() if k else None,

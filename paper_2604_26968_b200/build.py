@@ -11,7 +11,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvtier.so")
-SOURCES = ["kvtier_host.cu", "kv_score.cu", "kv_select.cu", "kv_select_persist.cu", "kv_blocks.cu", "kv_heads.cu", "kv_dedup.cu", "kv_move.cu", "kv_move_tma.cu"]
+SOURCES = ["kvtier_host.cu", "kv_score.cu", "kv_select.cu", "kv_select_persist.cu", "kv_blocks.cu", "kv_heads.cu", "kv_prefetch.cu", "kv_dedup.cu", "kv_move.cu", "kv_move_tma.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

@@ -8,13 +8,13 @@
 //
 //   A  every score becomes an order-preserving key (fused form: the entry pass
 //      itself produces it) and enters the first histogram.  With a hint -- tau of
-//      the previous selection -- the histogram covers a bracket of 2^22 keys
-//      around it; the pass also leaves in shared memory a bitmap "key below the
+//      the previous selection -- the histogram covers a bracket of 2^18 .. 2^22 keys
+//      around it (2,048 bins; the width follows how far tau moved lately); the pass also leaves in shared memory a bitmap "key below the
 //      bracket", and every thread notes the keys it saw inside the bracket
 //      (typically 5-10 % of the slice) in a few private slots: no vote, no atomic.
 //   B  the remaining histograms of the radix select.  When rank k falls inside
-//      the bracket, ONE more histogram (the 2^11 single keys of the bracket bin
-//      that holds rank k) finishes it, and it is built from the noted keys alone:
+//      the bracket, ONE more histogram (the single keys of the bracket bin
+//      that holds rank k, at most 2^11) finishes it, and it is built from the noted keys alone:
 //      no second pass over the scores.  Otherwise (no hint, a miss, a thread that
 //      ran out of slots) the keys are re-read from the score array, which then
 //      sits mostly in L2, and the last histogram of that path leaves the bitmaps
@@ -376,7 +376,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   // ---- phase A: keys and the first histogram ----
   // Without a hint the first histogram is digit 0 of a plain radix select (bits
   // 31..21 of every key).  With a hint it covers only the bracket [base0, base0 +
-  // 2^22) around the hinted tau in 2,048 bins of 2^11 keys; keys below base0 set
+  // 2,048 << bshift) around the hinted tau in 2,048 bins of 2^bshift keys (bshift 7..11); keys below base0 set
   // their bit in s_bit_l (and are counted), keys inside are noted: scores move
   // little from one epoch to the next, so the k-th key is almost always inside,
   // and then only the notes are looked at again.

@@ -4,6 +4,7 @@
 // kv_select.cu and kv_move.cu.
 #include <cstdlib>
 #include <cstring>
+#include <limits>
 #include <new>
 #include <vector>
 
@@ -112,6 +113,7 @@ struct kv_pool {
   uint32_t* h_sel_stats = nullptr;
   HeadWeights head{};       // head-granular importance matrices and weights
   uint32_t n_head_imp = 0, n_head_w = 0;
+  PrefetchState prefetch{}; // per-layer prefetch windows
   // a demotion whose later chunks are not enqueued yet (deferred packing)
   struct Pending {
     bool active = false, meta_done = false;
@@ -134,8 +136,12 @@ struct kv_pool {
 
 namespace {
 
+constexpr float kPrefetchSpanTokens = 2048.0f;   // span every layer starts with
+constexpr uint32_t kPrefetchWindowCap = 65535;      // default cap on a window, blocks
+
 struct Layout {
   uint64_t head_imp, head_mult, head_w;
+  uint64_t pf_span, pf_win, pf_counts;
   uint64_t delta, hist, sel, status, blend, block_score, block_state, block_victims, part_counts, tile_counts, tile_offsets, free_list, slot_list[kListBufs];
   uint64_t ring[4][6];
   uint64_t dev_total;
@@ -208,6 +214,13 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
   L->head_imp = take(g.n_head_imp * 4);
   L->head_mult = take(g.n_head_w * 4);
   L->head_w = take(g.n_head_w * 4);
+  {
+    uint64_t layers = 0;
+    for (int q = 0; q < g.n_parts; ++q) layers += g.layers[q];
+    L->pf_span = take(layers * 4);
+    L->pf_win = take(layers * 4);
+    L->pf_counts = take(kPrefetchChunks * 4);
+  }
   L->block_score = take(g.n_blocks * 4);
   L->block_state = take(g.n_blocks);
   L->block_victims = take(g.n_blocks * 4);
@@ -586,6 +599,22 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
     p->n_head_imp = (uint32_t)g.n_head_imp;
     p->n_head_w = (uint32_t)g.n_head_w;
   }
+  {
+    PrefetchState& pf = p->prefetch;
+    pf.span = reinterpret_cast<float*>(w + L.pf_span);
+    pf.win = reinterpret_cast<uint32_t*>(w + L.pf_win);
+    pf.chunk_counts = reinterpret_cast<uint32_t*>(w + L.pf_counts);
+    uint32_t o = 0;
+    for (int q = 0; q < 4; ++q) {
+      const bool in = q < g.n_parts;
+      pf.off[q] = o;
+      pf.layers[q] = in ? (uint32_t)g.layers[q] : 0u;
+      pf.heads[q] = in ? (uint32_t)g.heads[q] : 1u;
+      pf.block_tokens[q] = in ? (uint32_t)desc->part[q].block_tokens : 1u;
+      pf.w_max[q] = kPrefetchWindowCap;
+      o += pf.layers[q];
+    }
+  }
   for (int b = 0; b < 4; ++b) p->staging[b] = static_cast<uint8_t*>(desc->d_staging[b]);
   p->staging_bytes = desc->staging_bytes;
   p->bgeom.n_parts = g.n_parts;
@@ -627,6 +656,8 @@ int32_t kv_pool_create(const kv_pool_desc* desc, kv_stream_t stream, kv_pool** o
     e = launch_init(p->st, desc->d_hits, desc->d_misses, desc->d_P, p0, desc->d_loc, desc->n_tags,
                     p->geom, p->n_parts, p->ws, S(stream));
     if (e == cudaSuccess) e = launch_head_init(p->head, p->n_head_imp, p->n_head_w, S(stream));
+    for (int q = 0; q < g.n_parts && e == cudaSuccess; ++q)
+      e = launch_prefetch_window(p->prefetch, q, 1, nullptr, 0.0f, kPrefetchSpanTokens, p->ws, S(stream));
   }
   if (e != cudaSuccess) {
     for (int i = 0; i < made; ++i) cudaEventDestroy(*evs[(size_t)i]);
@@ -703,6 +734,45 @@ const float* kv_head_importance(kv_pool* p, int32_t q) {
 
 const float* kv_head_weights(kv_pool* p, int32_t q) {
   return (p && q >= 0 && q < p->n_parts) ? p->head.w + p->head.w_off[q] : nullptr;
+}
+
+int32_t kv_prefetch_window_update(kv_pool* p, int32_t q, const float* d_span, float decay, kv_stream_t stream) {
+  if (!p || q < 0 || q >= p->n_parts || !d_span) return KV_ERR_INVALID_ARG;
+  if (!(decay >= 0.0f) || !(decay <= 1.0f)) return KV_ERR_INVALID_ARG;
+  KV_CUDA(p, launch_prefetch_window(p->prefetch, q, 0, d_span, decay, 0.0f, p->ws, S(stream)));
+  return KV_OK;
+}
+
+int32_t kv_set_prefetch_window(kv_pool* p, int32_t q, float tokens, uint32_t max_blocks, kv_stream_t stream) {
+  if (!p || q < 0 || q >= p->n_parts || max_blocks < 1) return KV_ERR_INVALID_ARG;
+  if (!(tokens >= 0.0f) || !(tokens <= std::numeric_limits<float>::max())) return KV_ERR_INVALID_ARG;
+  p->prefetch.w_max[q] = max_blocks;
+  KV_CUDA(p, launch_prefetch_window(p->prefetch, q, 1, nullptr, 0.0f, tokens, p->ws, S(stream)));
+  return KV_OK;
+}
+
+const float* kv_prefetch_span(kv_pool* p, int32_t q) {
+  return (p && q >= 0 && q < p->n_parts) ? p->prefetch.span + p->prefetch.off[q] : nullptr;
+}
+
+const uint32_t* kv_prefetch_window(kv_pool* p, int32_t q) {
+  return (p && q >= 0 && q < p->n_parts) ? p->prefetch.win + p->prefetch.off[q] : nullptr;
+}
+
+int32_t kv_prefetch_list(kv_pool* p, int32_t q, const uint32_t* d_table, uint64_t n_pos, uint64_t pos0,
+                         int32_t direction, uint64_t* d_out_slots, uint64_t max_out, uint64_t* d_out_count,
+                         kv_stream_t stream) {
+  if (!p || q < 0 || q >= p->n_parts || !d_out_count || direction == 0) return KV_ERR_INVALID_ARG;
+  if (n_pos > 0 && (!d_table || pos0 >= n_pos)) return KV_ERR_INVALID_ARG;
+  if (max_out > 0 && !d_out_slots) return KV_ERR_INVALID_ARG;
+  if (n_pos > (1ull << 40) / ((uint64_t)p->prefetch.layers[q] * p->prefetch.heads[q])) return KV_ERR_INVALID_ARG;
+  // d_loc is written by demotions (compute stream, at the call) and by promotions (their copy stream)
+  const int32_t rc = join_promotions(p, S(stream));
+  if (rc != KV_OK) return rc;
+  KV_CUDA(p, launch_prefetch_list(p->prefetch, q, d_table, n_pos, pos0, direction, p->desc.d_loc, p->desc.n_tags,
+                                  reinterpret_cast<unsigned long long*>(d_out_slots), max_out,
+                                  reinterpret_cast<unsigned long long*>(d_out_count), S(stream)));
+  return KV_OK;
 }
 
 int32_t kv_select_victims(kv_pool* p, uint64_t k, uint32_t* d_victims, kv_stream_t stream) {

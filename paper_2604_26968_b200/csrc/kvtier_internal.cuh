@@ -155,6 +155,18 @@ struct HeadWeights {
   int n_parts;
 };
 
+// Per-layer prefetch windows (RoPE-aware prefetching section): per partition the EMA of
+// the observed attention span in tokens and the window in blocks derived from it.
+constexpr uint32_t kPrefetchChunks = 1024;   // most blocks of one prefetch-list launch
+struct PrefetchState {
+  float* span;             // [layers] per partition, partition q at off[q]
+  uint32_t* win;           // same layout
+  uint32_t* chunk_counts;  // [kPrefetchChunks] scratch of the list kernels
+  uint32_t off[4], layers[4], heads[4];
+  uint32_t block_tokens[4];
+  uint32_t w_max[4];       // cap on the window, blocks
+};
+
 struct Workspace {
   BlendState* blend;
   float* block_score;       // [blocks] aggregate score per paged block
@@ -186,6 +198,17 @@ cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* 
 cudaError_t launch_head_update(const HeadWeights& hw, int q, int mode, const float* src, float decay,
                                const Workspace& ws, cudaStream_t s);
 cudaError_t launch_head_init(const HeadWeights& hw, uint32_t n_imp, uint32_t n_w, cudaStream_t s);
+// kv_prefetch.cu: mode 0 = EMA step of partition q's per-layer span with observations x [L]
+// (any negative or non-finite value: nothing changes, flagged); mode 1 = every span = tokens.
+// Both recompute the windows.
+cudaError_t launch_prefetch_window(const PrefetchState& pf, int q, int mode, const float* x, float decay,
+                                   float tokens, const Workspace& ws, cudaStream_t s);
+// ring slots of the host-tier blocks of table [n_pos][L][H] inside the windows around
+// position-block pos0, ordered by (distance, layer, head); *count = how many qualified
+cudaError_t launch_prefetch_list(const PrefetchState& pf, int q, const uint32_t* table, uint64_t n_pos,
+                                 uint64_t pos0, int dir, const uint32_t* loc, uint64_t n_tags,
+                                 unsigned long long* out, uint64_t max_out, unsigned long long* count,
+                                 cudaStream_t s);
 // empties the sliding window of the blend (the estimates stay as they are)
 cudaError_t launch_blend_reset(const Workspace& ws, cudaStream_t s);
 

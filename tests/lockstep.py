@@ -162,8 +162,10 @@ class Lockstep:
                                   o.head_array(q, "weights").view(np.uint32)), ("weights", e, q)
 
     # ---- one epoch -----------------------------------------------------------
-    def epoch(self, e, k=None, check_payload=None, k_blocks=None):
-        """One epoch on both sides.  k_blocks selects whole paged blocks instead of k entries."""
+    def epoch(self, e, k=None, check_payload=None, k_blocks=None, before_demote=None, promote_with=None):
+        """One epoch on both sides.  k_blocks selects whole paged blocks instead of k entries.
+        before_demote(self) runs once the victims agree; promote_with(self) returns the
+        per-partition promote lists to use in place of the workload's."""
         w, g, o = self.w, self.gpu, self.ora
         k = w.k if k is None else k
         ev_entry, ev_hit = w.events(e, o.pair, self.fresh)
@@ -198,6 +200,8 @@ class Lockstep:
         g.pool.sync()
         got = g.victims[:k].cpu().numpy().view(np.uint32)
         assert np.array_equal(got, v), "epoch %d victims" % e
+        if before_demote is not None:
+            before_demote(self)
         assert o.demote(v) == O.OK
         if self.counted and len(w.parts) > 1:
             # the counts the selection left in pinned memory (the stream has been synchronised above)
@@ -210,7 +214,7 @@ class Lockstep:
         if not self.deferred:   # (a status read would enqueue the deferred chunks and undo the interleaving)
             self.compare_state("epoch %d demote" % e, scores=False)
             self.compare_ring("epoch %d demote" % e)
-        lists = g.promote_lists(e)
+        lists = g.promote_lists(e) if promote_with is None else promote_with(self)
         for q, lst in enumerate(lists):
             pieces = np.array_split(lst, self.split_promote) if self.split_promote > 1 else [lst]
             for piece in pieces:
