@@ -332,29 +332,37 @@ __device__ __forceinline__ EntryVec entry_load4(const EntryState& st, uint64_t v
   return x;
 }
 
-// touch and last_epoch are only written where an entry was touched.
+// touch and last_epoch are only written where an entry was touched.  kPlain: the caller
+// knows that the policy is the Bayesian product and that no partition is weighted (the
+// policy and weight tests then fold away at compile time).
+template <bool kPlain = false>
 __device__ __forceinline__ void entry_finish4(const EntryState& st, uint64_t v, EntryVec& x, const float* sP,
                                               int policy, uint32_t epoch, const HeadWeights& hw, float4& sc) {
   float4 w = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
-  if (hw.on) {
+  if (!kPlain && hw.on) {
     w.x = head_weight(hw, 4 * v + 0);
     w.y = head_weight(hw, 4 * v + 1);
     w.z = head_weight(hw, 4 * v + 2);
     w.w = head_weight(hw, 4 * v + 3);
   }
-  entry_step(x.e.x, x.d.x, x.t.x, x.pr.x, x.st.x, sP, policy, x.le.x, epoch, w.x, sc.x);
-  entry_step(x.e.y, x.d.y, x.t.y, x.pr.y, x.st.y, sP, policy, x.le.y, epoch, w.y, sc.y);
-  entry_step(x.e.z, x.d.z, x.t.z, x.pr.z, x.st.z, sP, policy, x.le.z, epoch, w.z, sc.z);
-  entry_step(x.e.w, x.d.w, x.t.w, x.pr.w, x.st.w, sP, policy, x.le.w, epoch, w.w, sc.w);
+  const int pol = kPlain ? 0 : policy;
+  entry_step(x.e.x, x.d.x, x.t.x, x.pr.x, x.st.x, sP, pol, x.le.x, epoch, w.x, sc.x);
+  entry_step(x.e.y, x.d.y, x.t.y, x.pr.y, x.st.y, sP, pol, x.le.y, epoch, w.y, sc.y);
+  entry_step(x.e.z, x.d.z, x.t.z, x.pr.z, x.st.z, sP, pol, x.le.z, epoch, w.z, sc.z);
+  entry_step(x.e.w, x.d.w, x.t.w, x.pr.w, x.st.w, sP, pol, x.le.w, epoch, w.w, sc.w);
   reinterpret_cast<float4*>(st.ema)[v] = x.e;
   reinterpret_cast<float4*>(st.score)[v] = sc;
   // touch counts of FREE entries are always zero (events on them are refused)
   if (x.t.x | x.t.y | x.t.z | x.t.w) {
     reinterpret_cast<uint4*>(st.touch)[v] = make_uint4(0, 0, 0, 0);
-    if (x.t.x) st.last_epoch[4 * v + 0] = epoch;
-    if (x.t.y) st.last_epoch[4 * v + 1] = epoch;
-    if (x.t.z) st.last_epoch[4 * v + 2] = epoch;
-    if (x.t.w) st.last_epoch[4 * v + 3] = epoch;
+    if (x.t.x && x.t.y && x.t.z && x.t.w) {   // a block that reported all its heads: one store
+      reinterpret_cast<uint4*>(st.last_epoch)[v] = make_uint4(epoch, epoch, epoch, epoch);
+    } else {
+      if (x.t.x) st.last_epoch[4 * v + 0] = epoch;
+      if (x.t.y) st.last_epoch[4 * v + 1] = epoch;
+      if (x.t.z) st.last_epoch[4 * v + 2] = epoch;
+      if (x.t.w) st.last_epoch[4 * v + 3] = epoch;
+    }
   }
 }
 

@@ -56,6 +56,11 @@ constexpr uint32_t kBracketShiftMax = 11;               // a bracket bin is at m
 constexpr uint32_t kBracketShiftMin = 7;                // ... and at least 2^7 (2^17 keys to either side)
 constexpr uint32_t kPIdxBits = 18;                      // index of an entry inside its slice
 constexpr uint32_t kPMaxSlice = 1u << kPIdxBits;        // entries per CTA the bitmaps are sized for (2 x 32 KB)
+// Fused form: the entry pass's inputs of one chunk in shared memory -- ema, decay and touch
+// (4,096 words each), pair and state bytes (1,024 words each)
+constexpr uint32_t kEntryStageWords = 3u * kPChunk + 2u * kPThreads;
+constexpr uint32_t kEntryStages = 2;                    // chunks in flight ahead of the one being finished
+constexpr uint32_t kPSlotsMin = 10;
 constexpr uint32_t kPSlotsMax = 32;                     // bracket keys a thread can note (its private slots)
 
 
@@ -111,6 +116,7 @@ struct PArgs {
   unsigned long long per; // entries per CTA slice (multiple of 4, at most kPMaxSlice)
   uint32_t words;         // 32-bit words of one bitmap of a slice (a multiple of 4)
   uint32_t slots;         // private slots per thread for keys inside the bracket (at least 10)
+  uint32_t entry_stages;  // fused form: stages of the entry pass's inputs behind the slots (0: direct loads)
   PartCounts pc;          // partitions of the pool (the victims per partition are a by-product)
   uint32_t* spill;        // [n] global scratch for the notes a thread's slots cannot hold (nullptr: none)
   // the scoring pass of the fused form
@@ -193,7 +199,8 @@ __device__ __forceinline__ void pick_bin(const uint32_t* __restrict__ hist, uint
   __syncthreads();
 }
 
-template <bool FUSED>
+// PLAIN (fused form only): the policy is the Bayesian product and no partition is weighted.
+template <bool FUSED, bool PLAIN>
 __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const PArgs a) {
   extern __shared__ __align__(16) uint32_t s_dyn[];
   uint32_t* const s_bit_l = s_dyn;                    // bit j: key of local entry j is below tau
@@ -201,9 +208,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   // [slot][thread]: (key - base0) | position in the vector << 22 | chunk << 24; later the
   // staging buffer of the ordered write
   uint32_t* const s_note = s_bit_e + a.words;
+  // behind the slots: the stages of the fused entry pass; once phase A is over both together
+  // are scratch (stages of the re-reading passes, staging of the ordered write)
+  uint32_t* const s_entry = s_note + a.slots * kPThreads;
+  const uint32_t scratch_words = a.slots * kPThreads + a.entry_stages * kEntryStageWords;
   __shared__ uint32_t s_hist[kPHistBins];
   __shared__ uint32_t s_warp[32];
   __shared__ uint32_t s_pick[2];
+  __shared__ uint2 s_bnd[3];   // last CTA: (below tau, equal to tau) over the CTAs before each partition boundary's CTA
   __shared__ float sP[16];
   const uint32_t t = threadIdx.x;
   const uint32_t lane = t & 31u;
@@ -287,7 +299,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   // itself, so waiting for its own copy groups is all the synchronisation there is.
   auto for_chunks_staged = [&](auto body) {
     constexpr uint32_t kStageWords = kPChunk + kPThreads;   // 4096 scores + 1024 state words
-    const uint32_t n_stages = (a.slots * kPThreads) / kStageWords;   // at least 2 (slots >= 10)
+    const uint32_t n_stages = scratch_words / kStageWords;   // at least 2 (slots >= 10)
     const uint32_t depth = n_stages < 8u ? n_stages : 8u;
     auto issue = [&](uint32_t c, uint32_t stage) {
       const uint32_t j0 = c * kPChunk + 4u * t;
@@ -387,11 +399,15 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   bshift = bshift < kBracketShiftMin ? kBracketShiftMin : (bshift > kBracketShiftMax ? kBracketShiftMax : bshift);
   const uint32_t bbits = bshift + 11u;                  // log2 of the bracket's width in keys
   const uint32_t bhalf = 1u << (bbits - 1u);
-  const uint32_t base0 = hint ? (hint_tau > bhalf ? hint_tau - bhalf : 0u) : 0u;
+  // (the bracket [base0, base0 + 2^bbits) must end below the excluded key 0xFFFFFFFF)
+  const uint32_t base_max = 0xFFFFFFFFu - (1u << bbits);
+  const uint32_t base_c = hint_tau > bhalf ? hint_tau - bhalf : 0u;
+  const uint32_t base0 = hint ? (base_c < base_max ? base_c : base_max) : 0u;
   const uint32_t shift0 = hint ? bshift : 21u;
   bool hint_hit = false;
   WarpHist wh;
   uint32_t n_noted = 0;   // keys of this thread inside the bracket
+  uint32_t a_bin = 0, a_cnt = 0;   // ... and its pending count for one bin of the bracket's histogram
   // notes beyond the thread's slots: the CTA's stretch of the global scratch, laid out like the slots
   uint32_t* const spill = a.spill ? a.spill + s0 : nullptr;
   auto note_at = [&](uint32_t i) { return i < a.slots ? s_note[i * kPThreads + t] : __ldcg(&spill[(i - a.slots) * kPThreads + t]); };
@@ -401,39 +417,53 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       for (int q = 0; q < 4; ++q) wh.add(s_hist, key[q] != kExcluded, key[q] >> 21);
       return;
     }
-    uint32_t nib_l = 0;
+    // A key lies inside the bracket iff (key - base0) >> bbits == 0: a key below base0 wraps
+    // around to a large difference, and the bracket ends below the excluded key (base0 is
+    // kept that far down).  The thread's in-bracket keys -- usually none or one of the four --
+    // are then handled one after the other, so that a warp runs the body as often as its
+    // busiest lane has such keys and not once per position.
+    uint32_t nib_l = 0, in = 0;
+    uint32_t d[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const uint32_t d = key[q] - base0;
-      const bool below = key[q] < base0;   // (an excluded key is 0xFFFFFFFF: never below)
-      nib_l |= (uint32_t)below << q;
-      if (!below && (d >> bbits) == 0u && key[q] != kExcluded) {
-        atomicAdd(&s_hist[d >> bshift], 1u);
-        const uint32_t note = d | ((uint32_t)q << 22) | (c << 24);
-        if (n_noted < a.slots) s_note[n_noted * kPThreads + t] = note;
-        else if (spill) spill[(n_noted - a.slots) * kPThreads + t] = note;   // (a dense slice: the rest goes to L2)
-        ++n_noted;
+      d[q] = key[q] - base0;
+      nib_l |= (uint32_t)(key[q] < base0) << q;
+      in |= (uint32_t)((d[q] >> bbits) == 0u) << q;
+    }
+    while (in) {
+      const uint32_t q = (in & 1u) ? 0u : (in & 2u) ? 1u : (in & 4u) ? 2u : 3u;
+      in &= in - 1u;
+      const uint32_t dq = q == 0u ? d[0] : q == 1u ? d[1] : q == 2u ? d[2] : d[3];
+      // the histogram count waits in the thread while the bin stays the same (entries with
+      // equal scores come in runs, and atomics of many threads on one hot bin serialise)
+      const uint32_t bq = dq >> bshift;
+      if (bq != a_bin) {
+        if (a_cnt) atomicAdd(&s_hist[a_bin], a_cnt);
+        a_bin = bq;
+        a_cnt = 0;
       }
+      ++a_cnt;
+      const uint32_t note = dq | (q << 22) | (c << 24);
+      if (n_noted < a.slots) s_note[n_noted * kPThreads + t] = note;
+      else if (spill) spill[(n_noted - a.slots) * kPThreads + t] = note;   // (a dense slice: the rest goes to L2)
+      ++n_noted;
     }
     store_word(s_bit_l, nib_l, c * kPChunk + 4u * t);
   };
   clear_hist();
   if constexpr (FUSED) {
     // the slice's entries go through the EMA and score update on the way
-    const int policy = a.pd.policy;
+    const int policy = PLAIN ? 0 : a.pd.policy;
     const uint32_t jt = 4u * t;
-    EntryVec cur;
-    if (jt + 4 <= len) cur = entry_load4(a.st, (s0 + jt) / 4, policy);
-    for (uint32_t c = 0; c < n_chunks; ++c) {
+    // finishes the thread's vector of chunk c (entries j0 .. j0+3 of the slice, loaded into cur
+    // when the whole vector lies inside the slice) and hands its keys to phase A
+    auto finish_chunk = [&](uint32_t c, EntryVec& cur) {
       const uint32_t j0 = c * kPChunk + jt;
       const unsigned long long i0 = s0 + j0;
-      // the next chunk's loads fly while this one is finished
-      EntryVec nxt;
-      if (c + 1 < n_chunks && j0 + kPChunk + 4 <= len) nxt = entry_load4(a.st, (i0 + kPChunk) / 4, policy);
       uint32_t key[4] = {kExcluded, kExcluded, kExcluded, kExcluded};
       if (j0 + 4 <= len) {
         float4 sc;
-        entry_finish4(a.st, i0 / 4, cur, sP, policy, a.epoch, a.hw, sc);
+        entry_finish4<PLAIN>(a.st, i0 / 4, cur, sP, policy, a.epoch, a.hw, sc);
         key[0] = cur.st.x == KV_STATE_RESIDENT ? p_score_key(sc.x) : kExcluded;
         key[1] = cur.st.y == KV_STATE_RESIDENT ? p_score_key(sc.y) : kExcluded;
         key[2] = cur.st.z == KV_STATE_RESIDENT ? p_score_key(sc.z) : kExcluded;
@@ -449,13 +479,76 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
           }
         }
       }
-      cur = nxt;
       phase_a(c, key);
+    };
+    // Full chunks stream through shared-memory stages filled by asynchronous copies, two
+    // chunks ahead of the one being finished: no registers hold data in flight, and the
+    // thread reads back only what it copied itself, so its own copy groups are all it
+    // waits for.  (The LRU policy also reads last_epoch, for which the stages have no
+    // room: it takes the direct loads, like the ragged last chunk.)
+    const uint32_t n_staged = (a.entry_stages == kEntryStages && policy != 2) ? len / kPChunk : 0u;
+    if (n_staged) {
+      auto issue = [&](uint32_t c, uint32_t stage) {
+        uint32_t* dst = s_entry + stage * kEntryStageWords;
+        const unsigned long long i0 = s0 + c * kPChunk + jt;
+        const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(dst + jt);
+        const uint32_t d1 = (uint32_t)__cvta_generic_to_shared(dst + 3u * kPChunk + t);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d0), "l"(a.st.ema + i0) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d0 + 4u * kPChunk), "l"(a.st.decay + i0) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d0 + 8u * kPChunk), "l"(a.st.touch + i0) : "memory");
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d1), "l"(a.st.pair + i0) : "memory");
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d1 + 4u * kPThreads), "l"(a.st.state + i0) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      };
+      for (uint32_t i = 0; i < kEntryStages; ++i) {
+        if (i < n_staged) issue(i, i);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+      }
+      for (uint32_t c = 0; c < n_staged; ++c) {
+        asm volatile("cp.async.wait_group 1;" ::: "memory");   // kEntryStages - 1 newer groups may be pending
+        const uint32_t stage = c % kEntryStages;
+        const uint32_t* src = s_entry + stage * kEntryStageWords;
+        EntryVec cur;
+        cur.e = *reinterpret_cast<const float4*>(src + jt);
+        cur.d = *reinterpret_cast<const float4*>(src + kPChunk + jt);
+        cur.t = *reinterpret_cast<const uint4*>(src + 2u * kPChunk + jt);
+        cur.pr = *reinterpret_cast<const uchar4*>(src + 3u * kPChunk + t);
+        cur.st = *reinterpret_cast<const uchar4*>(src + 3u * kPChunk + kPThreads + t);
+        cur.le = make_uint4(0, 0, 0, 0);
+        if (c + kEntryStages < n_staged) issue(c + kEntryStages, stage);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+        finish_chunk(c, cur);
+      }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    EntryVec cur;
+    if (n_staged < n_chunks && n_staged * kPChunk + jt + 4 <= len)
+      cur = entry_load4(a.st, (s0 + n_staged * kPChunk + jt) / 4, policy);
+    for (uint32_t c = n_staged; c < n_chunks; ++c) {
+      // the next chunk's loads fly while this one is finished
+      EntryVec nxt;
+      const uint32_t j1 = (c + 1u) * kPChunk + jt;
+      if (c + 1 < n_chunks && j1 + 4 <= len) nxt = entry_load4(a.st, (s0 + j1) / 4, policy);
+      finish_chunk(c, cur);
+      cur = nxt;
     }
   } else {
     for_chunks(phase_a);
   }
   wh.flush(s_hist);
+  // pending bracket counts: one atomic per bin value and warp
+  for (;;) {
+    const unsigned m = __ballot_sync(0xFFFFFFFFu, a_cnt != 0u);
+    if (m == 0) break;
+    const int leader = __ffs(m) - 1;
+    const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, a_bin, leader);
+    const bool mine = a_cnt != 0u && a_bin == b0;
+    uint32_t sum = mine ? a_cnt : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+    if ((int)lane == leader) atomicAdd(&s_hist[b0], sum);
+    if (mine) a_cnt = 0;
+  }
   flush_hist(a.hist, kPHistBins);   // (begins with a block barrier: the bitmap words are all written)
   if (hint) {
     uint32_t below = 0, cta_below0;
@@ -534,6 +627,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
           if ((int)lane == leader) atomicAdd(&s_hist[b0], sum);
           if (mine) p_cnt = 0;
         }
+        stamp(8);
       } else {
         // the last histogram (single keys) from the arrays; it also leaves the bitmaps "key
         // below the range" in s_bit_l and "key inside the range" in s_bit_e
@@ -553,6 +647,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       }
       w2.flush(s_hist);
       flush_hist(a.hist + h_new * kPHistBins, 1u << top);
+      stamp(9);
     };
     auto retire = [&](uint32_t h_old) {   // after a barrier: nobody reads histogram h_old any more
       if (blockIdx.x == 0) {
@@ -624,6 +719,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         else if (low == tau_low) atomicOr(&s_bit_e[j >> 5], 1u << (j & 31u));
       }
       __syncthreads();
+      stamp(10);
       for (uint32_t w = w0; w < w1; ++w) {
         c_l += (uint32_t)__popc(s_bit_l[w]);
         c_e += (uint32_t)__popc(s_bit_e[w]);
@@ -659,6 +755,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     const uint32_t ex_l = block_scan_excl(c_l, s_warp, tot_l);
     const uint32_t ex_e = block_scan_excl(c_e, s_warp, tot_e);
     if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(tot_l, tot_e);
+    stamp(11);
     // a partition boundary inside this slice: how many of the slice's marked entries lie before it
     for (int q = 1; q < a.pc.n_parts; ++q) {   // (the condition is the same for the whole CTA)
       if (a.pc.base[q] <= s0 || a.pc.base[q] >= s1) continue;
@@ -689,9 +786,15 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       }
       // (G <= 1024: one value per thread at most, each below 2^18)
       uint32_t tl, te;
-      (void)block_scan_excl((uint32_t)la, s_warp, tl);
-      (void)block_scan_excl((uint32_t)ea, s_warp, te);
+      const uint32_t pre_l = block_scan_excl((uint32_t)la, s_warp, tl);
+      const uint32_t pre_e = block_scan_excl((uint32_t)ea, s_warp, te);
       less_before = tl; eq_before = te;
+      stamp(12);
+      // the last CTA also reports the victims per partition: its thread g holds the sums over
+      // the CTAs before g, and the ones in front of each partition boundary's CTA are kept
+      if (blockIdx.x == G - 1)
+        for (int q = 1; q < a.pc.n_parts; ++q)
+          if (a.pc.base[q] < a.n && t == (uint32_t)(a.pc.base[q] / a.per)) s_bnd[q - 1] = make_uint2(pre_l, pre_e);
     }
     if (found) {
       // Position of a victim.  With L entries below tau and E entries equal to tau before it
@@ -706,13 +809,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       const uint32_t eq_room = eq_room64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)eq_room64;
       const uint32_t cta_total = tot_l + (tot_e < eq_room ? tot_e : eq_room);
       uint32_t* const s_stage = s_note;
-      const uint32_t stage_cap = a.slots * kPThreads;
+      const uint32_t stage_cap = scratch_words;
       // the thread's own victims are the consecutive positions [p_first, p_first + p_count)
       const uint32_t e0 = ex_e < eq_room ? ex_e : eq_room;
       const uint32_t e1 = ex_e + c_e < eq_room ? ex_e + c_e : eq_room;
       const uint32_t p_first = ex_l + e0, p_count = c_l + (e1 - e0);
       const uint32_t id_base = (uint32_t)s0;   // (ids fit 32 bits)
       __syncthreads();   // every thread is done with the notes
+      stamp(13);
       for (uint32_t r0 = 0; r0 < cta_total; r0 += stage_cap) {
         if (p_count != 0 && p_first < r0 + stage_cap && p_first + p_count > r0) {
           uint32_t n_l = ex_l, n_e = ex_e;   // counts inside the CTA before the current word
@@ -722,14 +826,26 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
             if (be == 0u) {
               // no entry at tau in this word: its victims take consecutive positions
               uint32_t pos = n_l + (n_e < eq_room ? n_e : eq_room) - r0;   // (wraps below r0: skipped)
-              uint32_t bits = bl;
-              while (bits) {
-                const uint32_t b = (uint32_t)__ffs(bits) - 1u;
-                bits &= bits - 1u;
-                if (pos < stage_cap) s_stage[pos] = id0 + b;
-                ++pos;
+              const uint32_t cnt = (uint32_t)__popc(bl);
+              if (cnt > 8u) {
+                // a dense word (a slice whose blocks mostly go): every bit in turn, no bit search
+#pragma unroll
+                for (uint32_t b = 0; b < 32u; ++b) {
+                  if ((bl >> b) & 1u) {
+                    if (pos < stage_cap) s_stage[pos] = id0 + b;
+                    ++pos;
+                  }
+                }
+              } else {
+                uint32_t bits = bl;
+                while (bits) {
+                  const uint32_t b = (uint32_t)__ffs(bits) - 1u;
+                  bits &= bits - 1u;
+                  if (pos < stage_cap) s_stage[pos] = id0 + b;
+                  ++pos;
+                }
               }
-              n_l += (uint32_t)__popc(bl);
+              n_l += cnt;
               continue;
             }
             uint32_t bits = bl | be;
@@ -756,10 +872,10 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         __syncthreads();
       }
     }
+    if (blockIdx.x == G - 1) __syncthreads();   // s_bnd
     if (blockIdx.x == G - 1 && t == 0) {
       // every entry has been counted: the selection must hold exactly k ids
-      unsigned long long tl = 0, te = 0;
-      for (uint32_t g = 0; g < G; ++g) { const uint2 cc = __ldcg(&a.cta_counts[g]); tl += cc.x; te += cc.y; }
+      const unsigned long long tl = less_before + tot_l, te = eq_before + tot_e;
       const unsigned long long got = tl + (te < need_eq ? te : need_eq);
       if (!found || got != a.k) atomicOr(a.status, KV_DEV_SELECT_MISMATCH);
       if (a.pc.n_parts > 1 && a.pc.d_counts) {
@@ -769,8 +885,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         for (int q = 1; q <= a.pc.n_parts; ++q) {
           if (q == a.pc.n_parts || a.pc.base[q] >= a.n) { before[q] = got; continue; }
           const uint32_t cb = (uint32_t)(a.pc.base[q] / a.per);          // the CTA whose slice holds the boundary
-          unsigned long long l = 0, e = 0;
-          for (uint32_t g = 0; g < cb && g < G; ++g) { const uint2 cc = __ldcg(&a.cta_counts[g]); l += cc.x; e += cc.y; }
+          unsigned long long l = s_bnd[q - 1].x, e = s_bnd[q - 1].y;     // sums over the CTAs before it
           if (a.pc.base[q] > (unsigned long long)cb * a.per) {            // strictly inside that slice
             const uint2 sp = __ldcg(&a.sel->bsplit[q - 1]);
             l += sp.x; e += sp.y;
@@ -848,8 +963,8 @@ PersistDevice g_persist[kPMaxDevices];
 
 // Dynamic shared memory of a launch: two bitmaps and the threads' private slots (which the
 // ordered write reuses as its staging buffer).
-inline size_t persist_smem(uint32_t words, uint32_t slots) {
-  return (size_t)words * 8u + (size_t)slots * kPThreads * 4u;
+inline size_t persist_smem(uint32_t words, uint32_t slots, uint32_t entry_stages = 0) {
+  return (size_t)words * 8u + (size_t)slots * kPThreads * 4u + (size_t)entry_stages * kEntryStageWords * 4u;
 }
 }  // namespace
 
@@ -872,26 +987,28 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
       cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
       cudaDeviceGetAttribute(&d.n_sm, cudaDevAttrMultiProcessorCount, dev);
       cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-      cudaFuncAttributes fa{}, fb{};
-      cudaError_t e = cudaFuncGetAttributes(&fa, select_persistent_kernel<false>);
-      if (e == cudaSuccess) e = cudaFuncGetAttributes(&fb, select_persistent_kernel<true>);
-      const size_t fixed = fa.sharedSizeBytes > fb.sharedSizeBytes ? fa.sharedSizeBytes : fb.sharedSizeBytes;
-      // the most a launch asks for: the largest bitmaps and the most slots
-      const size_t want = persist_smem(kPMaxSlice / 32, kPSlotsMax);
-      if ((size_t)optin < fixed + want) e = cudaErrorInvalidValue;
+      void* fns[3] = {(void*)select_persistent_kernel<false, false>, (void*)select_persistent_kernel<true, false>,
+                      (void*)select_persistent_kernel<true, true>};
+      cudaError_t e = cudaSuccess;
+      size_t fixed = 0;
+      for (void* fn : fns) {
+        cudaFuncAttributes fa{};
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fn);
+        if (fa.sharedSizeBytes > fixed) fixed = fa.sharedSizeBytes;
+      }
+      // the most a launch may ask for: everything a block can opt in to beyond the kernels' static
+      // share; the least that must fit: the largest bitmaps, the fewest slots, the entry stages
+      const size_t want = (size_t)optin > fixed ? ((size_t)optin - fixed) / 1024 * 1024 : 0;
+      if (want < persist_smem(kPMaxSlice / 32, kPSlotsMin, kEntryStages)) e = cudaErrorInvalidValue;
       d.smem_max = want;
-      if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(select_persistent_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)want);
-      if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(select_persistent_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)want);
-      if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, select_persistent_kernel<false>,
-                                                          (int)kPThreads, want);
-      if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_f, select_persistent_kernel<true>,
-                                                          (int)kPThreads, want);
+      blocks = 1;
+      for (void* fn : fns) {
+        int b = 0;
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, fn, (int)kPThreads, want);
+        if (b < blocks) blocks = b;
+      }
+      blocks_f = blocks;
       d.state = (e == cudaSuccess && coop && blocks >= 1 && blocks_f >= 1 && d.n_sm > 0) ? 1 : -1;
       (void)cudaGetLastError();
     }
@@ -922,10 +1039,14 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   // of the shared memory stays with the L1, whose lines hold the loads in flight of the streaming
   // entry pass.
   uint64_t slots = (a.per + kPThreads - 1) / kPThreads;   // as many as the thread sees keys, up to the maximum
-  if (slots < 10) slots = 10;   // (two stages of the re-reading passes fit)
+  if (slots < kPSlotsMin) slots = kPSlotsMin;   // (two stages of the re-reading passes fit)
   if (slots > kPSlotsMax) slots = kPSlotsMax;
+  // the fused form streams its entries through stages behind the slots; the slots give way
+  // (a thread's notes beyond them go to the global scratch)
+  a.entry_stages = fs ? kEntryStages : 0u;
+  while (slots > kPSlotsMin && persist_smem(a.words, (uint32_t)slots, a.entry_stages) > pd.smem_max) --slots;
   a.slots = (uint32_t)slots;
-  const size_t smem = persist_smem(a.words, a.slots);
+  const size_t smem = persist_smem(a.words, a.slots, a.entry_stages);
   if (smem > pd.smem_max) return cudaSuccess;
   a.pc = pc ? *pc : PartCounts{};
   a.spill = ws.free_list;   // (scratch of promotions and admissions: idle while a selection runs)
@@ -940,7 +1061,9 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
     a.epoch = fs->epoch;
   }
   void* args[] = {&a};
-  void* fn = fs ? (void*)select_persistent_kernel<true> : (void*)select_persistent_kernel<false>;
+  const bool plain = fs && fs->opt.policy == 0 && fs->hw.on == 0;
+  void* fn = !fs ? (void*)select_persistent_kernel<false, false>
+                 : plain ? (void*)select_persistent_kernel<true, true> : (void*)select_persistent_kernel<true, false>;
   cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(G), dim3(kPThreads), args, smem, s);
   if (e != cudaSuccess) return e;
   count_launches(1);

@@ -95,7 +95,7 @@ struct SelectScalars {
   uint32_t hint_last;          // (tau of the last one)
   unsigned long long hint_n;   // ... and the number of keys it ran over
   unsigned long long below;    // keys below the bracket (accumulated per launch, cleared inside it)
-  unsigned long long phase_ns[8];  // %globaltimer at the phase boundaries of the last persistent selection (CTA 0)
+  unsigned long long phase_ns[16]; // %globaltimer at the phase boundaries of the last persistent selection (CTA 0)
   // how the persistent selections went so far (kv_selection_stats)
   unsigned int n_select;       // selections run
   unsigned int n_hint_hit;     // ... whose hint's bracket held rank k
