@@ -56,6 +56,7 @@ constexpr uint32_t kBracketShiftMax = 11;               // a bracket bin is at m
 constexpr uint32_t kBracketShiftMin = 7;                // ... and at least 2^7 (2^17 keys to either side)
 constexpr uint32_t kPIdxBits = 18;                      // index of an entry inside its slice
 constexpr uint32_t kPMaxSlice = 1u << kPIdxBits;        // entries per CTA the bitmaps are sized for (2 x 32 KB)
+constexpr uint32_t kPMaxChunks = kPMaxSlice / kPChunk;  // chunks per CTA
 // Fused form: the entry pass's inputs of one chunk in shared memory -- ema, decay and touch
 // (4,096 words each), pair and state bytes (1,024 words each)
 constexpr uint32_t kEntryStageWords = 3u * kPChunk + 2u * kPThreads;
@@ -111,9 +112,10 @@ struct PArgs {
   uint32_t* victims;
   uint32_t* hist;         // [3][2048], zero on entry, zero again on exit
   SelectScalars* sel;
-  uint2* cta_counts;      // [gridDim.x]
+  uint2* chunk_counts;    // [total_chunks] (below tau, equal to tau) per chunk of the pool
+  uint32_t total_chunks;  // chunks of 4,096 entries in the pool
   uint32_t* status;
-  unsigned long long per; // entries per CTA slice (multiple of 4, at most kPMaxSlice)
+  unsigned long long per; // most entries of a CTA: whole chunks, at most kPMaxSlice
   uint32_t words;         // 32-bit words of one bitmap of a slice (a multiple of 4)
   uint32_t slots;         // private slots per thread for keys inside the bracket (at least 10)
   uint32_t entry_stages;  // fused form: stages of the entry pass's inputs behind the slots (0: direct loads)
@@ -215,32 +217,47 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   __shared__ uint32_t s_hist[kPHistBins];
   __shared__ uint32_t s_warp[32];
   __shared__ uint32_t s_pick[2];
+  __shared__ uint2 s_cex[kPMaxChunks + 1];    // (below, equal) counts the CTA holds before each of its chunks
+  __shared__ uint2 s_cpre[kPMaxChunks];       // ... and the pool holds before them
+  __shared__ uint32_t s_gstart[kPMaxChunks];  // where a chunk's victims start in the output
+  __shared__ uint32_t s_lstart[kPMaxChunks + 1];  // ... and in the stage of the ordered write
+  __shared__ uint2 s_rowtot[kPMaxChunks];     // totals of the rows of the chunk table, then the sums before each row
+  __shared__ uint2 s_all;                     // the table's total
   __shared__ uint2 s_bnd[3];   // last CTA: (below tau, equal to tau) over the CTAs before each partition boundary's CTA
   __shared__ float sP[16];
   const uint32_t t = threadIdx.x;
   const uint32_t lane = t & 31u;
   unsigned int* bar = &a.sel->bar_arrive;
   const unsigned int G = gridDim.x;
-  const unsigned long long s0 = (unsigned long long)blockIdx.x * a.per;
-  const unsigned long long s1 = (s0 + a.per < a.n) ? s0 + a.per : a.n;
-  const uint32_t len = s1 > s0 ? (uint32_t)(s1 - s0) : 0u;
-  const uint32_t n_chunks = (len + kPChunk - 1) / kPChunk;
+  // The CTA's entries: chunks blockIdx.x, blockIdx.x + G, ... of the pool (4,096 entries each),
+  // so that regions of the pool that cost more -- many touched entries, many keys near the
+  // threshold -- are spread over all CTAs.  Local chunk c is pool chunk c * G + blockIdx.x; the
+  // bitmaps and notes index entries by local position (chunk c, offset o) -> c * 4096 + o.
+  const uint32_t n_chunks = a.total_chunks > blockIdx.x ? (a.total_chunks - blockIdx.x + G - 1u) / G : 0u;
+  auto chunk_base = [&](uint32_t c) { return ((unsigned long long)c * G + blockIdx.x) * kPChunk; };
+  // pool id of local entry j
+  auto pool_id = [&](uint32_t j) { return chunk_base(j / kPChunk) + (j % kPChunk); };
   bool ok = true;
+  // Phase boundaries of CTA 0 for timing studies (compiled in with -DKV_PHASE_STAMPS only: a
+  // read of the global timer stalls the thread for a few hundred nanoseconds).
   auto stamp = [&](int i) {
+#ifdef KV_PHASE_STAMPS
     if (blockIdx.x == 0 && t == 0) {
       unsigned long long ns;
       asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns));
       a.sel->phase_ns[i] = ns;
     }
+#else
+    (void)i;
+#endif
   };
   stamp(0);
 
   // keys of the thread's vector (4 entries) of chunk c, computed from the arrays;
   // entries past the slice or not RESIDENT give kExcluded
   auto keys_from_arrays = [&](uint32_t c, uint32_t key[4]) {
-    const uint32_t j0 = c * kPChunk + 4u * t;
-    const unsigned long long i0 = s0 + j0;
-    if (j0 + 4 <= len) {
+    const unsigned long long i0 = chunk_base(c) + 4u * t;
+    if (i0 + 4 <= a.n) {
       const float4 sc = __ldcg(reinterpret_cast<const float4*>(a.score + i0));
       const uchar4 st = __ldcg(reinterpret_cast<const uchar4*>(a.state + i0));
       key[0] = st.x == KV_STATE_RESIDENT ? p_score_key(sc.x) : kExcluded;
@@ -250,7 +267,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     } else {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        key[j] = (j0 + j < len && a.state[i0 + j] == KV_STATE_RESIDENT) ? p_score_key(a.score[i0 + j])
+        key[j] = (i0 + j < a.n && a.state[i0 + j] == KV_STATE_RESIDENT) ? p_score_key(a.score[i0 + j])
                                                                         : kExcluded;
     }
   };
@@ -267,19 +284,18 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       uchar4 st[kAhead];
 #pragma unroll
       for (uint32_t u = 0; u < kAhead; ++u) {
-        const uint32_t j0 = (c - 1u - u) * kPChunk + 4u * t;
-        if (u < nb && j0 + 4 <= len) {
-          sc[u] = __ldcg(reinterpret_cast<const float4*>(a.score + s0 + j0));
-          st[u] = __ldcg(reinterpret_cast<const uchar4*>(a.state + s0 + j0));
+        const unsigned long long i0 = u < nb ? chunk_base(c - 1u - u) + 4u * t : a.n;
+        if (i0 + 4 <= a.n) {
+          sc[u] = __ldcg(reinterpret_cast<const float4*>(a.score + i0));
+          st[u] = __ldcg(reinterpret_cast<const uchar4*>(a.state + i0));
         }
       }
 #pragma unroll
       for (uint32_t u = 0; u < kAhead; ++u) {
         if (u < nb) {
           const uint32_t cc = c - 1u - u;
-          const uint32_t j0 = cc * kPChunk + 4u * t;
           uint32_t key[4];
-          if (j0 + 4 <= len) {
+          if (chunk_base(cc) + 4u * t + 4 <= a.n) {
             key[0] = st[u].x == KV_STATE_RESIDENT ? p_score_key(sc[u].x) : kExcluded;
             key[1] = st[u].y == KV_STATE_RESIDENT ? p_score_key(sc[u].y) : kExcluded;
             key[2] = st[u].z == KV_STATE_RESIDENT ? p_score_key(sc[u].z) : kExcluded;
@@ -302,13 +318,13 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     const uint32_t n_stages = scratch_words / kStageWords;   // at least 2 (slots >= 10)
     const uint32_t depth = n_stages < 8u ? n_stages : 8u;
     auto issue = [&](uint32_t c, uint32_t stage) {
-      const uint32_t j0 = c * kPChunk + 4u * t;
-      if (j0 + 4 <= len) {
+      const unsigned long long i0 = chunk_base(c) + 4u * t;
+      if (i0 + 4 <= a.n) {
         uint32_t* dst = s_note + stage * kStageWords;
         const uint32_t d_sc = (uint32_t)__cvta_generic_to_shared(dst + 4u * t);
         const uint32_t d_st = (uint32_t)__cvta_generic_to_shared(dst + kPChunk + t);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d_sc), "l"(a.score + s0 + j0) : "memory");
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d_st), "l"(a.state + s0 + j0) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d_sc), "l"(a.score + i0) : "memory");
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d_st), "l"(a.state + i0) : "memory");
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -329,9 +345,8 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
       }
       const uint32_t c = n_chunks - 1u - i, stage = i % depth;
-      const uint32_t j0 = c * kPChunk + 4u * t;
       uint32_t key[4];
-      if (j0 + 4 <= len) {
+      if (chunk_base(c) + 4u * t + 4 <= a.n) {
         const uint32_t* src = s_note + stage * kStageWords;
         const float4 sc = *reinterpret_cast<const float4*>(src + 4u * t);
         const uint32_t st4 = src[kPChunk + t];
@@ -369,8 +384,10 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       if (c) atomicAdd(&g_hist[b], c);
     }
   };
-  // every thread owns a contiguous run of bitmap words
-  const uint32_t wpt = (a.words + kPThreads - 1) / kPThreads;
+  // every thread owns a contiguous run of bitmap words inside one chunk (a chunk has 128 words;
+  // the run is 1, 2, 4 or 8 words long)
+  uint32_t wpt = 1;
+  while (wpt * kPThreads < a.words) wpt <<= 1;
   const uint32_t w0 = t * wpt < a.words ? t * wpt : a.words;
   const uint32_t w1 = w0 + wpt < a.words ? w0 + wpt : a.words;
 
@@ -409,8 +426,24 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   uint32_t n_noted = 0;   // keys of this thread inside the bracket
   uint32_t a_bin = 0, a_cnt = 0;   // ... and its pending count for one bin of the bracket's histogram
   // notes beyond the thread's slots: the CTA's stretch of the global scratch, laid out like the slots
-  uint32_t* const spill = a.spill ? a.spill + s0 : nullptr;
-  auto note_at = [&](uint32_t i) { return i < a.slots ? s_note[i * kPThreads + t] : __ldcg(&spill[(i - a.slots) * kPThreads + t]); };
+  // (row r of 1,024 notes lives in the stretch of the scratch that belongs to local chunk r / 4:
+  // a thread has noted at most four keys per chunk, so that chunk is already the CTA's own)
+  uint32_t* const spill = a.spill;
+  auto spill_at = [&](uint32_t r) { return spill + chunk_base(r >> 2) + (r & 3u) * kPThreads + t; };
+  // body(v) for every note of the thread: the slots first, then the spilled ones, whose loads
+  // (L2) are issued eight at a time before the first of them is used
+  auto for_notes = [&](auto body) {
+    const uint32_t in_slots = n_noted < a.slots ? n_noted : a.slots;
+    for (uint32_t i = 0; i < in_slots; ++i) body(s_note[i * kPThreads + t]);
+    for (uint32_t r = 0; a.slots + r < n_noted; r += 8u) {
+      uint32_t v[8];
+#pragma unroll
+      for (uint32_t u = 0; u < 8u; ++u) v[u] = (a.slots + r + u < n_noted) ? __ldcg(spill_at(r + u)) : 0xFFFFFFFFu;
+#pragma unroll
+      for (uint32_t u = 0; u < 8u; ++u)
+        if (a.slots + r + u < n_noted) body(v[u]);
+    }
+  };
   auto phase_a = [&](uint32_t c, const uint32_t key[4]) {
     if (!hint) {
 #pragma unroll
@@ -445,7 +478,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       ++a_cnt;
       const uint32_t note = dq | (q << 22) | (c << 24);
       if (n_noted < a.slots) s_note[n_noted * kPThreads + t] = note;
-      else if (spill) spill[(n_noted - a.slots) * kPThreads + t] = note;   // (a dense slice: the rest goes to L2)
+      else if (spill) *spill_at(n_noted - a.slots) = note;   // (a dense slice: the rest goes to L2)
       ++n_noted;
     }
     store_word(s_bit_l, nib_l, c * kPChunk + 4u * t);
@@ -458,10 +491,9 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     // finishes the thread's vector of chunk c (entries j0 .. j0+3 of the slice, loaded into cur
     // when the whole vector lies inside the slice) and hands its keys to phase A
     auto finish_chunk = [&](uint32_t c, EntryVec& cur) {
-      const uint32_t j0 = c * kPChunk + jt;
-      const unsigned long long i0 = s0 + j0;
+      const unsigned long long i0 = chunk_base(c) + jt;
       uint32_t key[4] = {kExcluded, kExcluded, kExcluded, kExcluded};
-      if (j0 + 4 <= len) {
+      if (i0 + 4 <= a.n) {
         float4 sc;
         entry_finish4<PLAIN>(a.st, i0 / 4, cur, sP, policy, a.epoch, a.hw, sc);
         key[0] = cur.st.x == KV_STATE_RESIDENT ? p_score_key(sc.x) : kExcluded;
@@ -471,7 +503,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       } else {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          if (j0 + j < len) {
+          if (i0 + j < a.n) {
             float sc;
             uint32_t s1;
             entry_update1(a.st, i0 + j, sP, policy, a.epoch, a.hw, sc, s1);
@@ -486,11 +518,13 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     // thread reads back only what it copied itself, so its own copy groups are all it
     // waits for.  (The LRU policy also reads last_epoch, for which the stages have no
     // room: it takes the direct loads, like the ragged last chunk.)
-    const uint32_t n_staged = (a.entry_stages == kEntryStages && policy != 2) ? len / kPChunk : 0u;
+    // (all of the CTA's chunks are full but the pool's last one, which may be ragged)
+    const uint32_t n_full = (n_chunks && chunk_base(n_chunks - 1u) + kPChunk > a.n) ? n_chunks - 1u : n_chunks;
+    const uint32_t n_staged = (a.entry_stages == kEntryStages && policy != 2) ? n_full : 0u;
     if (n_staged) {
       auto issue = [&](uint32_t c, uint32_t stage) {
         uint32_t* dst = s_entry + stage * kEntryStageWords;
-        const unsigned long long i0 = s0 + c * kPChunk + jt;
+        const unsigned long long i0 = chunk_base(c) + jt;
         const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(dst + jt);
         const uint32_t d1 = (uint32_t)__cvta_generic_to_shared(dst + 3u * kPChunk + t);
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d0), "l"(a.st.ema + i0) : "memory");
@@ -522,13 +556,13 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
       asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     EntryVec cur;
-    if (n_staged < n_chunks && n_staged * kPChunk + jt + 4 <= len)
-      cur = entry_load4(a.st, (s0 + n_staged * kPChunk + jt) / 4, policy);
+    if (n_staged < n_chunks && chunk_base(n_staged) + jt + 4 <= a.n)
+      cur = entry_load4(a.st, (chunk_base(n_staged) + jt) / 4, policy);
     for (uint32_t c = n_staged; c < n_chunks; ++c) {
       // the next chunk's loads fly while this one is finished
       EntryVec nxt;
-      const uint32_t j1 = (c + 1u) * kPChunk + jt;
-      if (c + 1 < n_chunks && j1 + 4 <= len) nxt = entry_load4(a.st, (s0 + j1) / 4, policy);
+      const unsigned long long i1 = c + 1 < n_chunks ? chunk_base(c + 1u) + jt : a.n;
+      if (i1 + 4 <= a.n) nxt = entry_load4(a.st, i1 / 4, policy);
       finish_chunk(c, cur);
       cur = nxt;
     }
@@ -598,8 +632,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         // notes; noted keys of earlier bins are below the final range: their bit joins s_bit_l
         const uint32_t bin_k = (base - base0) >> bshift;
         uint32_t p_bin = 0, p_cnt = 0;   // the thread's pending count for one key value
-        for (uint32_t i = 0; i < n_noted; ++i) {
-          const uint32_t v = note_at(i);
+        for_notes([&](uint32_t v) {
           const uint32_t d = v & ((1u << 22) - 1u), b = d >> bshift;
           if (b < bin_k) {
             const uint32_t j = (v >> 24) * kPChunk + 4u * t + ((v >> 22) & 3u);
@@ -613,7 +646,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
             }
             ++p_cnt;
           }
-        }
+        });
         // pending counts: one atomic per key value and warp
         for (;;) {
           const unsigned m = __ballot_sync(0xFFFFFFFFu, p_cnt != 0u);
@@ -709,15 +742,14 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     uint32_t c_l = 0, c_e = 0;
     if (use_notes) {
       const uint32_t bin_k = (base - base0) >> bshift;
-      for (uint32_t i = 0; i < n_noted; ++i) {
-        const uint32_t v = note_at(i);
+      for_notes([&](uint32_t v) {
         const uint32_t d = v & ((1u << 22) - 1u);
-        if ((d >> bshift) != bin_k) continue;
+        if ((d >> bshift) != bin_k) return;
         const uint32_t low = d & ((1u << bshift) - 1u);
         const uint32_t j = (v >> 24) * kPChunk + 4u * t + ((v >> 22) & 3u);
         if (low < tau_low) atomicOr(&s_bit_l[j >> 5], 1u << (j & 31u));
         else if (low == tau_low) atomicOr(&s_bit_e[j >> 5], 1u << (j & 31u));
-      }
+      });
       __syncthreads();
       stamp(10);
       for (uint32_t w = w0; w < w1; ++w) {
@@ -740,7 +772,7 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
           while (bits) {
             const uint32_t b = (uint32_t)__ffs(bits) - 1u;
             bits &= bits - 1u;
-            const uint32_t key = p_score_key(__ldcg(a.score + s0 + 32u * w + b));
+            const uint32_t key = p_score_key(__ldcg(a.score + pool_id(32u * w + b)));
             if (key != tau) be &= ~(1u << b);
             if (key < tau) bl |= 1u << b;
           }
@@ -754,14 +786,27 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     uint32_t tot_l, tot_e;
     const uint32_t ex_l = block_scan_excl(c_l, s_warp, tot_l);
     const uint32_t ex_e = block_scan_excl(c_e, s_warp, tot_e);
-    if (t == 0) a.cta_counts[blockIdx.x] = make_uint2(tot_l, tot_e);
+    // The counts of every chunk go to the pool-wide table (pool order = chunk order): the scan's
+    // value at a chunk's first thread is what the CTA holds before that chunk.
+    const uint32_t tpc = 128u / wpt;   // threads per chunk
+    const uint32_t my_c = t / tpc;     // local chunk of this thread's words
+    if (t % tpc == 0u && my_c < n_chunks) s_cex[my_c] = make_uint2(ex_l, ex_e);
+    if (t == 0) s_cex[n_chunks] = make_uint2(tot_l, tot_e);
+    __syncthreads();
+    if (t < n_chunks) {
+      const uint2 c0 = s_cex[t], c1 = s_cex[t + 1u];
+      a.chunk_counts[t * G + blockIdx.x] = make_uint2(c1.x - c0.x, c1.y - c0.y);
+    }
     stamp(11);
-    // a partition boundary inside this slice: how many of the slice's marked entries lie before it
+    // a partition boundary strictly inside one of this CTA's chunks: how many of the chunk's
+    // marked entries lie before it
     for (int q = 1; q < a.pc.n_parts; ++q) {   // (the condition is the same for the whole CTA)
-      if (a.pc.base[q] <= s0 || a.pc.base[q] >= s1) continue;
-      const uint32_t jb = (uint32_t)(a.pc.base[q] - s0);   // first local entry of partition q
+      const unsigned long long bq = a.pc.base[q];
+      if (bq >= a.n || (bq % kPChunk) == 0u || (bq / kPChunk) % G != blockIdx.x) continue;
+      const uint32_t lc = (uint32_t)((bq / kPChunk) / G);
+      const uint32_t jb = lc * kPChunk + (uint32_t)(bq % kPChunk);   // first local entry of partition q
       uint32_t bl = 0, be = 0;
-      for (uint32_t w = t; w <= (jb >> 5) && w < a.words; w += kPThreads) {
+      for (uint32_t w = lc * 128u + t; w <= (jb >> 5); w += kPThreads) {
         const uint32_t m = w < (jb >> 5) ? 0xFFFFFFFFu : ((1u << (jb & 31u)) - 1u);
         bl += (uint32_t)__popc(s_bit_l[w] & m);
         be += (uint32_t)__popc(s_bit_e[w] & m);
@@ -777,75 +822,151 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
     if (!ok) goto fail;
     retire(h);
 
-    unsigned long long less_before, eq_before;
+    // The table read as rows of G chunks (row r = every CTA's local chunk r): what the pool holds
+    // before this CTA's chunk of row r is the rows before r plus the row's columns before the
+    // CTA's own.  A warp sums a row -- all of it and the part before the CTA -- with its loads
+    // in flight together; one warp then scans the row totals.
+    uint32_t all_l, all_e;
     {
-      unsigned long long la = 0, ea = 0;  // sums over the CTAs before this one
-      for (uint32_t g = t; g < blockIdx.x; g += kPThreads) {
-        const uint2 cc = __ldcg(&a.cta_counts[g]);
-        la += cc.x; ea += cc.y;
+      const uint32_t n_rows = (a.total_chunks + G - 1u) / G;   // at most kPMaxChunks
+      const uint32_t warp = t >> 5;
+      for (uint32_t r = warp; r < n_rows; r += kPThreads / 32u) {
+        uint32_t tl = 0, te = 0, pl = 0, pe = 0;
+        for (uint32_t g0 = 0; g0 < G; g0 += 128u) {
+          uint2 cc[4];
+#pragma unroll
+          for (uint32_t u = 0; u < 4u; ++u) {
+            const uint32_t gg = g0 + 32u * u + lane, cid = r * G + gg;
+            cc[u] = (gg < G && cid < a.total_chunks) ? __ldcg(&a.chunk_counts[cid]) : make_uint2(0u, 0u);
+          }
+#pragma unroll
+          for (uint32_t u = 0; u < 4u; ++u) {
+            tl += cc[u].x; te += cc[u].y;
+            if (g0 + 32u * u + lane < blockIdx.x) { pl += cc[u].x; pe += cc[u].y; }
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          tl += __shfl_xor_sync(0xFFFFFFFFu, tl, o); te += __shfl_xor_sync(0xFFFFFFFFu, te, o);
+          pl += __shfl_xor_sync(0xFFFFFFFFu, pl, o); pe += __shfl_xor_sync(0xFFFFFFFFu, pe, o);
+        }
+        if (lane == 0) { s_rowtot[r] = make_uint2(tl, te); s_cpre[r] = make_uint2(pl, pe); }
       }
-      // (G <= 1024: one value per thread at most, each below 2^18)
-      uint32_t tl, te;
-      const uint32_t pre_l = block_scan_excl((uint32_t)la, s_warp, tl);
-      const uint32_t pre_e = block_scan_excl((uint32_t)ea, s_warp, te);
-      less_before = tl; eq_before = te;
+      __syncthreads();
+      if (t < 32u) {
+        // exclusive scan of the row totals (two rows per lane); s_rowtot becomes "before row r"
+        const uint2 v0 = lane < n_rows ? s_rowtot[lane] : make_uint2(0u, 0u);
+        const uint2 v1 = lane + 32u < n_rows ? s_rowtot[lane + 32u] : make_uint2(0u, 0u);
+        uint32_t l0 = v0.x, e0 = v0.y, l1 = v1.x, e1 = v1.y;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t a0 = __shfl_up_sync(0xFFFFFFFFu, l0, o), b0 = __shfl_up_sync(0xFFFFFFFFu, e0, o);
+          const uint32_t a1 = __shfl_up_sync(0xFFFFFFFFu, l1, o), b1 = __shfl_up_sync(0xFFFFFFFFu, e1, o);
+          if (lane >= (uint32_t)o) { l0 += a0; e0 += b0; l1 += a1; e1 += b1; }
+        }
+        const uint32_t tl0 = __shfl_sync(0xFFFFFFFFu, l0, 31), te0 = __shfl_sync(0xFFFFFFFFu, e0, 31);
+        s_rowtot[lane] = make_uint2(l0 - v0.x, e0 - v0.y);
+        s_rowtot[lane + 32u] = make_uint2(tl0 + l1 - v1.x, te0 + e1 - v1.y);
+        if (lane == 31u) s_all = make_uint2(tl0 + l1, te0 + e1);
+      }
+      __syncthreads();
+      if (t < n_rows) {
+        const uint2 rp = s_rowtot[t], cp = s_cpre[t];
+        s_cpre[t] = make_uint2(rp.x + cp.x, rp.y + cp.y);
+      }
+      all_l = s_all.x; all_e = s_all.y;
+      // the last CTA also reports the victims per partition: warp q - 1 sums what lies in front of
+      // partition q's first chunk
+      if (blockIdx.x == G - 1 && (int)warp + 1 < a.pc.n_parts && a.pc.base[warp + 1u] < a.n) {
+        const uint32_t cb = (uint32_t)(a.pc.base[warp + 1u] / kPChunk), r = cb / G, gq = cb % G;
+        uint32_t pl = 0, pe = 0;
+        for (uint32_t gg = lane; gg < gq; gg += 32u) {
+          const uint2 cc = __ldcg(&a.chunk_counts[r * G + gg]);
+          pl += cc.x; pe += cc.y;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          pl += __shfl_xor_sync(0xFFFFFFFFu, pl, o); pe += __shfl_xor_sync(0xFFFFFFFFu, pe, o);
+        }
+        if (lane == 0) s_bnd[warp] = make_uint2(s_rowtot[r].x + pl, s_rowtot[r].y + pe);
+      }
+      __syncthreads();
       stamp(12);
-      // the last CTA also reports the victims per partition: its thread g holds the sums over
-      // the CTAs before g, and the ones in front of each partition boundary's CTA are kept
-      if (blockIdx.x == G - 1)
-        for (int q = 1; q < a.pc.n_parts; ++q)
-          if (a.pc.base[q] < a.n && t == (uint32_t)(a.pc.base[q] / a.per)) s_bnd[q - 1] = make_uint2(pre_l, pre_e);
     }
     if (found) {
       // Position of a victim.  With L entries below tau and E entries equal to tau before it
       // in id order, an entry below tau goes to L + min(E, need_eq) and an entry equal to tau,
-      // taken while E < need_eq, to L + E.  The CTA's victims form one contiguous piece of the
-      // output, starting at p0.  Every thread walks the set bits of its own words and puts the
-      // ids in order in shared memory (the notes' space, free by now), from where they leave
-      // as full-line stores, a stage-full per round.
-      const unsigned long long eq_taken_before = eq_before < need_eq ? eq_before : need_eq;
-      const unsigned long long p0 = less_before + eq_taken_before;
-      const unsigned long long eq_room64 = need_eq - eq_taken_before;
-      const uint32_t eq_room = eq_room64 > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)eq_room64;
-      const uint32_t cta_total = tot_l + (tot_e < eq_room ? tot_e : eq_room);
+      // taken while E < need_eq, to L + E.  The victims of a chunk form one contiguous piece of
+      // the output.  Every thread walks the set bits of its own words and puts the ids in
+      // order in shared memory (the notes' space, free by now), the CTA's chunks one after the
+      // other; from there they leave as full-line stores, a stage-full per round.
+      const uint32_t eq_room = need_eq > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)need_eq;
+      auto taken = [&](uint32_t e) { return e < eq_room ? e : eq_room; };
+      if (t < 32u) {
+        // where each chunk's piece starts: in the output (s_gstart) and in the stage (s_lstart)
+        uint32_t v[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const uint32_t lc = lane + 32u * u;
+          v[u] = 0;
+          if (lc < n_chunks) {
+            const uint2 c0 = s_cex[lc], c1 = s_cex[lc + 1u], pre = s_cpre[lc];
+            v[u] = (c1.x - c0.x) + (taken(pre.y + (c1.y - c0.y)) - taken(pre.y));
+            s_gstart[lc] = pre.x + taken(pre.y);
+          }
+        }
+        uint32_t i0 = v[0], i1 = v[1];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t y0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), y1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
+          if (lane >= (uint32_t)o) { i0 += y0; i1 += y1; }
+        }
+        const uint32_t tot0 = __shfl_sync(0xFFFFFFFFu, i0, 31);
+        s_lstart[lane] = i0 - v[0];
+        s_lstart[lane + 32u] = tot0 + i1 - v[1];
+        if (lane == 31u) s_lstart[64] = tot0 + i1;
+      }
+      __syncthreads();
+      stamp(14);
+      const uint32_t cta_total = s_lstart[64];
       uint32_t* const s_stage = s_note;
       const uint32_t stage_cap = scratch_words;
-      // the thread's own victims are the consecutive positions [p_first, p_first + p_count)
-      const uint32_t e0 = ex_e < eq_room ? ex_e : eq_room;
-      const uint32_t e1 = ex_e + c_e < eq_room ? ex_e + c_e : eq_room;
-      const uint32_t p_first = ex_l + e0, p_count = c_l + (e1 - e0);
-      const uint32_t id_base = (uint32_t)s0;   // (ids fit 32 bits)
+      // A thread whose words are full writes positions 32 * wpt apart from its neighbour's: the
+      // stage is indexed with the bank bits folded over by that stride, which keeps those writes
+      // and the consecutive reads of the copy-out both free of bank conflicts.
+      const uint32_t fold = 5u + (uint32_t)__ffs(wpt) - 1u;
+      auto stage_at = [&](uint32_t p) { return p ^ ((p >> fold) & 31u); };
+      // entries below / equal to tau in front of this thread's words, in the whole pool
+      const uint32_t mc = my_c < n_chunks ? my_c : 0u;   // (threads past the last chunk hold nothing)
+      const uint32_t Lg = s_cpre[mc].x + (ex_l - s_cex[mc].x), Eg = s_cpre[mc].y + (ex_e - s_cex[mc].y);
+      // from a position in the output to one in the stage (modulo 2^32)
+      const uint32_t to_stage = s_lstart[mc] - s_gstart[mc];
+      // the thread's own victims are the consecutive stage positions [p_first, p_first + p_count)
+      const uint32_t p_first = Lg + taken(Eg) + to_stage, p_count = c_l + (taken(Eg + c_e) - taken(Eg));
       __syncthreads();   // every thread is done with the notes
       stamp(13);
       for (uint32_t r0 = 0; r0 < cta_total; r0 += stage_cap) {
         if (p_count != 0 && p_first < r0 + stage_cap && p_first + p_count > r0) {
-          uint32_t n_l = ex_l, n_e = ex_e;   // counts inside the CTA before the current word
+          // entries below tau before the current word (shifted into stage positions), entries at tau
+          uint32_t n_l = Lg + to_stage, n_e = Eg;
           for (uint32_t w = w0; w < w1; ++w) {
             const uint32_t bl = s_bit_l[w], be = s_bit_e[w];
-            const uint32_t id0 = id_base + 32u * w;
-            if (be == 0u) {
-              // no entry at tau in this word: its victims take consecutive positions
+            const uint32_t id0 = (uint32_t)pool_id(32u * w);   // (ids fit 32 bits)
+            const uint32_t ce = (uint32_t)__popc(be);
+            if (be == 0u || n_e >= eq_room || n_e + ce <= eq_room) {
+              // no entry at tau in this word, none of them taken any more, or all of them taken:
+              // the word's victims take consecutive positions
+              const uint32_t vb = (be == 0u || n_e >= eq_room) ? bl : (bl | be);
               uint32_t pos = n_l + (n_e < eq_room ? n_e : eq_room) - r0;   // (wraps below r0: skipped)
-              const uint32_t cnt = (uint32_t)__popc(bl);
-              if (cnt > 8u) {
-                // a dense word (a slice whose blocks mostly go): every bit in turn, no bit search
-#pragma unroll
-                for (uint32_t b = 0; b < 32u; ++b) {
-                  if ((bl >> b) & 1u) {
-                    if (pos < stage_cap) s_stage[pos] = id0 + b;
-                    ++pos;
-                  }
-                }
-              } else {
-                uint32_t bits = bl;
-                while (bits) {
-                  const uint32_t b = (uint32_t)__ffs(bits) - 1u;
-                  bits &= bits - 1u;
-                  if (pos < stage_cap) s_stage[pos] = id0 + b;
-                  ++pos;
-                }
+              uint32_t bits = vb;
+              while (bits) {
+                const uint32_t b = (uint32_t)__ffs(bits) - 1u;
+                bits &= bits - 1u;
+                if (pos < stage_cap) s_stage[stage_at(pos)] = id0 + b;
+                ++pos;
               }
-              n_l += cnt;
+              n_l += (uint32_t)__popc(bl);
+              n_e += ce;
               continue;
             }
             uint32_t bits = bl | be;
@@ -860,22 +981,31 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
                 if (n_e < eq_room) pos = n_l + n_e;
                 ++n_e;
               }
-              if (pos >= r0 && pos - r0 < stage_cap) s_stage[pos - r0] = id0 + b;
+              if (pos >= r0 && pos - r0 < stage_cap) s_stage[stage_at(pos - r0)] = id0 + b;
             }
           }
         }
         __syncthreads();
         stamp(4);
-        const uint32_t n_out = cta_total - r0 < stage_cap ? cta_total - r0 : stage_cap;
-        for (uint32_t i = t; i < n_out; i += kPThreads)
-          if (p0 + r0 + i < a.k) a.victims[p0 + r0 + i] = s_stage[i];
+        const uint32_t r1 = cta_total - r0 < stage_cap ? cta_total : r0 + stage_cap;
+        {
+          // stage position i belongs to the chunk lc with s_lstart[lc] <= i < s_lstart[lc + 1]; a
+          // thread's positions ascend, so its chunk only moves forward
+          uint32_t lc = 0, le = s_lstart[1];
+          for (uint32_t i = r0 + t; i < r1; i += kPThreads) {
+            while (i >= le) { ++lc; le = s_lstart[lc + 1u]; }
+            const unsigned long long g = (unsigned long long)s_gstart[lc] + (i - s_lstart[lc]);
+            if (g < a.k) a.victims[g] = s_stage[stage_at(i - r0)];
+          }
+        }
+        stamp(15);
         __syncthreads();
       }
     }
     if (blockIdx.x == G - 1) __syncthreads();   // s_bnd
     if (blockIdx.x == G - 1 && t == 0) {
       // every entry has been counted: the selection must hold exactly k ids
-      const unsigned long long tl = less_before + tot_l, te = eq_before + tot_e;
+      const unsigned long long tl = all_l, te = all_e;
       const unsigned long long got = tl + (te < need_eq ? te : need_eq);
       if (!found || got != a.k) atomicOr(a.status, KV_DEV_SELECT_MISMATCH);
       if (a.pc.n_parts > 1 && a.pc.d_counts) {
@@ -884,9 +1014,8 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         unsigned long long before[5] = {0, 0, 0, 0, 0};
         for (int q = 1; q <= a.pc.n_parts; ++q) {
           if (q == a.pc.n_parts || a.pc.base[q] >= a.n) { before[q] = got; continue; }
-          const uint32_t cb = (uint32_t)(a.pc.base[q] / a.per);          // the CTA whose slice holds the boundary
-          unsigned long long l = s_bnd[q - 1].x, e = s_bnd[q - 1].y;     // sums over the CTAs before it
-          if (a.pc.base[q] > (unsigned long long)cb * a.per) {            // strictly inside that slice
+          unsigned long long l = s_bnd[q - 1].x, e = s_bnd[q - 1].y;     // sums over the chunks before the boundary's
+          if (a.pc.base[q] % kPChunk) {                                   // strictly inside that chunk
             const uint2 sp = __ldcg(&a.sel->bsplit[q - 1]);
             l += sp.x; e += sp.y;
           }
@@ -1016,11 +1145,11 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   }
   if (pd.state != 1) return cudaSuccess;
   unsigned int G = (unsigned int)pd.n_sm;
-  if (G > kPThreads) G = kPThreads;  // the prefix over the per-CTA counts takes one CTA per thread
-  const uint64_t min_per = kPChunk;  // do not spread tiny pools over more CTAs than they have chunks
-  if ((st.n + min_per - 1) / min_per < G) G = (unsigned int)((st.n + min_per - 1) / min_per);
+  if (G > kPThreads) G = kPThreads;
+  const uint64_t total_chunks = (st.n + kPChunk - 1) / kPChunk;
+  if (total_chunks < G) G = (unsigned int)total_chunks;   // tiny pools: not more CTAs than chunks
   if (G == 0) G = 1;
-  if (G + 2 > ws.n_tiles) return cudaSuccess;  // cta_counts live in the tile-count scratch
+  if (total_chunks + 2 > ws.n_tiles) return cudaSuccess;  // the per-chunk counts live in the tile-count scratch
   PArgs a;
   a.score = st.score;
   a.state = st.state;
@@ -1029,11 +1158,12 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   a.victims = d_victims;
   a.hist = ws.hist;
   a.sel = ws.sel;
-  a.cta_counts = ws.tile_counts;
+  a.chunk_counts = ws.tile_counts;
+  a.total_chunks = (uint32_t)total_chunks;
   a.status = ws.status;
-  a.per = ((st.n + G - 1) / G + 3) / 4 * 4;
-  if (a.per > kPMaxSlice) return cudaSuccess;  // slices beyond the bitmaps: the multi-launch selection runs
-  a.words = (uint32_t)((a.per + 31) / 32 + 3) / 4 * 4;
+  a.per = (total_chunks + G - 1) / G * kPChunk;   // the most entries a CTA holds: its chunks, whole
+  if (a.per > kPMaxSlice) return cudaSuccess;  // more than the bitmaps hold: the multi-launch selection runs
+  a.words = (uint32_t)(a.per / 32);
   // The hint's bracket typically holds 5-10 % of a slice's keys, but slices differ (blocks of one
   // history sit together), and a thread that runs out of slots sends its CTA the long way.  What this kernel does not take
   // of the shared memory stays with the L1, whose lines hold the loads in flight of the streaming

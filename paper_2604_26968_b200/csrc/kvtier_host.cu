@@ -227,7 +227,7 @@ void make_layout(const kv_pool_desc* d, const Derived& g, Layout* L) {
   L->part_counts = take(4 * 8);
   L->tile_counts = take((uint64_t)L->n_tiles * 8);
   L->tile_offsets = take((uint64_t)L->n_tiles * 8);
-  L->free_list = take(g.N * 4);
+  L->free_list = take((g.N + 4096) * 4);   // (the selection's note scratch is addressed by whole chunks of 4,096)
   for (int b = 0; b < kListBufs; ++b) L->slot_list[b] = take(d->max_promote * 4);
   for (int q = 0; q < g.n_parts; ++q) {
     const uint64_t R = d->part[q].ring_slots;
