@@ -431,17 +431,19 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
   uint32_t* const spill = a.spill;
   auto spill_at = [&](uint32_t r) { return spill + chunk_base(r >> 2) + (r & 3u) * kPThreads + t; };
   // body(v) for every note of the thread: the slots first, then the spilled ones, whose loads
-  // (L2) are issued eight at a time before the first of them is used
+  // (L2) are issued eight at a time before the first of them is used.  body may rewrite the
+  // list in place at positions up to the note it has been given.
   auto for_notes = [&](auto body) {
     const uint32_t in_slots = n_noted < a.slots ? n_noted : a.slots;
-    for (uint32_t i = 0; i < in_slots; ++i) body(s_note[i * kPThreads + t]);
-    for (uint32_t r = 0; a.slots + r < n_noted; r += 8u) {
+    for (uint32_t i = 0; i < in_slots; ++i) body(s_note[i * kPThreads + t]);   // (read before body may overwrite slot <= i)
+    const uint32_t n_all = n_noted;   // (body may shorten the list behind the note it is given)
+    for (uint32_t r = 0; a.slots + r < n_all; r += 8u) {
       uint32_t v[8];
 #pragma unroll
-      for (uint32_t u = 0; u < 8u; ++u) v[u] = (a.slots + r + u < n_noted) ? __ldcg(spill_at(r + u)) : 0xFFFFFFFFu;
+      for (uint32_t u = 0; u < 8u; ++u) v[u] = (a.slots + r + u < n_all) ? __ldcg(spill_at(r + u)) : 0xFFFFFFFFu;
 #pragma unroll
       for (uint32_t u = 0; u < 8u; ++u)
-        if (a.slots + r + u < n_noted) body(v[u]);
+        if (a.slots + r + u < n_all) body(v[u]);
     }
   };
   auto phase_a = [&](uint32_t c, const uint32_t key[4]) {
@@ -632,6 +634,9 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
         // notes; noted keys of earlier bins are below the final range: their bit joins s_bit_l
         const uint32_t bin_k = (base - base0) >> bshift;
         uint32_t p_bin = 0, p_cnt = 0;   // the thread's pending count for one key value
+        // the notes of bin_k are all that phase C looks at again: they move to the front of the
+        // thread's list (never ahead of the note being read) and the list shrinks to them
+        uint32_t n_kept = 0;
         for_notes([&](uint32_t v) {
           const uint32_t d = v & ((1u << 22) - 1u), b = d >> bshift;
           if (b < bin_k) {
@@ -645,8 +650,12 @@ __global__ void __launch_bounds__(kPThreads, 1) select_persistent_kernel(const P
               p_cnt = 0;
             }
             ++p_cnt;
+            if (n_kept < a.slots) s_note[n_kept * kPThreads + t] = v;
+            else *spill_at(n_kept - a.slots) = v;
+            ++n_kept;
           }
         });
+        n_noted = n_kept;
         // pending counts: one atomic per key value and warp
         for (;;) {
           const unsigned m = __ballot_sync(0xFFFFFFFFu, p_cnt != 0u);
