@@ -48,7 +48,7 @@ PACK_KERNEL_NAME = "move_tma_kernel<true> (pack)"
 # select_persistent_kernel<true>) from ncu, bytes per launch pair, keyed by pool number: captured
 # at the pool's full entry count with --tiny-entries (these kernels never touch block payload).
 # None = no capture of the kernels as they stand.
-NCU_SCORE_SELECT_TRAFFIC = {5: 547.2e6, 3: 423.7e6}
+NCU_SCORE_SELECT_TRAFFIC = {5: 547.0e6, 3: 420.9e6}
 
 
 def parse():
