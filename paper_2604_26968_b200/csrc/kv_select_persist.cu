@@ -3,19 +3,24 @@
 // The multi-launch selection in kv_select.cu spends most of its time between
 // kernels when the pool has a few million entries: ten dependent launches of
 // 3-10 us each.  Here one CTA per SM stays resident for the whole selection.
-// Each CTA owns a contiguous slice of the entries; the phases of the selection
-// are separated by grid-wide barriers instead of kernel boundaries:
+// CTA g owns the chunks g, g + G, g + 2G, ... of the pool (4,096 entries each): a
+// region of the pool that costs more than others -- many touched entries, many
+// keys near the threshold -- is spread over all CTAs, and the one barrier that
+// ends a phase waits for no overloaded CTA.  Bitmaps and notes index the CTA's
+// entries by (local chunk, offset).  The phases of the selection are separated by
+// grid-wide barriers instead of kernel boundaries:
 //
 //   A  every score becomes an order-preserving key (fused form: the entry pass
 //      itself produces it) and enters the first histogram.  With a hint -- tau of
 //      the previous selection -- the histogram covers a bracket of 2^18 .. 2^22 keys
-//      around it (2,048 bins; the width follows how far tau moved lately); the pass also leaves in shared memory a bitmap "key below the
+//      around it (2,048 bins; the width follows how far tau moved lately); the
+//      pass also leaves in shared memory a bitmap "key below the
 //      bracket", and every thread notes the keys it saw inside the bracket
 //      (typically 5-10 % of the slice) in a few private slots: no vote, no atomic.
 //   B  the remaining histograms of the radix select.  When rank k falls inside
 //      the bracket, ONE more histogram (the single keys of the bracket bin
-//      that holds rank k, at most 2^11) finishes it, and it is built from the noted keys alone:
-//      no second pass over the scores.  Otherwise (no hint, a miss, a thread that
+//      that holds rank k, at most 2^11) finishes it, and it is built from the
+//      noted keys alone: no second pass over the scores.  Otherwise (no hint, a miss, a thread that
 //      ran out of slots) the keys are re-read from the score array, which then
 //      sits mostly in L2, and the last histogram of that path leaves the bitmaps
 //      "key below the final range" and "key inside the final range".
@@ -24,9 +29,10 @@
 //      the keys inside the range (not even those when the CTA's own histogram
 //      shows that all of them equal tau: a tie, the usual case when few distinct
 //      scores exist).
-//   D  per-CTA counts = population counts of the two bitmaps; after the last
-//      barrier every CTA knows how many victims precede its slice and writes its
-//      own victims in ascending id order straight from the bitmaps.
+//   D  per-chunk counts = population counts of the two bitmaps, kept in a
+//      pool-wide table; after the last barrier every CTA sums the table's rows
+//      and knows how many victims precede each of its chunks; it writes its own
+//      victims, chunk by chunk in ascending id order, straight from the bitmaps.
 //
 // The grid barrier is a counter in global memory that every CTA increments and
 // then polls.  A cooperative launch guarantees that all CTAs are resident, so
@@ -34,8 +40,9 @@
 // KV_DEV_WAIT_EXPIRED and leaves (every other CTA then runs into the same limit).
 //
 // The same kernel also exists fused with the per-entry scoring pass (FUSED =
-// true): every CTA first updates the entries of its own slice (posterior, EMA,
-// score) and turns the fresh scores straight into keys -- a kernel boundary
+// true): every CTA first updates the entries of its own chunks (posterior, EMA,
+// score), their inputs streamed through shared-memory stages by asynchronous
+// copies, and turns the fresh scores straight into keys -- a kernel boundary
 // disappears.  The event reduction stays a launch of its own ahead of it: its
 // scattered gathers and atomics ran 2.5x slower inside this kernel when that was
 // tried, and a grid barrier costs about what the launch boundary does.
