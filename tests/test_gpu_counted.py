@@ -63,3 +63,30 @@ def test_counts_that_do_not_add_up_are_refused_before_anything_changes():
     assert o.demote(v) == 0
     ls.compare_state("demotion", scores=False)
     ls.close()
+
+
+def test_counts_over_several_rows_of_chunks():
+    """1.2 M entries: every CTA of the persistent selection holds two chunks, the victims per
+    partition come from the pool-wide chunk table (metadata only: no block bytes move)."""
+    from lockstep import Lockstep
+    ls = Lockstep(_pool5(scale=1 / 16), payload=False, batch_bytes=8 << 20, fused=True, counted=True)
+    for e in range(4):
+        ls.epoch(e)
+    assert ls.gpu.pool.kv_get_stats()["host_waits"] == 0
+    ls.close()
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_partition_boundaries_on_chunk_boundaries(fused):
+    """Partitions of exactly 4,096 and 8,192 entries: the boundaries between them coincide with
+    the chunks of the persistent selection (no chunk is split between two partitions)."""
+    from lockstep import Lockstep
+    parts = [W.gqa(2, 8, 4, 8, 4, 512, 3000, "entry"),      # 2 * 512 * 4 = 4,096 entries
+             W.mha(2, 8, 8, 4, 512, 6000, "entry"),         # 2 * 512 * 8 = 8,192
+             W.mla(3, 24, 8, 2, 333, 1000, "entry")]        # 999, ragged
+    w = W.Workload("aligned_parts", parts, 0.2, 0.1, seed=5, promote_style="recent", epochs=8)
+    ls = Lockstep(w, payload=False, batch_bytes=1 << 20, fused=fused, counted=True)
+    for e in range(6):
+        ls.epoch(e)
+    assert ls.gpu.pool.kv_get_stats()["host_waits"] == 0
+    ls.close()
