@@ -184,3 +184,35 @@ def test_prefetch_errors_and_edges():
             pf.lists(pos0, 1)
             pf.lists(pos0, -1)
     ls.close()
+
+
+def test_prefetch_list_at_the_launch_limit():
+    """1.3 M candidates (2,048 position-blocks x 80 layers x 8 heads, the sequence's table tiled
+    from the partition's 84 blocks): the list kernels run their full 1,024 chunks of more than
+    one tile each; windows from 1 block to the whole table, both directions, a cut list."""
+    from lockstep import Lockstep
+    w = W.config(5, scale=1 / 128)
+    for p in w.parts:
+        p.ring_slots = w.k + 64
+    ls = Lockstep(w, payload=False, batch_bytes=4 << 20, fused=True)
+    pf = Prefetch(ls, 1)
+    state = {}
+
+    def before(ls_):
+        t = pf.build_table(pf.NB, 7)
+        state["table"] = np.ascontiguousarray(np.tile(t, (25, 1, 1))[:2048])
+
+    ls.epoch(0, before_demote=before)
+    ls.epoch(1)
+    pf.table = state["table"]
+    r = np.random.default_rng(9)
+    span = (r.random(pf.L) * 16 * 2048).astype(np.float32)
+    span[0], span[-1] = 1.0, 16.0 * 4096
+    pf.set(0.0, 4096)
+    pf.update(span, 0.0)
+    for pos0, direction in ((0, 1), (2047, -1), (1000, 1), (1000, -1)):
+        lst, n = pf.lists(pos0, direction)
+        assert n > 10000
+    pf.lists(5, 1, max_out=1000)
+    assert ls.gpu.pool.kv_device_status() == 0
+    ls.close()
