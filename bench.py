@@ -523,6 +523,7 @@ def main():
                 flush.fill_((e + i) & 0xFF)
 
     tot = {"ss": 0.0, "dem": 0.0, "pro": 0.0, "all": 0.0, "events": 0, "promoted_bytes": 0}
+    ss_steps = []   # score + select of every timed step of this rank, us
     sampler = ClockSampler(local)
     epoch = 0
     launches0 = 0
@@ -547,6 +548,7 @@ def main():
         launches_step = pool.kv_get_stats()["kernel_launches"] - launches_before
         if timed:
             tot["ss"] += ev[0].elapsed_time(ev[1])
+            ss_steps.append(round(1e3 * ev[0].elapsed_time(ev[1]), 1))
             tot["dem"] += ev[1].elapsed_time(ev[2])
             tot["pro"] += ev[4].elapsed_time(ev[5])
             tot["all"] += max(ev[0].elapsed_time(ev[2]), ev[0].elapsed_time(ev[3]), ev[0].elapsed_time(ev[5]))
@@ -687,6 +689,7 @@ def main():
                          "fresh blocks admitted between steps)"},
         "phases": {
             "score_select_ms": ss_ms,
+            "score_select_us_per_step": ss_steps,
             "score_select_effective_gbs": ss_gbs,
             "demote_ms": dem_ms, "demote_gbs": demoted_per_step / (dem_ms * 1e-3) / 1e9,
             "promote_ms": pro_ms, "promote_gbs": promoted_per_step / max(pro_ms * 1e-3, 1e-12) / 1e9,
@@ -707,6 +710,7 @@ def main():
                      "algorithmic_bytes_per_launch": ss_bytes,
                      "algorithmic_bytes": "39 B/entry (30 scoring + 9 selection) + 5 B/event + 4 B/victim",
                      "launch_us": 1e3 * ss_ms,
+                     "launch_us_median": float(np.median(ss_steps)) if ss_steps else None,
                      "selection_hints": {"selections": sel1["selections"] - sel0["selections"],
                                          "hits": sel1["hint_hits"] - sel0["hint_hits"],
                                          "misses": sel1["hint_misses"] - sel0["hint_misses"],
