@@ -383,6 +383,25 @@ int32_t kv_prefetch_list(kv_pool* pool, int32_t q, const uint32_t* d_table, uint
  * even near 0.8 MB per run); 0 = always per-run transfers. */
 int32_t kv_set_gather_threshold(kv_pool* pool, uint64_t run_bytes);
 
+/* L2 residency of a state array (off by default).  The event reduction scatters atomics
+ * over the touch counts and gathers pair bytes, and the entry pass then streams both
+ * arrays once more; between the two, and from one epoch to the next, the gigabytes that
+ * the block movement sends through the L2 evict them.  With a budget > 0 the scoring
+ * kernels (event reduction, entry pass, fused selection) are launched with an access-policy
+ * window that keeps ONE array in the persisting part of the L2: the touch counts (4 B per
+ * entry) when they fit the budget whole, else the pair bytes (1 B per entry), a fraction
+ * of them if even those do not fit.  Measured on a B200 (126 MB L2): 47 MB of touch counts
+ * resident take 20 us off a 150 us pass; 75 MB resident leave too little L2 for the
+ * streaming entry pass and cost more than they save, hence the rule.  A budget of 3/8 of
+ * the L2 is a good choice.  Results are bit for bit the same.
+ * The call sets the persisting-L2 set-aside of the CUDA context (cudaLimitPersistingL2CacheSize)
+ * to what it uses, a setting of the calling process's context, shared by everything in it;
+ * budget_bytes == 0 switches the window off and sets the set-aside to 0.  Nothing is
+ * enqueued; it takes effect for calls made after it.  kv_pool_destroy of a pool with a window
+ * turns the context's persisting lines back into ordinary ones (the set-aside stays as it
+ * is).  KV_ERR_UNIMPLEMENTED on devices without a persisting L2. */
+int32_t kv_set_l2_residency(kv_pool* pool, uint64_t budget_bytes);
+
 /* Lazy decay of promoted entries (off by default).  The head-granular eviction
  * section updates importance on every step for blocks in HBM; the paper does not
  * say what a block's importance is when it returns from a lower tier.  Off, the

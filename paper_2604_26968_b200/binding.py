@@ -89,7 +89,7 @@ EXPORTS = ("kv_size_bytes", "kv_infer_variant", "kv_entry_bytes", "kv_workspace_
            "kv_epoch_update", "kv_set_policy", "kv_set_lazy_decay", "kv_hash_entries", "kv_dedup_table_slots", "kv_dedup_digests", "kv_set_confidence_blend", "kv_reuse_estimate", "kv_head_importance_update", "kv_set_head_multipliers", "kv_head_importance", "kv_head_weights", "kv_prefetch_window_update", "kv_set_prefetch_window", "kv_prefetch_span", "kv_prefetch_window", "kv_prefetch_list", "kv_select_victims", "kv_select_victim_blocks", "kv_select_victims_static", "kv_demote",
            "kv_promote", "kv_set_deferred_packing", "kv_flush", "kv_max_batch_bytes", "kv_admit", "kv_get_stats", "kv_ring_query",
            "kv_last_demote_counts", "kv_device_status", "kv_timing_enable", "kv_timing_read",
-           "kv_set_select_variant", "kv_selection_stats", "kv_demote_counted", "kv_victim_counts", "kv_set_gather_threshold", "kv_last_cuda_error", "kv_status_string",
+           "kv_set_select_variant", "kv_selection_stats", "kv_demote_counted", "kv_victim_counts", "kv_set_gather_threshold", "kv_set_l2_residency", "kv_last_cuda_error", "kv_status_string",
            "kv_version")
 
 _lib = None
@@ -149,6 +149,8 @@ def load():
     L.kv_head_importance.argtypes = [vp, i32]
     L.kv_head_weights.restype = vp
     L.kv_head_weights.argtypes = [vp, i32]
+    L.kv_set_l2_residency.restype = i32
+    L.kv_set_l2_residency.argtypes = [vp, C.c_uint64]
     L.kv_prefetch_window_update.restype = i32
     L.kv_prefetch_window_update.argtypes = [vp, i32, vp, C.c_float, vp]
     L.kv_set_prefetch_window.restype = i32
@@ -454,6 +456,9 @@ class Pool:
                                          d_out_slots.data_ptr() if d_out_slots is not None else None, int(max_out),
                                          d_out_count.data_ptr() if d_out_count is not None else None,
                                          _stream_ptr(self.compute))
+
+    def kv_set_l2_residency(self, budget_bytes):
+        return self.lib.kv_set_l2_residency(self._h, int(budget_bytes))
 
     def kv_select_victims(self, k, d_victims):
         return self.lib.kv_select_victims(self._h, int(k), d_victims.data_ptr() if k else None,

@@ -27,10 +27,16 @@ cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit,
   if (blocks == 0) blocks = 1;
   const uint64_t cap = (uint64_t)sm_count() * 4;  // measured: 4 blocks per SM beat 8 and 2
   if (blocks > cap) blocks = cap;
-  event_reduce_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(ev_entry, ev_hit, n_events, st.pair, st.touch,
-                                                            st.n, ws.delta, ws.status);
+  const uint8_t* pair = st.pair;
+  uint32_t* touch = st.touch;
+  uint64_t n = st.n;
+  unsigned long long* delta = ws.delta;
+  uint32_t* status = ws.status;
+  void* args[] = {&ev_entry, &ev_hit, &n_events, &pair, &touch, &n, &delta, &status};
+  const cudaError_t e = launch_scoring_kernel((const void*)event_reduce_kernel, dim3((unsigned)blocks),
+                                              dim3(kThreads), args, 0, s, false, ws);
   count_launches(1);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // ---- entry pass ----------------------------------------------------------------------
@@ -103,9 +109,14 @@ cudaError_t launch_entry_update(const EntryState& st, uint64_t* hits, uint64_t* 
   if (blocks > cap) blocks = cap;
   const Predictor pd{hits,       misses,    P,          alpha0, beta0, ws.delta, &ws.sel->update_ticket,
                      opt.policy, opt.kappa, opt.window, ws.blend};
-  entry_update_kernel<<<(unsigned)blocks, kThreads, 0, s>>>(st, pd, hw, epoch);
+  EntryState st_arg = st;
+  Predictor pd_arg = pd;
+  HeadWeights hw_arg = hw;
+  void* args[] = {&st_arg, &pd_arg, &hw_arg, &epoch};
+  const cudaError_t e = launch_scoring_kernel((const void*)entry_update_kernel, dim3((unsigned)blocks),
+                                              dim3(kThreads), args, 0, s, false, ws);
   count_launches(1);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace kvt

@@ -1210,7 +1210,7 @@ cudaError_t launch_select_persistent(const EntryState& st, uint64_t k, uint32_t*
   const bool plain = fs && fs->opt.policy == 0 && fs->hw.on == 0;
   void* fn = !fs ? (void*)select_persistent_kernel<false, false>
                  : plain ? (void*)select_persistent_kernel<true, true> : (void*)select_persistent_kernel<true, false>;
-  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(G), dim3(kPThreads), args, smem, s);
+  cudaError_t e = launch_scoring_kernel(fn, dim3(G), dim3(kPThreads), args, smem, s, true, ws);
   if (e != cudaSuccess) return e;
   count_launches(1);
   *used = true;

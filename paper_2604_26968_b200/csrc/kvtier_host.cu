@@ -676,6 +676,10 @@ int32_t kv_pool_destroy(kv_pool* p) {
     for (cudaEvent_t* ev : evs) cudaEventDestroy(*ev);
   }
   for (auto& t : p->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+  if (p->ws.l2_bytes) {   // the pool's lines in the persisting part of the L2 become ordinary lines again
+    (void)cudaCtxResetPersistingL2Cache();
+    (void)cudaGetLastError();
+  }
   delete p;
   return KV_OK;
 }
@@ -1211,6 +1215,41 @@ int32_t kv_flush(kv_pool* p) {
 int32_t kv_set_gather_threshold(kv_pool* p, uint64_t run_bytes) {
   if (!p) return KV_ERR_INVALID_ARG;
   p->gather_run_bytes = run_bytes;
+  return KV_OK;
+}
+
+int32_t kv_set_l2_residency(kv_pool* p, uint64_t budget_bytes) {
+  if (!p) return KV_ERR_INVALID_ARG;
+  int dev = 0, max_persist = 0, max_window = 0;
+  KV_CUDA(p, cudaGetDevice(&dev));
+  KV_CUDA(p, cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev));
+  KV_CUDA(p, cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, dev));
+  if (budget_bytes == 0) {
+    if (p->ws.l2_bytes) {
+      p->ws.l2_base = nullptr;
+      p->ws.l2_bytes = 0;
+      p->ws.l2_ratio = 0.0f;
+      KV_CUDA(p, cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, 0));
+    }
+    return KV_OK;
+  }
+  if (max_persist <= 0 || max_window <= 0) return KV_ERR_UNIMPLEMENTED;
+  uint64_t budget = budget_bytes < (uint64_t)max_persist ? budget_bytes : (uint64_t)max_persist;
+  const uint64_t touch_bytes = p->st.n * 4, pair_bytes = p->st.n;
+  const void* base;
+  uint64_t bytes, set_aside;
+  if (touch_bytes <= budget && touch_bytes <= (uint64_t)max_window) {   // the touch counts, whole
+    base = p->st.touch;
+    bytes = set_aside = touch_bytes;
+  } else {                                                               // the pair bytes, as far as they fit
+    base = p->st.pair;
+    bytes = pair_bytes < (uint64_t)max_window ? pair_bytes : (uint64_t)max_window;
+    set_aside = bytes < budget ? bytes : budget;
+  }
+  KV_CUDA(p, cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, (size_t)set_aside));
+  p->ws.l2_base = base;
+  p->ws.l2_bytes = (size_t)bytes;
+  p->ws.l2_ratio = set_aside >= bytes ? 1.0f : (float)((double)set_aside / (double)bytes);
   return KV_OK;
 }
 

@@ -182,7 +182,42 @@ struct Workspace {
   uint32_t* slot_list[8];      // [max_promote] promote lists (ring slots), used in turn
   unsigned long long* part_counts;  // [4] victims per partition
   uint32_t n_tiles;
+  // One of the state arrays kept in the persisting part of the L2 (kv_set_l2_residency):
+  // the scoring kernels are launched with this access-policy window.  bytes == 0: none.
+  const void* l2_base = nullptr;
+  size_t l2_bytes = 0;
+  float l2_ratio = 0.0f;
 };
+
+// Launches fn (kernel taking the arguments in args) with the workspace's L2 window, if it has
+// one, as a launch attribute; cooperative launches carry that attribute too.
+inline cudaError_t launch_scoring_kernel(const void* fn, dim3 grid, dim3 block, void** args, size_t smem,
+                                         cudaStream_t s, bool cooperative, const Workspace& ws) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  if (cooperative) {
+    attr[n].id = cudaLaunchAttributeCooperative;
+    attr[n].val.cooperative = 1;
+    ++n;
+  }
+  if (ws.l2_bytes) {
+    attr[n].id = cudaLaunchAttributeAccessPolicyWindow;
+    attr[n].val.accessPolicyWindow.base_ptr = const_cast<void*>(ws.l2_base);
+    attr[n].val.accessPolicyWindow.num_bytes = ws.l2_bytes;
+    attr[n].val.accessPolicyWindow.hitRatio = ws.l2_ratio;
+    attr[n].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+    attr[n].val.accessPolicyWindow.missProp = cudaAccessPropertyNormal;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelExC(&cfg, fn, args);
+}
 
 // ---- kv_score.cu ----
 cudaError_t launch_event_reduce(const uint32_t* ev_entry, const uint8_t* ev_hit, uint64_t n_events,

@@ -37,7 +37,7 @@ def oracle_admit(w, pool, epoch, key=None):
 class Lockstep:
     def __init__(self, w, payload=True, batch_bytes=1 << 20, staging_bytes=None, host_meta=True,
                  policy=0, blend=None, deferred=False, fused=False, heads=None, lazy=False,
-                 split_promote=1, counted=False, select_variant=1):
+                 split_promote=1, counted=False, select_variant=1, l2_budget=None):
         self.w = w
         self.payload = payload
         self.gpu = EpochRunner(w, batch_bytes=batch_bytes, staging_bytes=staging_bytes,
@@ -53,6 +53,8 @@ class Lockstep:
         if deferred:
             assert self.gpu.pool.kv_set_deferred_packing(True) == 0
         assert self.gpu.pool.kv_set_select_variant(select_variant) == 0
+        if l2_budget is not None:   # one state array kept in the persisting part of the L2
+            assert self.gpu.pool.kv_set_l2_residency(l2_budget) == 0
         # room for any k a test may ask for
         self.gpu.victims = self.gpu.torch.empty(max(w.N, 4), dtype=self.gpu.torch.int32,
                                                 device=self.gpu.pool.device)
